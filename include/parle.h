@@ -1,0 +1,174 @@
+/*
+ * parle.h -- C ABI of the single-GPU Parle round (arXiv 1707.00424, Section 3).
+ *
+ * One Parle round over n replicas of an MLP:
+ *     reset   y^a <- x^a, z^a <- x^a                                  (Section 3, text after Eq. parle)
+ *     L times y^a <- y^a - eta' [ grad f(y^a) + (y^a - x^a)/gamma ]   (Eq. parle_y)
+ *             z^a <- alpha z^a + (1 - alpha) y^a                      (Eq. parle_z)
+ *     once    x^a <- x^a - eta (x^a - z^a) - (eta/rho)(x^a - xbar)    (Eq. parle_xa)
+ *             xbar <- (1/n) sum_a x^a                                  (Eq. parle_x with eta'' = rho/n, Section 3.1)
+ * grad f is the minibatch gradient of the mean softmax cross-entropy of a
+ * ReLU MLP (Section 1.1 / 2.1).
+ *
+ * General rules
+ *   - Every function returns PARLE_OK (0) or a negative PARLE_E* code; nothing
+ *     throws, aborts or synchronises the host.  All device work is enqueued on
+ *     the stream given to parle_bind(); results are valid once the caller has
+ *     synchronised that stream.
+ *   - The library allocates no device memory.  All state and scratch buffers
+ *     are device pointers owned by the caller (parle_buffers).  The context
+ *     itself is host memory owned by the library (freed by parle_destroy).
+ *   - Pointers marked "dev" are device pointers, "host" are host pointers.
+ *   - Parameter vectors are fp32, laid out [n, stride]: replica a starts at
+ *     element a*stride.  Inside one replica the packing is
+ *         [ W_1 | b_1 | W_2 | b_2 | ... ],   W_l row-major [d_l, d_{l-1}],
+ *     each segment starting at a multiple of 32 elements (128 bytes); the
+ *     padding elements must be zero in x and stay zero.  parle_layer_offset()
+ *     reports the offsets.  With n_layers == 0 the vector has no structure
+ *     (dims[0] elements): only the update entry points can be used.
+ */
+#ifndef PARLE_H
+#define PARLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PARLE_OK            0
+#define PARLE_EINVAL       -1   /* bad argument (n, dims, batch, alpha not in [0,1), gamma/rho/eta <= 0, NULL) */
+#define PARLE_ENOTBOUND    -2   /* parle_bind() has not been called */
+#define PARLE_EALIGN       -3   /* a buffer is not 128-byte aligned */
+#define PARLE_ECUDA        -4   /* a CUDA call failed; parle_last_cuda_error() has the code */
+#define PARLE_ESTATE       -5   /* call out of order (e.g. inner step before parle_round_begin) */
+#define PARLE_EWORKSPACE   -6   /* workspace smaller than parle_workspace_bytes() */
+#define PARLE_EUNSUPPORTED -7   /* shape not supported by the requested GEMM path */
+
+/* bits of the device status word, see parle_status() */
+#define PARLE_FLAG_NONFINITE   1   /* an update kernel produced a NaN or Inf */
+#define PARLE_FLAG_WAIT_LIMIT  2   /* a bounded wait inside a GEMM pipeline gave up */
+#define PARLE_FLAG_BAD_LABEL   4   /* a label outside [0, d_last) was seen (treated as no target) */
+
+#define PARLE_GEMM_FP32 0   /* fp32 operands, fp32 FMA accumulation */
+#define PARLE_GEMM_BF16 1   /* bf16 operands on the tcgen05 tensor cores, fp32 accumulation;
+                               needs batch % 8 == 0 and every d_l % 8 == 0 except the last */
+
+#define PARLE_MAX_LAYERS 16
+#define PARLE_MAX_REPLICAS 64
+
+typedef struct parle_ctx parle_ctx;      /* opaque; host memory owned by the library */
+
+typedef struct {
+    int n_layers;        /* number of affine layers (0: flat vector mode)                 */
+    const int *dims;     /* host, n_layers+1 entries d_0 ... d_last (copied by parle_init) */
+    int batch;           /* minibatch size B per replica (ignored when n_layers == 0)      */
+    int gemm_dtype;      /* PARLE_GEMM_FP32 or PARLE_GEMM_BF16                             */
+} parle_model;
+
+typedef struct {
+    float *x;            /* dev [n, stride]  replicas x^a (in/out)                    */
+    float *y;            /* dev [n, stride]  inner iterates y^a                       */
+    float *z;            /* dev [n, stride]  exponential averages z^a                 */
+    float *grad;         /* dev [n, stride]  minibatch gradient, same packing         */
+    float *xbar;         /* dev [stride]     reference variable (in/out)              */
+    void  *workspace;    /* dev, >= parle_workspace_bytes(); contents are scratch     */
+    size_t workspace_bytes;
+} parle_buffers;
+
+/* Create a context for n replicas (Section 3: a <= n) of `model`, with the
+ * scalars of Eq. (parle).  gamma and rho may be +INFINITY, which switches the
+ * corresponding coupling off (1/gamma = 0 or 1/rho = 0 exactly).
+ * EINVAL: out == NULL, n outside [1, PARLE_MAX_REPLICAS], bad dims/batch,
+ * alpha outside [0,1), gamma <= 0, rho <= 0, eta <= 0, eta_prime <= 0.
+ * EUNSUPPORTED: PARLE_GEMM_BF16 with shapes it cannot take. */
+int parle_init(parle_ctx **out, int n, const parle_model *model,
+               double gamma, double rho, double alpha, double eta, double eta_prime);
+
+/* Free the context (host memory only; caller buffers are untouched). NULL ok. */
+void parle_destroy(parle_ctx *ctx);
+
+/* Number of real parameters P of one replica, and the padded length `stride`
+ * (>= P, multiple of 32) of one replica's vector.  0 if ctx is NULL. */
+size_t parle_param_count(const parle_ctx *ctx);
+size_t parle_stride(const parle_ctx *ctx);
+
+/* Bytes of scratch the caller must provide in parle_buffers.workspace. */
+size_t parle_workspace_bytes(const parle_ctx *ctx);
+
+/* Element offsets of W_layer and b_layer inside one replica's vector
+ * (layer in [0, n_layers)).  EINVAL for a bad layer or NULL output. */
+int parle_layer_offset(const parle_ctx *ctx, int layer, size_t *w_off, size_t *b_off);
+
+/* Attach the caller's device buffers and CUDA stream (a cudaStream_t passed as
+ * void*, NULL = default stream).  The context keeps the pointers, not copies.
+ * Must be called with the buffers' device current.  EALIGN if a pointer is not
+ * 128-byte aligned, EWORKSPACE if the workspace is too small, EINVAL on NULL.
+ * After binding, x and xbar hold the caller's initial state; x must not be
+ * modified behind the library's back without binding again. */
+int parle_bind(parle_ctx *ctx, const parle_buffers *buffers, void *cuda_stream);
+
+/* Start a round: y^a <- x^a and z^a <- x^a (text after Eq. parle).  The copy is
+ * folded into the first inner step of the round, which reads x^a in place of
+ * y^a and z^a; y and z hold the round's values from that step on. */
+int parle_round_begin(parle_ctx *ctx);
+
+/* One inner step for all replicas: forward/backward of the MLP on each
+ * replica's own minibatch at y^a (Section 2.1), then Eq. (parle_y), (parle_z).
+ *   inputs  dev [n, B, d_0] fp32, labels dev [n, B] int32 in [0, d_last)
+ *   loss_out dev [n] fp32 or NULL: mean cross-entropy of each replica's batch
+ * ESTATE if no round is open; EINVAL in flat vector mode. */
+int parle_inner_step(parle_ctx *ctx, const float *inputs, const int32_t *labels,
+                     float *loss_out);
+
+/* Same step with host buffers: inputs/labels are copied to the device and the
+ * losses copied back on the bound stream (asynchronously if the host memory is
+ * pinned).  loss_out_host may be NULL. */
+int parle_inner_step_host(parle_ctx *ctx, const float *inputs_host,
+                          const int32_t *labels_host, float *loss_out_host);
+
+/* Eq. (parle_y), (parle_z) only, from a caller-supplied gradient
+ * grad dev [n, stride] (may be the bound grad buffer).  Reads grad, y, x, z
+ * once and writes y, z once. */
+int parle_inner_update(parle_ctx *ctx, const float *grad);
+
+/* Eq. (parle_xa) for every replica, using the xbar left by the previous mean,
+ * and -- fused in the same pass -- the new replica mean written to xbar
+ * (Eq. parle_x with eta'' = rho/n).  Closes the round.  ESTATE if the round
+ * had no inner step. */
+int parle_outer_step(parle_ctx *ctx);
+
+/* xbar <- (1/n) sum_a x^a (Eq. parle_x, Section 3.1).  After parle_outer_step
+ * this recomputes the same values; use it after writing x directly. */
+int parle_mean(parle_ctx *ctx);
+
+/* A whole round in one call: parle_round_begin, L inner steps on
+ * inputs dev [L, n, B, d_0] / labels dev [L, n, B], parle_outer_step.
+ * loss_out dev [L, n] or NULL. */
+int parle_round(parle_ctx *ctx, int L, const float *inputs, const int32_t *labels,
+                float *loss_out);
+
+/* Change gamma, rho (Eq. scoping changes them between rounds) or the step
+ * sizes eta, eta' between calls.  +INFINITY allowed for gamma and rho. */
+int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);
+int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
+
+/* Non-blocking read of the device status word (PARLE_FLAG_* bits) set by the
+ * kernels launched so far; clears nothing.  parle_clear_status resets it. */
+int parle_status(parle_ctx *ctx, int *device_flags);
+int parle_clear_status(parle_ctx *ctx);
+
+/* Kernels launched by this context since creation (for accounting). */
+long long parle_launch_count(const parle_ctx *ctx);
+
+/* Last CUDA error code recorded by a call that returned PARLE_ECUDA. */
+int parle_last_cuda_error(const parle_ctx *ctx);
+
+/* Static string for a PARLE_* code. */
+const char *parle_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PARLE_H */

@@ -1,0 +1,202 @@
+"""ctypes binding of libparle.so: argument marshalling only.
+
+PyTorch appears here for device memory and streams alone; there is no CPU or
+PyTorch fallback -- if the CUDA library cannot be loaded every call fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+from typing import Optional, Sequence
+
+GEMM_FP32, GEMM_BF16 = 0, 1
+FLAG_NONFINITE, FLAG_WAIT_LIMIT, FLAG_BAD_LABEL = 1, 2, 4
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB: Optional[C.CDLL] = None
+
+
+class ParleError(RuntimeError):
+    def __init__(self, code: int, what: str, cuda: int = 0):
+        self.code = code
+        msg = f"{what}: {lib().parle_strerror(code).decode()} ({code})"
+        if cuda:
+            msg += f" [CUDA error {cuda}]"
+        super().__init__(msg)
+
+
+class _Model(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("dims", C.POINTER(C.c_int)), ("batch", C.c_int), ("gemm_dtype", C.c_int)]
+
+
+class _Buffers(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("y", C.c_void_p), ("z", C.c_void_p), ("grad", C.c_void_p),
+                ("xbar", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libparle.so")
+
+
+def lib() -> C.CDLL:
+    """Load the CUDA library (building it first if the sources are newer)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        from .build import build
+        build()
+    L = C.CDLL(path)
+    vp, ci, cd, sz = C.c_void_p, C.c_int, C.c_double, C.c_size_t
+    sig = {
+        "parle_init": (ci, [C.POINTER(vp), ci, C.POINTER(_Model), cd, cd, cd, cd, cd]),
+        "parle_destroy": (None, [vp]),
+        "parle_param_count": (sz, [vp]),
+        "parle_stride": (sz, [vp]),
+        "parle_workspace_bytes": (sz, [vp]),
+        "parle_layer_offset": (ci, [vp, ci, C.POINTER(sz), C.POINTER(sz)]),
+        "parle_bind": (ci, [vp, C.POINTER(_Buffers), vp]),
+        "parle_round_begin": (ci, [vp]),
+        "parle_inner_step": (ci, [vp, vp, vp, vp]),
+        "parle_inner_step_host": (ci, [vp, vp, vp, vp]),
+        "parle_inner_update": (ci, [vp, vp]),
+        "parle_outer_step": (ci, [vp]),
+        "parle_mean": (ci, [vp]),
+        "parle_round": (ci, [vp, ci, vp, vp, vp]),
+        "parle_set_coupling": (ci, [vp, cd, cd]),
+        "parle_set_lr": (ci, [vp, cd, cd]),
+        "parle_status": (ci, [vp, C.POINTER(ci)]),
+        "parle_clear_status": (ci, [vp]),
+        "parle_launch_count": (C.c_longlong, [vp]),
+        "parle_last_cuda_error": (ci, [vp]),
+        "parle_strerror": (C.c_char_p, [ci]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = res, args
+    _LIB = L
+    return L
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor / raw int / None."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+class Parle:
+    """One context = n replicas of one MLP with the scalars of Eq. (parle).
+
+    Mirrors the C entry points one to one (same names without the prefix).
+    `alloc()` makes the caller-owned state with torch and binds it.
+    """
+
+    def __init__(self, n: int, dims: Sequence[int], batch: int = 0, gemm_dtype: int = GEMM_FP32, *,
+                 gamma: float = 1.0, rho: float = 1.0, alpha: float = 0.75, eta: float = 0.1,
+                 eta_prime: float = 0.1):
+        self._L = lib()
+        self.n, self.dims, self.batch, self.gemm_dtype = n, tuple(int(d) for d in dims), batch, gemm_dtype
+        arr = (C.c_int * len(self.dims))(*self.dims)
+        model = _Model(len(self.dims) - 1, arr, batch, gemm_dtype)
+        h = C.c_void_p()
+        rc = self._L.parle_init(C.byref(h), n, C.byref(model), gamma, rho, alpha, eta, eta_prime)
+        if rc != 0:
+            raise ParleError(rc, "parle_init")
+        self._h = h
+        self.param_count = self._L.parle_param_count(h)
+        self.stride = self._L.parle_stride(h)
+        self.workspace_bytes = self._L.parle_workspace_bytes(h)
+        self.x = self.y = self.z = self.grad = self.xbar = self.workspace = None
+
+    # -- life cycle -------------------------------------------------------
+    def close(self):
+        if getattr(self, "_h", None):
+            self._L.parle_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, what: str):
+        if rc != 0:
+            raise ParleError(rc, what, self._L.parle_last_cuda_error(self._h))
+
+    # -- layout -----------------------------------------------------------
+    def layer_offset(self, layer: int):
+        w, b = C.c_size_t(), C.c_size_t()
+        self._check(self._L.parle_layer_offset(self._h, layer, C.byref(w), C.byref(b)), "parle_layer_offset")
+        return w.value, b.value
+
+    # -- memory -----------------------------------------------------------
+    def alloc(self, device="cuda:0", stream=None):
+        """Allocate x, y, z, grad, xbar and the workspace with torch and bind them."""
+        import torch
+        dev = torch.device(device)
+        with torch.cuda.device(dev):
+            mk = lambda *s: torch.zeros(*s, dtype=torch.float32, device=dev)
+            self.x, self.y, self.z, self.grad = (mk(self.n, self.stride) for _ in range(4))
+            self.xbar = mk(self.stride)
+            self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=dev)
+            self.bind(self.x, self.y, self.z, self.grad, self.xbar, self.workspace, stream)
+        return self
+
+    def bind(self, x, y, z, grad, xbar, workspace, stream=None):
+        import torch
+        if stream is None:
+            stream = torch.cuda.current_stream(x.device)
+        self._stream = stream
+        b = _Buffers(_ptr(x), _ptr(y), _ptr(z), _ptr(grad), _ptr(xbar), _ptr(workspace),
+                     workspace.numel() * workspace.element_size())
+        sp = stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream or 0)
+        with torch.cuda.device(x.device):
+            self._check(self._L.parle_bind(self._h, C.byref(b), C.c_void_p(sp)), "parle_bind")
+        self.x, self.y, self.z, self.grad, self.xbar, self.workspace = x, y, z, grad, xbar, workspace
+
+    # -- the round --------------------------------------------------------
+    def round_begin(self):
+        self._check(self._L.parle_round_begin(self._h), "parle_round_begin")
+
+    def inner_step(self, inputs, labels, loss_out=None):
+        self._check(self._L.parle_inner_step(self._h, _ptr(inputs), _ptr(labels), _ptr(loss_out)), "parle_inner_step")
+
+    def inner_step_host(self, inputs_host, labels_host, loss_out_host=None):
+        self._check(self._L.parle_inner_step_host(self._h, _ptr(inputs_host), _ptr(labels_host), _ptr(loss_out_host)),
+                    "parle_inner_step_host")
+
+    def inner_update(self, grad):
+        self._check(self._L.parle_inner_update(self._h, _ptr(grad)), "parle_inner_update")
+
+    def outer_step(self):
+        self._check(self._L.parle_outer_step(self._h), "parle_outer_step")
+
+    def mean(self):
+        self._check(self._L.parle_mean(self._h), "parle_mean")
+
+    def round(self, L: int, inputs, labels, loss_out=None):
+        self._check(self._L.parle_round(self._h, L, _ptr(inputs), _ptr(labels), _ptr(loss_out)), "parle_round")
+
+    def set_coupling(self, gamma: float, rho: float):
+        self._check(self._L.parle_set_coupling(self._h, gamma, rho), "parle_set_coupling")
+
+    def set_lr(self, eta: float, eta_prime: float):
+        self._check(self._L.parle_set_lr(self._h, eta, eta_prime), "parle_set_lr")
+
+    def status(self) -> int:
+        f = C.c_int()
+        self._check(self._L.parle_status(self._h, C.byref(f)), "parle_status")
+        return f.value
+
+    def clear_status(self):
+        self._check(self._L.parle_clear_status(self._h), "parle_clear_status")
+
+    @property
+    def launch_count(self) -> int:
+        return self._L.parle_launch_count(self._h)

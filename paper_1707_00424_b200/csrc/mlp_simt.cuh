@@ -1,0 +1,195 @@
+// fp32 path of the replica-batched MLP forward/backward (Section 1.1 / 2.1:
+// minibatch gradient of the mean cross-entropy): a strided, replica-grouped
+// SGEMM on the FMA pipes with fused bias / ReLU / ReLU-mask epilogues, the
+// softmax cross-entropy backward, and the bias gradient (column sums).
+#pragma once
+
+#include "common.cuh"
+
+namespace parle {
+
+enum SimtEpilogue { EPI_PLAIN = 0, EPI_BIAS = 1, EPI_BIAS_RELU = 2, EPI_MASK = 3 };
+
+struct SimtGemmArgs {
+    const float *A, *B;
+    float *C;
+    long long a_gs, b_gs, c_gs;        // per-replica strides (elements)
+    int M, N, K;
+    long long a_ms, a_ks;              // A(m,k) = A[m*a_ms + k*a_ks]
+    long long b_ks, b_ns;              // B(k,n) = B[k*b_ks + n*b_ns]
+    int ldc;
+    const float *bias; long long bias_gs;          // EPI_BIAS*: bias[n]
+    const float *mask; long long mask_gs; int ldmask;   // EPI_MASK: C *= (mask[m,n] > 0)
+};
+
+constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
+
+// C[g] = A[g] * B[g] for every replica g = blockIdx.z; 64x64 tile per CTA, 4x4 per thread.
+template <int EPI>
+__global__ void __launch_bounds__(SG_THREADS) simt_gemm_kernel(SimtGemmArgs p) {
+    __shared__ float As[SG_BK][SG_BM + 4];
+    __shared__ float Bs[SG_BK][SG_BN + 4];
+    const int g = blockIdx.z;
+    const float *A = p.A + (long long)g * p.a_gs;
+    const float *B = p.B + (long long)g * p.b_gs;
+    float *C = p.C + (long long)g * p.c_gs;
+    const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
+    const int t = threadIdx.x, tx = t % 16, ty = t / 16;
+    const bool a_kfast = (p.a_ks == 1), b_kfast = (p.b_ks == 1);
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < p.K; k0 += SG_BK) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = t + i * SG_THREADS;
+            int mm, kk;
+            if (a_kfast) { kk = e % SG_BK; mm = e / SG_BK; } else { mm = e % SG_BM; kk = e / SG_BM; }
+            const int m = m0 + mm, k = k0 + kk;
+            As[kk][mm] = (m < p.M && k < p.K) ? A[(long long)m * p.a_ms + (long long)k * p.a_ks] : 0.f;
+            int nn, kb;
+            if (b_kfast) { kb = e % SG_BK; nn = e / SG_BK; } else { nn = e % SG_BN; kb = e / SG_BN; }
+            const int n = n0 + nn, k2 = k0 + kb;
+            Bs[kb][nn] = (n < p.N && k2 < p.K) ? B[(long long)k2 * p.b_ks + (long long)n * p.b_ns] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < SG_BK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4 *>(&Bs[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    const float *bias = (EPI == EPI_BIAS || EPI == EPI_BIAS_RELU) ? p.bias + (long long)g * p.bias_gs : nullptr;
+    const float *mask = (EPI == EPI_MASK) ? p.mask + (long long)g * p.mask_gs : nullptr;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= p.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n >= p.N) continue;
+            float v = acc[i][j];
+            if (EPI == EPI_BIAS || EPI == EPI_BIAS_RELU) v += bias[n];
+            if (EPI == EPI_BIAS_RELU) v = fmaxf(v, 0.f);
+            if (EPI == EPI_MASK) v = (mask[(long long)m * p.ldmask + n] > 0.f) ? v : 0.f;
+            C[(long long)m * p.ldc + n] = v;
+        }
+    }
+}
+
+// Softmax cross-entropy backward, one warp per batch row:
+//   p = softmax(logits) (row max subtracted), dlogits = (p - onehot)/B,
+//   row_loss = logsumexp - logits[label].
+// Writes fp32 dlogits [rows, C] (d32 != NULL) and/or bf16 copies in both
+// layouts: dbf [B, ld_b] per replica and dbfT [C, B] per replica.
+__global__ void __launch_bounds__(256)
+softmax_ce_backward_kernel(const float *__restrict__ logits, const int32_t *__restrict__ labels,
+                           float *__restrict__ d32, __nv_bfloat16 *__restrict__ dbf,
+                           __nv_bfloat16 *__restrict__ dbfT, float *__restrict__ row_loss,
+                           int rows, int B, int C, int ld_b, int *status) {
+    const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (row >= rows) return;
+    const float *lg = logits + (size_t)row * C;
+    float mx = -INFINITY;
+    for (int j = lane; j < C; j += 32) mx = fmaxf(mx, lg[j]);
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float s = 0.f;
+    for (int j = lane; j < C; j += 32) s += __expf(lg[j] - mx);
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const int label = labels[row];
+    const bool label_ok = (label >= 0 && label < C);
+    const float inv_s = 1.f / s, inv_B = 1.f / (float)B;
+    const int g = row / B, i = row % B;
+    for (int j = lane; j < C; j += 32) {
+        float d = __expf(lg[j] - mx) * inv_s;
+        if (j == label) d -= 1.f;
+        d *= inv_B;
+        if (d32) d32[(size_t)row * C + j] = d;
+        if (dbf) {
+            const __nv_bfloat16 h = __float2bfloat16_rn(d);
+            dbf[((size_t)g * B + i) * ld_b + j] = h;
+            dbfT[((size_t)g * C + j) * B + i] = h;
+        }
+    }
+    if (lane == 0) {
+        row_loss[row] = label_ok ? (mx + __logf(s) - lg[label]) : 0.f;
+        if (!label_ok) status[SLOT_BAD_LABEL] = 1;
+    }
+}
+
+// loss[g] = (1/B) sum_i row_loss[g, i]; one block per replica, fixed-order tree.
+__global__ void __launch_bounds__(256)
+loss_mean_kernel(const float *__restrict__ row_loss, float *__restrict__ loss, int B) {
+    __shared__ float sh[256];
+    const int g = blockIdx.x;
+    float s = 0.f;
+    for (int i = threadIdx.x; i < B; i += 256) s += row_loss[(size_t)g * B + i];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) loss[g] = sh[0] / (float)B;
+}
+
+// db[g, j] = sum_i dH[g, i, j] from fp32 dH [n, B, d] (thread per column).
+__global__ void __launch_bounds__(256)
+bias_grad_f32_kernel(const float *__restrict__ dH, float *__restrict__ grad, long long grad_gs,
+                     int B, int d) {
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    const int g = blockIdx.y;
+    if (j >= d) return;
+    const float *p = dH + (size_t)g * B * d + j;
+    float s = 0.f;
+    for (int i = 0; i < B; ++i) s += p[(size_t)i * d];
+    grad[(long long)g * grad_gs + j] = s;
+}
+
+// db[g, j] = sum_i dH^T[g, j, i] from the bf16 transposed copy [n, d, B] (warp per row).
+__global__ void __launch_bounds__(256)
+bias_grad_bf16_kernel(const __nv_bfloat16 *__restrict__ dHT, float *__restrict__ grad,
+                      long long grad_gs, int B, int d) {
+    const int j = blockIdx.x * 8 + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    const int g = blockIdx.y;
+    if (j >= d) return;
+    const __nv_bfloat16 *p = dHT + ((size_t)g * d + j) * B;
+    float s = 0.f;
+    for (int i = lane; i < B; i += 32) s += __bfloat162float(p[i]);
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) grad[(long long)g * grad_gs + j] = s;
+}
+
+// Minibatch inputs fp32 [n, B, d] -> bf16 [n, B, d] and its transpose [n, d, B]
+// (the K-major operand of the first layer's weight-gradient product).
+__global__ void __launch_bounds__(256)
+input_to_bf16_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ Xb,
+                     __nv_bfloat16 *__restrict__ XbT, int B, int d) {
+    __shared__ float tile[32][33];
+    const int g = blockIdx.z;
+    const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;   // 32 x 8
+    for (int r = ty; r < 32; r += 8) {
+        const int i = i0 + r, j = j0 + tx;
+        float v = 0.f;
+        if (i < B && j < d) {
+            v = X[((size_t)g * B + i) * d + j];
+            Xb[((size_t)g * B + i) * d + j] = __float2bfloat16_rn(v);
+        }
+        tile[r][tx] = v;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int j = j0 + r, i = i0 + tx;
+        if (i < B && j < d) XbT[((size_t)g * d + j) * B + i] = __float2bfloat16_rn(tile[tx][r]);
+    }
+}
+
+}  // namespace parle

@@ -1,0 +1,574 @@
+// C ABI of the Parle round: context, planning, launches.  See include/parle.h
+// for the contract of every entry point.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+#include "mlp_simt.cuh"
+#include "umma_gemm.cuh"
+#include "update_kernels.cuh"
+
+using namespace parle;
+
+namespace {
+
+constexpr size_t kWsAlign = 1024;
+
+struct Workspace {
+    // byte offsets into parle_buffers.workspace; index = layer (0-based)
+    size_t act[PARLE_MAX_LAYERS];      // fp32 mode: output of layer l  [n,B,d_{l+1}] fp32 (last = logits)
+    size_t dact[PARLE_MAX_LAYERS];     // fp32 mode: gradient w.r.t. layer l's output [n,B,d_{l+1}] fp32
+    size_t logits;                     // bf16 mode: fp32 logits [n,B,C]
+    size_t shadow;                     // bf16 mode: bf16 copy of the GEMM operand vector [n,stride]
+    size_t xb, xbT;                    // bf16 mode: inputs [n,B,d_0] and transposed [n,d_0,B]
+    size_t hb[PARLE_MAX_LAYERS], hbT[PARLE_MAX_LAYERS];      // hidden activations, both layouts
+    size_t dhb[PARLE_MAX_LAYERS], dhbT[PARLE_MAX_LAYERS];    // their gradients, both layouts
+    int dh_ld[PARLE_MAX_LAYERS];       // row pitch of dhb[l] (d_{l+1} rounded up to 8)
+    size_t row_loss;                   // [n,B] fp32
+    size_t stage_in, stage_lab, stage_loss;   // staging for the host-buffer entry point
+    size_t total;
+};
+
+}  // namespace
+
+struct parle_ctx {
+    int n, n_layers, batch, gemm_dtype;
+    int dims[PARLE_MAX_LAYERS + 1];
+    float inv_gamma, inv_rho, alpha, eta, eta_prime;
+    size_t P, stride;
+    LayerPlan layers[PARLE_MAX_LAYERS];
+    Workspace ws;
+    bool bound;
+    parle_buffers buf;
+    cudaStream_t stream;
+    int *status_host, *status_dev;
+    bool round_open, fresh, shadow_is_x;
+    int steps_in_round;
+    long long launches;
+    int last_cuda;
+    int sm_count;
+    CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
+    CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
+    CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
+};
+
+namespace {
+
+inline int cuda_fail(parle_ctx *c, cudaError_t e) {
+    c->last_cuda = (int)e;
+    return PARLE_ECUDA;
+}
+#define PARLE_CUDA(c, expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
+#define PARLE_LAUNCHED(c) do { (c)->launches++; cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
+#define PARLE_TRY(expr) do { int rc_ = (expr); if (rc_ != PARLE_OK) return rc_; } while (0)
+
+inline bool coupling_ok(double v) { return v > 0.0 && !isnan(v); }
+inline float inverse_or_zero(double v) { return isinf(v) ? 0.0f : (float)(1.0 / v); }
+
+void plan_workspace(parle_ctx *c) {
+    Workspace &w = c->ws;
+    memset(&w, 0, sizeof(w));
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, kWsAlign); return o; };
+    const size_t n = c->n, B = c->batch;
+    const int nl = c->n_layers;
+    if (nl == 0) { w.total = kWsAlign; return; }
+    const size_t C = c->dims[nl];
+    if (c->gemm_dtype == PARLE_GEMM_FP32) {
+        for (int l = 0; l < nl; ++l) w.act[l] = take(n * B * c->dims[l + 1] * sizeof(float));
+        for (int l = 0; l < nl; ++l) w.dact[l] = take(n * B * c->dims[l + 1] * sizeof(float));
+    } else {
+        w.shadow = take(n * c->stride * 2);
+        w.xb = take(n * B * c->dims[0] * 2);
+        w.xbT = take(n * B * c->dims[0] * 2);
+        for (int l = 0; l + 1 < nl; ++l) {
+            w.hb[l] = take(n * B * c->dims[l + 1] * 2);
+            w.hbT[l] = take(n * B * c->dims[l + 1] * 2);
+        }
+        w.logits = take(n * B * C * sizeof(float));
+        for (int l = 0; l < nl; ++l) {
+            w.dh_ld[l] = (int)round_up(c->dims[l + 1], 8);
+            w.dhb[l] = take(n * B * w.dh_ld[l] * 2);
+            w.dhbT[l] = take(n * B * c->dims[l + 1] * 2);
+        }
+    }
+    w.row_loss = take(n * B * sizeof(float));
+    w.stage_in = take(n * B * c->dims[0] * sizeof(float));
+    w.stage_lab = take(n * B * sizeof(int32_t));
+    w.stage_loss = take(n * sizeof(float));
+    w.total = off;
+}
+
+template <typename T> inline T *ws_ptr(parle_ctx *c, size_t off) {
+    return reinterpret_cast<T *>(static_cast<char *>(c->buf.workspace) + off);
+}
+
+// ---------------------------------------------------------------- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+int get_encoder(parle_ctx *c, EncodeTiledFn *fn) {
+    static EncodeTiledFn cached = nullptr;
+    if (!cached) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        PARLE_CUDA(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q));
+        if (!p || q != cudaDriverEntryPointSuccess) return cuda_fail(c, cudaErrorNotSupported);
+        cached = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    *fn = cached;
+    return PARLE_OK;
+}
+
+// bf16 tensor [groups][rows][cols] (cols contiguous), row pitch and group pitch
+// in elements; box = box_cols x box_rows x 1, 128-byte swizzle, zero fill.
+int encode_bf16_map(parle_ctx *c, CUtensorMap *tm, const void *base, size_t cols, size_t rows, size_t groups,
+                    size_t row_pitch, size_t group_pitch, unsigned box_cols, unsigned box_rows) {
+    EncodeTiledFn enc;
+    PARLE_TRY(get_encoder(c, &enc));
+    cuuint64_t dims[3] = {cols, rows, groups};
+    cuuint64_t strides[2] = {row_pitch * 2, (group_pitch ? group_pitch : row_pitch * rows) * 2};
+    cuuint32_t box[3] = {box_cols, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
+    return PARLE_OK;
+}
+
+int build_tensor_maps(parle_ctx *c) {
+    const Workspace &w = c->ws;
+    const size_t n = c->n, B = c->batch;
+    const __nv_bfloat16 *shadow = ws_ptr<__nv_bfloat16>(c, w.shadow);
+    for (int l = 0; l < c->n_layers; ++l) {
+        const size_t din = c->dims[l], dout = c->dims[l + 1];
+        const __nv_bfloat16 *a_in = l == 0 ? ws_ptr<__nv_bfloat16>(c, w.xb) : ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]);
+        const __nv_bfloat16 *a_inT = l == 0 ? ws_ptr<__nv_bfloat16>(c, w.xbT) : ws_ptr<__nv_bfloat16>(c, w.hbT[l - 1]);
+        const __nv_bfloat16 *W = shadow + c->layers[l].w_off;
+        // forward: A = layer input [B, din], B = W [dout, din], both K-major (K = din)
+        PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_a[l], a_in, din, B, n, din, B * din, UM_BK, UM_BM));
+        PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_b[l], W, din, dout, n, din, c->stride, UM_BK, UM_BN));
+        // weight gradient: A = dH^T [dout, B], B = input^T [din, B], both K-major (K = batch)
+        PARLE_TRY(encode_bf16_map(c, &c->tm_wg_a[l], ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), B, dout, n, B, dout * B, UM_BK, UM_BM));
+        PARLE_TRY(encode_bf16_map(c, &c->tm_wg_b[l], a_inT, B, din, n, B, din * B, UM_BK, UM_BN));
+        if (l > 0) {
+            // data gradient: A = dH [B, dout] K-major (K = dout); B = W [dout (K), din (N)] MN-major,
+            // fetched as 64 k-rows x 64 n-columns boxes
+            PARLE_TRY(encode_bf16_map(c, &c->tm_dg_a[l], ws_ptr<__nv_bfloat16>(c, w.dhb[l]), dout, B, n,
+                                      w.dh_ld[l], B * (size_t)w.dh_ld[l], UM_BK, UM_BM));
+            PARLE_TRY(encode_bf16_map(c, &c->tm_dg_b[l], W, din, dout, n, din, c->stride, 64, UM_BK));
+        }
+    }
+    return PARLE_OK;
+}
+
+template <int EPI, bool B_MN>
+int launch_umma(parle_ctx *c, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
+    p.groups = c->n;
+    p.tiles_m = (p.M + UM_BM - 1) / UM_BM;
+    p.tiles_n = (p.N + UM_BN - 1) / UM_BN;
+    p.status = c->status_dev;
+    const int tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    umma_gemm_kernel<EPI, B_MN><<<grid, UM_THREADS, UM_SMEM_BYTES, c->stream>>>(a, b, p);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+
+template <int EPI, bool B_MN>
+cudaError_t allow_big_smem() {
+    return cudaFuncSetAttribute(umma_gemm_kernel<EPI, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)UM_SMEM_BYTES);
+}
+
+template <int EPI>
+int launch_simt(parle_ctx *c, const SimtGemmArgs &a) {
+    dim3 grid((a.N + SG_BN - 1) / SG_BN, (a.M + SG_BM - 1) / SG_BM, c->n);
+    simt_gemm_kernel<EPI><<<grid, SG_THREADS, 0, c->stream>>>(a);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+
+inline int stream_grid(const parle_ctx *c, size_t items, int per_thread) {
+    size_t blocks = (items + (size_t)kUpdThreads * per_thread - 1) / ((size_t)kUpdThreads * per_thread);
+    size_t cap = (size_t)c->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+// ---------------------------------------------------------------- the steps
+int run_inner_update(parle_ctx *c, const float *grad) {
+    const size_t n4 = (size_t)c->n * c->stride / 4;
+    constexpr int U = 2;
+    const int grid = stream_grid(c, n4, U);
+    const float4 *g = reinterpret_cast<const float4 *>(grad);
+    float4 *y = reinterpret_cast<float4 *>(c->buf.y), *z = reinterpret_cast<float4 *>(c->buf.z);
+    const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
+    const bool sh = c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0;
+    uint2 *shadow = sh ? ws_ptr<uint2>(c, c->ws.shadow) : nullptr;
+#define PARLE_UPD(F, S) inner_update_kernel<F, S, U><<<grid, kUpdThreads, 0, c->stream>>>( \
+        g, y, x, z, shadow, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev)
+    if (c->fresh) { if (sh) PARLE_UPD(true, true); else PARLE_UPD(true, false); }
+    else          { if (sh) PARLE_UPD(false, true); else PARLE_UPD(false, false); }
+#undef PARLE_UPD
+    PARLE_LAUNCHED(c);
+    c->fresh = false;
+    c->shadow_is_x = false;
+    c->steps_in_round++;
+    return PARLE_OK;
+}
+
+int forward_backward_fp32(parle_ctx *c, const float *inputs, const int32_t *labels, float *loss_out) {
+    const Workspace &w = c->ws;
+    const int nl = c->n_layers, n = c->n, B = c->batch;
+    const float *params = c->fresh ? c->buf.x : c->buf.y;      // folded reset: y == x on the first step
+    const long long S = (long long)c->stride;
+    for (int l = 0; l < nl; ++l) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        SimtGemmArgs a = {};
+        a.A = l == 0 ? inputs : ws_ptr<float>(c, w.act[l - 1]);
+        a.a_gs = (long long)B * din; a.a_ms = din; a.a_ks = 1;
+        a.B = params + c->layers[l].w_off; a.b_gs = S; a.b_ks = 1; a.b_ns = din;
+        a.C = ws_ptr<float>(c, w.act[l]); a.c_gs = (long long)B * dout; a.ldc = dout;
+        a.M = B; a.N = dout; a.K = din;
+        a.bias = params + c->layers[l].b_off; a.bias_gs = S;
+        if (l + 1 < nl) PARLE_TRY(launch_simt<EPI_BIAS_RELU>(c, a)); else PARLE_TRY(launch_simt<EPI_BIAS>(c, a));
+    }
+    const int C = c->dims[nl], rows = n * B;
+    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+        ws_ptr<float>(c, w.act[nl - 1]), labels, ws_ptr<float>(c, w.dact[nl - 1]), nullptr, nullptr,
+        ws_ptr<float>(c, w.row_loss), rows, B, C, 0, c->status_dev);
+    PARLE_LAUNCHED(c);
+    if (loss_out) {
+        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
+        PARLE_LAUNCHED(c);
+    }
+    for (int l = nl - 1; l >= 0; --l) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        const float *act_in = l == 0 ? inputs : ws_ptr<float>(c, w.act[l - 1]);
+        SimtGemmArgs a = {};                                    // dW_l = dH_l^T * H_{l-1}
+        a.A = ws_ptr<float>(c, w.dact[l]); a.a_gs = (long long)B * dout; a.a_ms = 1; a.a_ks = dout;
+        a.B = act_in; a.b_gs = (long long)B * din; a.b_ks = din; a.b_ns = 1;
+        a.C = c->buf.grad + c->layers[l].w_off; a.c_gs = S; a.ldc = din;
+        a.M = dout; a.N = din; a.K = B;
+        PARLE_TRY(launch_simt<EPI_PLAIN>(c, a));
+        bias_grad_f32_kernel<<<dim3((dout + 255) / 256, n), 256, 0, c->stream>>>(
+            ws_ptr<float>(c, w.dact[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
+        PARLE_LAUNCHED(c);
+        if (l > 0) {                                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
+            SimtGemmArgs d = {};
+            d.A = ws_ptr<float>(c, w.dact[l]); d.a_gs = (long long)B * dout; d.a_ms = dout; d.a_ks = 1;
+            d.B = params + c->layers[l].w_off; d.b_gs = S; d.b_ks = din; d.b_ns = 1;
+            d.C = ws_ptr<float>(c, w.dact[l - 1]); d.c_gs = (long long)B * din; d.ldc = din;
+            d.M = B; d.N = din; d.K = dout;
+            d.mask = ws_ptr<float>(c, w.act[l - 1]); d.mask_gs = (long long)B * din; d.ldmask = din;
+            PARLE_TRY(launch_simt<EPI_MASK>(c, d));
+        }
+    }
+    return PARLE_OK;
+}
+
+int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labels, float *loss_out) {
+    const Workspace &w = c->ws;
+    const int nl = c->n_layers, n = c->n, B = c->batch;
+    const long long S = (long long)c->stride;
+    const float *params = c->fresh ? c->buf.x : c->buf.y;      // fp32 biases come from the master copy
+    {
+        const int d0 = c->dims[0];
+        input_to_bf16_kernel<<<dim3((d0 + 31) / 32, (B + 31) / 32, n), 256, 0, c->stream>>>(
+            inputs, ws_ptr<__nv_bfloat16>(c, w.xb), ws_ptr<__nv_bfloat16>(c, w.xbT), B, d0);
+        PARLE_LAUNCHED(c);
+    }
+    for (int l = 0; l < nl; ++l) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        UmmaParams p = {};
+        p.M = B; p.N = dout; p.K = din;
+        p.bias = params + c->layers[l].b_off; p.bias_gs = S;
+        if (l + 1 < nl) {
+            p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
+            p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
+            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, false>(c, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+        } else {
+            p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
+            PARLE_TRY((launch_umma<UEPI_FWD_LAST, false>(c, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+        }
+    }
+    const int C = c->dims[nl], rows = n * B;
+    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+        ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
+        ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
+        c->status_dev);
+    PARLE_LAUNCHED(c);
+    if (loss_out) {
+        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
+        PARLE_LAUNCHED(c);
+    }
+    for (int l = nl - 1; l >= 0; --l) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        UmmaParams p = {};                                      // dW_l = dH_l^T * H_{l-1}
+        p.M = dout; p.N = din; p.K = B;
+        p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
+        PARLE_TRY((launch_umma<UEPI_WGRAD, false>(c, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+        bias_grad_bf16_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
+            ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
+        PARLE_LAUNCHED(c);
+        if (l > 0) {                                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
+            UmmaParams d = {};
+            d.M = B; d.N = din; d.K = dout;
+            d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
+            d.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); d.outT_gs = (long long)B * din; d.outT_ld = B;
+            d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
+            PARLE_TRY((launch_umma<UEPI_DGRAD, true>(c, c->tm_dg_a[l], c->tm_dg_b[l], d)));
+        }
+    }
+    return PARLE_OK;
+}
+
+int check_bound(const parle_ctx *c) {
+    if (!c) return PARLE_EINVAL;
+    if (!c->bound) return PARLE_ENOTBOUND;
+    return PARLE_OK;
+}
+
+}  // namespace
+
+// =========================================================================== C ABI
+extern "C" {
+
+int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, double rho, double alpha,
+               double eta, double eta_prime) {
+    if (!out) return PARLE_EINVAL;
+    *out = nullptr;
+    if (!model || !model->dims) return PARLE_EINVAL;
+    if (n < 1 || n > PARLE_MAX_REPLICAS) return PARLE_EINVAL;
+    if (model->n_layers < 0 || model->n_layers > PARLE_MAX_LAYERS) return PARLE_EINVAL;
+    if (model->gemm_dtype != PARLE_GEMM_FP32 && model->gemm_dtype != PARLE_GEMM_BF16) return PARLE_EINVAL;
+    if (!coupling_ok(gamma) || !coupling_ok(rho)) return PARLE_EINVAL;
+    if (!(alpha >= 0.0 && alpha < 1.0)) return PARLE_EINVAL;
+    if (!(eta > 0.0) || !(eta_prime > 0.0) || isinf(eta) || isinf(eta_prime)) return PARLE_EINVAL;
+    for (int l = 0; l <= model->n_layers; ++l)
+        if (model->dims[l] < 1) return PARLE_EINVAL;
+    if (model->n_layers > 0 && model->batch < 1) return PARLE_EINVAL;
+    if (model->n_layers > 0 && model->gemm_dtype == PARLE_GEMM_BF16) {
+        if (model->batch % 8) return PARLE_EUNSUPPORTED;
+        for (int l = 0; l < model->n_layers; ++l)
+            if (model->dims[l] % 8) return PARLE_EUNSUPPORTED;
+    }
+    parle_ctx *c = new (std::nothrow) parle_ctx;
+    if (!c) return PARLE_EINVAL;
+    memset(c, 0, sizeof(*c));
+    c->n = n; c->n_layers = model->n_layers; c->batch = model->n_layers ? model->batch : 0;
+    c->gemm_dtype = model->gemm_dtype;
+    for (int l = 0; l <= model->n_layers; ++l) c->dims[l] = model->dims[l];
+    c->inv_gamma = inverse_or_zero(gamma); c->inv_rho = inverse_or_zero(rho);
+    c->alpha = (float)alpha; c->eta = (float)eta; c->eta_prime = (float)eta_prime;
+    size_t off = 0, P = 0;
+    if (c->n_layers == 0) {
+        P = (size_t)c->dims[0];
+        off = round_up(P, 32);
+    } else {
+        for (int l = 0; l < c->n_layers; ++l) {
+            LayerPlan &lp = c->layers[l];
+            lp.d_in = c->dims[l]; lp.d_out = c->dims[l + 1];
+            lp.w_off = off; off = round_up(off + (size_t)lp.d_in * lp.d_out, 32);
+            lp.b_off = off; off = round_up(off + (size_t)lp.d_out, 32);
+            P += (size_t)lp.d_in * lp.d_out + lp.d_out;
+        }
+    }
+    c->P = P; c->stride = off;
+    plan_workspace(c);
+    *out = c;
+    return PARLE_OK;
+}
+
+void parle_destroy(parle_ctx *c) {
+    if (!c) return;
+    if (c->status_host) cudaFreeHost(c->status_host);
+    delete c;
+}
+
+size_t parle_param_count(const parle_ctx *c) { return c ? c->P : 0; }
+size_t parle_stride(const parle_ctx *c) { return c ? c->stride : 0; }
+size_t parle_workspace_bytes(const parle_ctx *c) { return c ? c->ws.total : 0; }
+
+int parle_layer_offset(const parle_ctx *c, int layer, size_t *w_off, size_t *b_off) {
+    if (!c || !w_off || !b_off || layer < 0 || layer >= c->n_layers) return PARLE_EINVAL;
+    *w_off = c->layers[layer].w_off;
+    *b_off = c->layers[layer].b_off;
+    return PARLE_OK;
+}
+
+int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
+    if (!c || !b) return PARLE_EINVAL;
+    if (!b->x || !b->y || !b->z || !b->grad || !b->xbar || !b->workspace) return PARLE_EINVAL;
+    const void *ptrs[6] = {b->x, b->y, b->z, b->grad, b->xbar, b->workspace};
+    for (const void *p : ptrs)
+        if (reinterpret_cast<uintptr_t>(p) % 128) return PARLE_EALIGN;
+    if (b->workspace_bytes < c->ws.total) return PARLE_EWORKSPACE;
+    c->bound = false;
+    int dev = 0;
+    PARLE_CUDA(c, cudaGetDevice(&dev));
+    PARLE_CUDA(c, cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    if (!c->status_host) {
+        // host memory (pinned, mapped): the one allocation the library makes
+        PARLE_CUDA(c, cudaHostAlloc(reinterpret_cast<void **>(&c->status_host), SLOT_COUNT * sizeof(int), cudaHostAllocMapped));
+        memset(c->status_host, 0, SLOT_COUNT * sizeof(int));
+        PARLE_CUDA(c, cudaHostGetDevicePointer(reinterpret_cast<void **>(&c->status_dev), c->status_host, 0));
+    }
+    c->buf = *b;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    if (c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16) {
+        int major = 0;
+        PARLE_CUDA(c, cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major != 10) return PARLE_EUNSUPPORTED;             // tcgen05 kernels need sm_100
+        PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, false>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, false>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, false>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, true>()));
+        PARLE_TRY(build_tensor_maps(c));
+    }
+    c->bound = true;
+    c->round_open = false; c->fresh = false; c->shadow_is_x = false; c->steps_in_round = 0;
+    return PARLE_OK;
+}
+
+int parle_round_begin(parle_ctx *c) {
+    PARLE_TRY(check_bound(c));
+    if (c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16 && !c->shadow_is_x) {
+        const size_t n4 = (size_t)c->n * c->stride / 4;
+        to_bf16_kernel<<<stream_grid(c, n4, 1), kUpdThreads, 0, c->stream>>>(
+            reinterpret_cast<const float4 *>(c->buf.x), ws_ptr<uint2>(c, c->ws.shadow), n4);
+        PARLE_LAUNCHED(c);
+        c->shadow_is_x = true;
+    }
+    c->round_open = true; c->fresh = true; c->steps_in_round = 0;
+    return PARLE_OK;
+}
+
+int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, float *loss_out) {
+    PARLE_TRY(check_bound(c));
+    if (c->n_layers == 0 || !inputs || !labels) return PARLE_EINVAL;
+    if (!c->round_open) return PARLE_ESTATE;
+    if (c->gemm_dtype == PARLE_GEMM_BF16) PARLE_TRY(forward_backward_bf16(c, inputs, labels, loss_out));
+    else PARLE_TRY(forward_backward_fp32(c, inputs, labels, loss_out));
+    return run_inner_update(c, c->buf.grad);
+}
+
+int parle_inner_step_host(parle_ctx *c, const float *inputs_host, const int32_t *labels_host, float *loss_out_host) {
+    PARLE_TRY(check_bound(c));
+    if (c->n_layers == 0 || !inputs_host || !labels_host) return PARLE_EINVAL;
+    if (!c->round_open) return PARLE_ESTATE;
+    const size_t nb = (size_t)c->n * c->batch;
+    float *din = ws_ptr<float>(c, c->ws.stage_in);
+    int32_t *dlab = ws_ptr<int32_t>(c, c->ws.stage_lab);
+    float *dloss = ws_ptr<float>(c, c->ws.stage_loss);
+    PARLE_CUDA(c, cudaMemcpyAsync(din, inputs_host, nb * c->dims[0] * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    PARLE_CUDA(c, cudaMemcpyAsync(dlab, labels_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+    PARLE_TRY(parle_inner_step(c, din, dlab, loss_out_host ? dloss : nullptr));
+    if (loss_out_host)
+        PARLE_CUDA(c, cudaMemcpyAsync(loss_out_host, dloss, c->n * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    return PARLE_OK;
+}
+
+int parle_inner_update(parle_ctx *c, const float *grad) {
+    PARLE_TRY(check_bound(c));
+    if (!grad) return PARLE_EINVAL;
+    if (reinterpret_cast<uintptr_t>(grad) % 16) return PARLE_EALIGN;
+    if (!c->round_open) return PARLE_ESTATE;
+    return run_inner_update(c, grad);
+}
+
+int parle_outer_step(parle_ctx *c) {
+    PARLE_TRY(check_bound(c));
+    if (!c->round_open || c->steps_in_round == 0) return PARLE_ESTATE;
+    const size_t s4 = c->stride / 4;
+    const int grid = stream_grid(c, s4, 1);
+    float4 *x = reinterpret_cast<float4 *>(c->buf.x), *xbar = reinterpret_cast<float4 *>(c->buf.xbar);
+    const float4 *z = reinterpret_cast<const float4 *>(c->buf.z);
+    const bool sh = c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0;
+    if (sh)
+        outer_mean_kernel<true, 4><<<grid, kUpdThreads, 0, c->stream>>>(
+            x, z, xbar, ws_ptr<uint2>(c, c->ws.shadow), s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
+    else
+        outer_mean_kernel<false, 4><<<grid, kUpdThreads, 0, c->stream>>>(
+            x, z, xbar, nullptr, s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
+    PARLE_LAUNCHED(c);
+    c->shadow_is_x = sh;
+    c->round_open = false; c->fresh = false; c->steps_in_round = 0;
+    return PARLE_OK;
+}
+
+int parle_mean(parle_ctx *c) {
+    PARLE_TRY(check_bound(c));
+    const size_t s4 = c->stride / 4;
+    mean_kernel<4><<<stream_grid(c, s4, 1), kUpdThreads, 0, c->stream>>>(
+        reinterpret_cast<const float4 *>(c->buf.x), reinterpret_cast<float4 *>(c->buf.xbar), s4, c->n, (float)c->n);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+
+int parle_round(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
+    PARLE_TRY(check_bound(c));
+    if (L < 1 || c->n_layers == 0 || !inputs || !labels) return PARLE_EINVAL;
+    PARLE_TRY(parle_round_begin(c));
+    const size_t nb = (size_t)c->n * c->batch;
+    for (int l = 0; l < L; ++l)
+        PARLE_TRY(parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
+                                   loss_out ? loss_out + (size_t)l * c->n : nullptr));
+    return parle_outer_step(c);
+}
+
+int parle_set_coupling(parle_ctx *c, double gamma, double rho) {
+    if (!c || !coupling_ok(gamma) || !coupling_ok(rho)) return PARLE_EINVAL;
+    c->inv_gamma = inverse_or_zero(gamma); c->inv_rho = inverse_or_zero(rho);
+    return PARLE_OK;
+}
+
+int parle_set_lr(parle_ctx *c, double eta, double eta_prime) {
+    if (!c || !(eta > 0.0) || !(eta_prime > 0.0) || isinf(eta) || isinf(eta_prime)) return PARLE_EINVAL;
+    c->eta = (float)eta; c->eta_prime = (float)eta_prime;
+    return PARLE_OK;
+}
+
+int parle_status(parle_ctx *c, int *device_flags) {
+    if (!c || !device_flags) return PARLE_EINVAL;
+    int f = 0;
+    if (c->status_host) {
+        volatile int *s = c->status_host;
+        if (s[SLOT_NONFINITE]) f |= PARLE_FLAG_NONFINITE;
+        if (s[SLOT_WAIT_LIMIT]) f |= PARLE_FLAG_WAIT_LIMIT;
+        if (s[SLOT_BAD_LABEL]) f |= PARLE_FLAG_BAD_LABEL;
+    }
+    *device_flags = f;
+    return PARLE_OK;
+}
+
+int parle_clear_status(parle_ctx *c) {
+    if (!c) return PARLE_EINVAL;
+    if (c->status_host) memset(c->status_host, 0, SLOT_COUNT * sizeof(int));
+    return PARLE_OK;
+}
+
+long long parle_launch_count(const parle_ctx *c) { return c ? c->launches : 0; }
+int parle_last_cuda_error(const parle_ctx *c) { return c ? c->last_cuda : 0; }
+
+const char *parle_strerror(int code) {
+    switch (code) {
+        case PARLE_OK: return "ok";
+        case PARLE_EINVAL: return "invalid argument";
+        case PARLE_ENOTBOUND: return "buffers not bound";
+        case PARLE_EALIGN: return "buffer not 128-byte aligned";
+        case PARLE_ECUDA: return "CUDA error";
+        case PARLE_ESTATE: return "call out of order";
+        case PARLE_EWORKSPACE: return "workspace too small";
+        case PARLE_EUNSUPPORTED: return "shape or device not supported by this GEMM path";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

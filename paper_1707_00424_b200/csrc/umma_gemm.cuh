@@ -1,0 +1,347 @@
+// Replica-grouped bf16 GEMMs on the sm_100a tensor cores for the MLP
+// forward / backward (Section 1.1 / 2.1: the minibatch gradient of f):
+//   forward      H_l      = act(H_{l-1} W_l^T + b_l)           A=[B,d_in]   K-major, B=W [d_out,d_in] K-major
+//   data grad    dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]        A=[B,d_out]  K-major, B=W [d_out(K), d_in(N)] MN-major
+//   weight grad  dW_l     = dH_l^T H_{l-1}                     A=dH^T [d_out,B] K-major, B=H^T [d_in,B] K-major
+// One persistent CTA per SM walks (replica, m-tile, n-tile) work items.
+// Warp 0 stages 128x64 operand tiles with TMA (128-byte swizzle) through a ring
+// of shared-memory buffers, warp 1 issues tcgen05.mma (M=128, N=128, K=16,
+// fp32 accumulators in tensor memory, two accumulator buffers), warps 2-5 read
+// the accumulators back with tcgen05.ld and run the fused epilogue.
+// Every wait is bounded: on a time-out the CTA records it in the status block,
+// drains and returns (tensor memory is always released).
+#pragma once
+
+#include "common.cuh"
+
+namespace parle {
+
+constexpr int UM_BM = 128, UM_BN = 128, UM_BK = 64;
+constexpr int UM_STAGES = 6;
+constexpr int UM_A_BYTES = UM_BM * UM_BK * 2;              // 16 KiB
+constexpr int UM_B_BYTES = UM_BN * UM_BK * 2;              // 16 KiB
+constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
+constexpr int UM_THREADS = 192;
+constexpr int UM_TMEM_COLS = 256;                          // two 128-column accumulators
+constexpr size_t UM_SMEM_BYTES = (size_t)UM_STAGES * UM_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long UM_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
+
+enum UmmaEpilogue {
+    UEPI_FWD_HIDDEN = 0,   // + bias[n], ReLU, bf16 out [M,ld] and transposed out [N,ldT]
+    UEPI_FWD_LAST = 1,     // + bias[n], fp32 out [M,ld]
+    UEPI_DGRAD = 2,        // * (mask[m,n] > 0), bf16 out and transposed out
+    UEPI_WGRAD = 3         // fp32 out [M,ld]
+};
+
+struct UmmaParams {
+    int M, N, K;                 // per-replica problem: D[M,N] = A[M,K] * B[N,K]^T
+    int groups, tiles_m, tiles_n;
+    const float *bias; long long bias_gs;
+    __nv_bfloat16 *out; long long out_gs; int out_ld;
+    __nv_bfloat16 *outT; long long outT_gs; int outT_ld;
+    float *outf; long long outf_gs; int outf_ld;
+    const __nv_bfloat16 *mask; long long mask_gs; int mask_ld;
+    int *status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the limit passed or another role of this
+// CTA already gave up (abort_flag, shared memory).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > UM_WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar,
+                                            int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a 128-byte-swizzled operand tile.
+//   K-major tile  : rows of 64 bf16 (128 B), 8-row groups 1024 B apart (SBO).
+//   MN-major tile : 64 k-rows of 64 MN-elements (128 B), 8-row groups 1024 B
+//                   apart (SBO); the next 64 MN-elements start lbo_bytes later.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;          // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;          // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128.
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn_major, bool b_mn_major) {
+    return (1u << 4)                       // D format fp32
+         | (1u << 7) | (1u << 10)          // A, B format bf16
+         | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16)
+         | ((uint32_t)(UM_BN >> 3) << 17) | ((uint32_t)(UM_BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void tile_coords(const UmmaParams &p, int t, int &g, int &m0, int &n0) {
+    const int per_g = p.tiles_m * p.tiles_n;
+    g = t / per_g;
+    const int r = t - g * per_g;
+    m0 = (r % p.tiles_m) * UM_BM;
+    n0 = (r / p.tiles_m) * UM_BN;
+}
+
+template <int EPI, bool B_MN>
+__global__ void __launch_bounds__(UM_THREADS, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const UmmaParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // 1024-byte aligned (swizzle atom)
+    uint8_t *ctl = smem_raw + (tiles_base - raw) + (size_t)UM_STAGES * UM_STAGE_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);                  // full[S], empty[S], tfull[2], tempty[2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * (2 * UM_STAGES + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * UM_STAGES;
+    const uint32_t bar_tfull = bar_empty + 8 * UM_STAGES, bar_tempty = bar_tfull + 16;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int num_kb = (p.K + UM_BK - 1) / UM_BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < UM_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)UM_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int g, m0, n0; tile_coords(p, t, g, m0, n0);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = tiles_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
+                    const uint32_t fb = bar_full + 8 * stage;
+                    mbar_expect_tx(fb, UM_STAGE_BYTES);
+                    tma_load_3d(sa, &tmA, fb, kb * UM_BK, m0, g);
+                    if (!B_MN) {
+                        tma_load_3d(sb, &tmB, fb, kb * UM_BK, n0, g);
+                    } else {
+                        tma_load_3d(sb, &tmB, fb, n0, kb * UM_BK, g);
+                        tma_load_3d(sb + UM_B_BYTES / 2, &tmB, fb, n0 + 64, kb * UM_BK, g);
+                    }
+                    if (++stage == UM_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // gave up: let the copies already issued land before the CTA exits
+                // (slots below `stage` were armed in this pass of the ring, the others in the previous one)
+                for (int s = 0; s < UM_STAGES; ++s) {
+                    const uint32_t armed_parity = (s < stage) ? phase : (phase ^ 1u);
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(false, B_MN);
+            int stage = 0; uint32_t phase = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * UM_BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = tiles_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
+                    const uint64_t adesc = make_smem_desc(sa, 16, 1024);
+                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, UM_B_BYTES / 2, 1024)
+                                                : make_smem_desc(sb, 16, 1024);
+#pragma unroll
+                    for (int k = 0; k < UM_BK / 16; ++k) {
+                        // K-major: 16 bf16 = 32 B further along the row; MN-major: two 8-row groups = 2048 B
+                        const uint64_t a_k = adesc + (uint64_t)(k * 2);
+                        const uint64_t b_k = bdesc + (uint64_t)(B_MN ? k * 128 : k * 2);
+                        tc_mma_bf16(d_tmem, a_k, b_k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty + 8 * stage);        // frees the smem slot when these MMAs retire
+                    if (++stage == UM_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(bar_tfull + 8 * acc);              // accumulator complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                              // TMEM lane quarter this warp may read
+        int acc = 0; uint32_t acc_phase = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            int g, m0, n0; tile_coords(p, t, g, m0, n0);
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const int m = m0 + q * 32 + lane;                // output row of this thread
+            const bool m_ok = m < p.M;
+#pragma unroll 1
+            for (int c = 0; c < UM_BN / 32; ++c) {
+                const int nb = n0 + c * 32;
+                if (nb >= p.N) break;                        // warp-uniform
+                uint32_t r[32];
+                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * UM_BN + c * 32), r);
+                tc_wait_ld();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_FWD_LAST) {
+                    const float *bias = p.bias + (long long)g * p.bias_gs;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float b = (nb + j < p.N) ? __ldg(bias + nb + j) : 0.f;
+                        v[j] += b;
+                        if (EPI == UEPI_FWD_HIDDEN) v[j] = fmaxf(v[j], 0.f);
+                    }
+                }
+                if (EPI == UEPI_DGRAD) {
+                    if (m_ok) {
+                        const __nv_bfloat16 *mk = p.mask + (long long)g * p.mask_gs + (long long)m * p.mask_ld + nb;
+#pragma unroll
+                        for (int j8 = 0; j8 < 32; j8 += 8) {
+                            if (nb + j8 < p.N) {             // N % 8 == 0: whole group in range
+                                const uint4 raw4 = *reinterpret_cast<const uint4 *>(mk + j8);
+                                const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&raw4);
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    if (!(__bfloat162float(h[j]) > 0.f)) v[j8 + j] = 0.f;
+                            }
+                        }
+                    }
+                }
+                if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_DGRAD) {
+                    // row-major bf16 [M, ld]: each thread owns 32 consecutive columns of its row
+                    if (m_ok) {
+                        __nv_bfloat16 *o = p.out + (long long)g * p.out_gs + (long long)m * p.out_ld + nb;
+#pragma unroll
+                        for (int j8 = 0; j8 < 32; j8 += 8) {
+                            if (nb + j8 < p.N) {
+                                uint4 pk;
+                                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[j8 + 0], v[j8 + 1]);
+                                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[j8 + 2], v[j8 + 3]);
+                                __nv_bfloat162 t2 = __floats2bfloat162_rn(v[j8 + 4], v[j8 + 5]);
+                                __nv_bfloat162 t3 = __floats2bfloat162_rn(v[j8 + 6], v[j8 + 7]);
+                                pk.x = *reinterpret_cast<uint32_t *>(&t0); pk.y = *reinterpret_cast<uint32_t *>(&t1);
+                                pk.z = *reinterpret_cast<uint32_t *>(&t2); pk.w = *reinterpret_cast<uint32_t *>(&t3);
+                                *reinterpret_cast<uint4 *>(o + j8) = pk;
+                            }
+                        }
+                        // transposed bf16 [N, ldT]: the 32 lanes write 32 consecutive batch rows
+                        __nv_bfloat16 *oT = p.outT + (long long)g * p.outT_gs + m;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N) oT[(long long)(nb + j) * p.outT_ld] = __float2bfloat16_rn(v[j]);
+                    }
+                }
+                if (EPI == UEPI_FWD_LAST || EPI == UEPI_WGRAD) {
+                    if (m_ok) {
+                        float *o = p.outf + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
+                        if (EPI == UEPI_WGRAD) {             // N % 8 == 0 and ld % 8 == 0: 16-byte stores
+#pragma unroll
+                            for (int j4 = 0; j4 < 32; j4 += 4)
+                                if (nb + j4 < p.N)
+                                    *reinterpret_cast<float4 *>(o + j4) = make_float4(v[j4], v[j4 + 1], v[j4 + 2], v[j4 + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + j < p.N) o[j] = v[j];
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) p.status[SLOT_WAIT_LIMIT] = 1;
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)UM_TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace parle

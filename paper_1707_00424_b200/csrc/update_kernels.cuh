@@ -1,0 +1,154 @@
+// Streaming kernels of the Parle round: the fused inner update
+// (Eq. parle_y + Eq. parle_z), the fused outer update + replica mean
+// (Eq. parle_xa + Eq. parle_x with eta'' = rho/n), the stand-alone mean and the
+// bf16 shadow conversion.  All are HBM-bound: every vector is touched once,
+// with 16-byte accesses, consecutive threads on consecutive addresses.
+#pragma once
+
+#include "common.cuh"
+
+namespace parle {
+
+constexpr int kUpdThreads = 256;
+
+__device__ __forceinline__ bool finite4(const float4 &v) {
+    // NaN and Inf both fail "|v| <= FLT_MAX"
+    return (fabsf(v.x) <= 3.402823466e+38f) & (fabsf(v.y) <= 3.402823466e+38f) &
+           (fabsf(v.z) <= 3.402823466e+38f) & (fabsf(v.w) <= 3.402823466e+38f);
+}
+
+__device__ __forceinline__ uint2 pack_bf16x4(const float4 &v) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 r;
+    r.x = *reinterpret_cast<uint32_t *>(&lo);
+    r.y = *reinterpret_cast<uint32_t *>(&hi);
+    return r;
+}
+
+// Eq. (parle_y): y <- y - eta' (g + (y - x)/gamma), Eq. (parle_z): z <- alpha z + (1-alpha) y_new.
+// FIRST: first inner step of a round, where y = z = x (the reset is folded in:
+// x is read in place of y and z, which are only written).
+// SHADOW: also write y_new rounded to bf16 (the GEMM operand copy).
+template <bool FIRST, bool SHADOW, int UNROLL>
+__global__ void __launch_bounds__(kUpdThreads)
+inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const float4 *__restrict__ x,
+                    float4 *__restrict__ z, uint2 *__restrict__ shadow, size_t n4,
+                    float eta_p, float inv_gamma, float alpha, int *status) {
+    const size_t tid = (size_t)blockIdx.x * kUpdThreads + threadIdx.x;
+    const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
+    const float one_m_alpha = 1.0f - alpha;
+    bool ok = true;
+    for (size_t base = tid; base < n4; base += nthreads * UNROLL) {
+        float4 gv[UNROLL], yv[UNROLL], xv[UNROLL], zv[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const size_t i = base + (size_t)u * nthreads;
+            if (i < n4) {
+                gv[u] = __ldcs(g + i);
+                xv[u] = __ldg(x + i);
+                if (!FIRST) {
+                    yv[u] = y[i];
+                    zv[u] = z[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const size_t i = base + (size_t)u * nthreads;
+            if (i < n4) {
+                float4 yo = FIRST ? xv[u] : yv[u];
+                float4 zo = FIRST ? xv[u] : zv[u];
+                float4 yn, zn;
+                yn.x = yo.x - eta_p * fmaf(inv_gamma, yo.x - xv[u].x, gv[u].x);
+                yn.y = yo.y - eta_p * fmaf(inv_gamma, yo.y - xv[u].y, gv[u].y);
+                yn.z = yo.z - eta_p * fmaf(inv_gamma, yo.z - xv[u].z, gv[u].z);
+                yn.w = yo.w - eta_p * fmaf(inv_gamma, yo.w - xv[u].w, gv[u].w);
+                zn.x = fmaf(alpha, zo.x, one_m_alpha * yn.x);
+                zn.y = fmaf(alpha, zo.y, one_m_alpha * yn.y);
+                zn.z = fmaf(alpha, zo.z, one_m_alpha * yn.z);
+                zn.w = fmaf(alpha, zo.w, one_m_alpha * yn.w);
+                ok &= finite4(yn);
+                y[i] = yn;
+                z[i] = zn;
+                if (SHADOW) shadow[i] = pack_bf16x4(yn);
+            }
+        }
+    }
+    if (!ok) status[SLOT_NONFINITE] = 1;
+}
+
+// Eq. (parle_xa) for all replicas of a coordinate, then Eq. (parle_x): each
+// thread owns four consecutive coordinates, walks the replica axis in a fixed
+// order (deterministic sum, no atomics) and writes the new mean.
+// SHADOW: also write bf16(x_new), the GEMM operand of the next round's first step.
+template <bool SHADOW, int RCHUNK>
+__global__ void __launch_bounds__(kUpdThreads)
+outer_mean_kernel(float4 *__restrict__ x, const float4 *__restrict__ z, float4 *__restrict__ xbar,
+                  uint2 *__restrict__ shadow, size_t stride4, int n, float eta, float eta_over_rho,
+                  float n_as_float, int *status) {
+    const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
+    bool ok = true;
+    for (size_t j = (size_t)blockIdx.x * kUpdThreads + threadIdx.x; j < stride4; j += nthreads) {
+        const float4 xb = xbar[j];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int a0 = 0; a0 < n; a0 += RCHUNK) {
+            float4 xv[RCHUNK], zv[RCHUNK];
+#pragma unroll
+            for (int r = 0; r < RCHUNK; ++r) {
+                if (a0 + r < n) {
+                    const size_t i = (size_t)(a0 + r) * stride4 + j;
+                    xv[r] = x[i];
+                    zv[r] = __ldcs(z + i);
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < RCHUNK; ++r) {
+                if (a0 + r < n) {
+                    const size_t i = (size_t)(a0 + r) * stride4 + j;
+                    float4 xn;
+                    xn.x = xv[r].x - eta * (xv[r].x - zv[r].x) - eta_over_rho * (xv[r].x - xb.x);
+                    xn.y = xv[r].y - eta * (xv[r].y - zv[r].y) - eta_over_rho * (xv[r].y - xb.y);
+                    xn.z = xv[r].z - eta * (xv[r].z - zv[r].z) - eta_over_rho * (xv[r].z - xb.z);
+                    xn.w = xv[r].w - eta * (xv[r].w - zv[r].w) - eta_over_rho * (xv[r].w - xb.w);
+                    ok &= finite4(xn);
+                    x[i] = xn;
+                    if (SHADOW) shadow[i] = pack_bf16x4(xn);
+                    acc.x += xn.x; acc.y += xn.y; acc.z += xn.z; acc.w += xn.w;
+                }
+            }
+        }
+        xbar[j] = make_float4(acc.x / n_as_float, acc.y / n_as_float, acc.z / n_as_float, acc.w / n_as_float);
+    }
+    if (!ok) status[SLOT_NONFINITE] = 1;
+}
+
+// Eq. (parle_x) with eta'' = rho/n alone: xbar <- (1/n) sum_a x^a.
+template <int RCHUNK>
+__global__ void __launch_bounds__(kUpdThreads)
+mean_kernel(const float4 *__restrict__ x, float4 *__restrict__ xbar, size_t stride4, int n, float n_as_float) {
+    const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
+    for (size_t j = (size_t)blockIdx.x * kUpdThreads + threadIdx.x; j < stride4; j += nthreads) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int a0 = 0; a0 < n; a0 += RCHUNK) {
+            float4 xv[RCHUNK];
+#pragma unroll
+            for (int r = 0; r < RCHUNK; ++r)
+                if (a0 + r < n) xv[r] = __ldcs(x + (size_t)(a0 + r) * stride4 + j);
+#pragma unroll
+            for (int r = 0; r < RCHUNK; ++r)
+                if (a0 + r < n) { acc.x += xv[r].x; acc.y += xv[r].y; acc.z += xv[r].z; acc.w += xv[r].w; }
+        }
+        xbar[j] = make_float4(acc.x / n_as_float, acc.y / n_as_float, acc.z / n_as_float, acc.w / n_as_float);
+    }
+}
+
+// bf16 copy of an fp32 vector (round to nearest even).
+__global__ void __launch_bounds__(kUpdThreads)
+to_bf16_kernel(const float4 *__restrict__ src, uint2 *__restrict__ dst, size_t n4) {
+    const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
+    for (size_t i = (size_t)blockIdx.x * kUpdThreads + threadIdx.x; i < n4; i += nthreads)
+        dst[i] = pack_bf16x4(src[i]);
+}
+
+}  // namespace parle

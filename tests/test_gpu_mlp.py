@@ -1,0 +1,191 @@
+"""GPU parity of the whole round (forward/backward, Eq. parle_y .. parle_x)
+against the fp64 oracle on seeded inputs, through the C ABI.
+
+Bounds: relative L2 error of every parameter tensor after a round
+<= 1e-4 for fp32 GEMMs and <= 2e-2 for bf16 GEMM operands."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_1707_00424_b200 as pb
+import synth_inputs as si
+from oracle import parle_oracle as po
+from _util import padding_mask, rel_l2, to_dense, to_padded
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOL = {pb.GEMM_FP32: 1e-4, pb.GEMM_BF16: 2e-2}
+
+
+def make(cfg, **over):
+    hyper = dict(gamma=cfg.gamma, rho=cfg.rho, alpha=cfg.alpha, eta=cfg.eta, eta_prime=cfg.eta_prime)
+    hyper.update(over)
+    m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, **hyper).alloc(DEV)
+    x0 = np.stack([po.pack(si.init_replica(cfg, a)) for a in range(cfg.n)])
+    m.x.copy_(torch.from_numpy(to_padded(m, x0)))
+    m.mean(); torch.cuda.synchronize()
+    xbar0 = x0.mean(axis=0)
+    return m, x0, xbar0, po.Hyper(hyper["eta"], hyper["eta_prime"], hyper["alpha"], hyper["gamma"], hyper["rho"])
+
+
+def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False):
+    m, xo, xb, hp = make(cfg)
+    tol = TOL[cfg.gemm_dtype]
+    pad = torch.from_numpy(padding_mask(m)).to(DEV)
+    for r in range(rounds):
+        X, c = si.round_batches(cfg, r)
+        Xd, cd = torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)
+        loss = torch.zeros(cfg.L, cfg.n, device=DEV)
+        if use_round_call:
+            m.round(cfg.L, Xd, cd, loss)
+            y_gpu = z_gpu = None
+        else:
+            m.round_begin()
+            for l in range(cfg.L):
+                m.inner_step(Xd[l], cd[l], loss[l])
+            y_gpu, z_gpu = to_dense(m, m.y.cpu().numpy()), to_dense(m, m.z.cpu().numpy())
+            m.outer_step()
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        out = po.parle_round(xo, xb, po.mlp_grad_fn(cfg.dims, X, c), cfg.L, hp)
+        x_gpu, xb_gpu = to_dense(m, m.x.cpu().numpy()), to_dense(m, m.xbar.cpu().numpy())
+        errs = {"xbar": rel_l2(xb_gpu, out["xbar"])}
+        for a in range(cfg.n):
+            errs[f"x{a}"] = rel_l2(x_gpu[a], out["x"][a])
+            if y_gpu is not None:
+                errs[f"y{a}"] = rel_l2(y_gpu[a], out["y"][a])
+                errs[f"z{a}"] = rel_l2(z_gpu[a], out["z"][a])
+        assert max(errs.values()) <= tol, errs
+        # stricter, on the displacement of the round (what the round actually computed)
+        disp = rel_l2(x_gpu - xo, out["x"] - xo)
+        if disp_tol is not None:
+            assert disp <= disp_tol, disp
+        np.testing.assert_allclose(loss.cpu().numpy(), out["loss"], rtol=50 * tol, atol=1e-5)
+        assert torch.all(m.x[:, pad] == 0) and torch.all(m.xbar[pad] == 0)
+        # invariant of Section 3.1: xbar is the mean of the current replicas
+        np.testing.assert_allclose(xb_gpu, x_gpu.mean(axis=0), rtol=1e-5, atol=1e-6)
+        xo, xb = out["x"], out["xbar"]
+    return m
+
+
+def grad_check(cfg, tol):
+    """One inner step: the gradient buffer against the oracle's gradient, layer by layer."""
+    m, xo, xb, hp = make(cfg)
+    X, c = si.round_batches(cfg.scaled(L=1), 0)
+    loss = torch.zeros(cfg.n, device=DEV)
+    m.round_begin(); m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV), loss)
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    g_gpu = to_dense(m, m.grad.cpu().numpy())
+    for a in range(cfg.n):
+        lo, g = po.mlp_loss_grad(xo[a], cfg.dims, X[0, a], c[0, a])
+        assert abs(loss[a].item() - lo) <= 20 * tol * max(1.0, abs(lo)), (a, loss[a].item(), lo)
+        got, want = po.unpack(g_gpu[a], cfg.dims), po.unpack(g, cfg.dims)
+        for l, ((gW, gb), (wW, wb)) in enumerate(zip(got, want)):
+            assert rel_l2(gW, wW) <= tol, ("dW", a, l, rel_l2(gW, wW))
+            assert rel_l2(gb, wb) <= tol, ("db", a, l, rel_l2(gb, wb))
+    return m
+
+
+# ------------------------------------------------------------------ fp32 GEMMs
+def test_c1_gradient_fp32():
+    grad_check(si.C1, 1e-5)
+
+
+def test_c1_two_rounds_fp32():
+    run_rounds(si.C1, si.C1.rounds, disp_tol=1e-4)
+
+
+def test_ragged_shapes_fp32():
+    cfg = si.C1.scaled(name="ragged", n=2, dims=(37, 19, 23, 7), batch=5, L=3)
+    grad_check(cfg, 1e-5)
+    run_rounds(cfg, 2, disp_tol=1e-4)
+    cfg = si.C1.scaled(name="tiles", n=3, dims=(130, 67, 129), batch=70, L=2)   # several tiles + tails
+    grad_check(cfg, 1e-5)
+    run_rounds(cfg, 1, disp_tol=1e-4, use_round_call=True)
+
+
+def test_single_layer_and_single_replica_fp32():
+    run_rounds(si.C1.scaled(name="linear", n=1, dims=(20, 6), batch=9, L=4), 2, disp_tol=1e-4)
+
+
+def test_couplings_off_is_plain_sgd_on_gpu():
+    cfg = si.C1.scaled(L=1)
+    m, xo, xb, hp = make(cfg, gamma=math.inf, rho=math.inf, eta=1.0, alpha=0.0)
+    X, c = si.round_batches(cfg, 0)
+    m.round(1, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
+    x_gpu = to_dense(m, m.x.cpu().numpy())
+    for a in range(cfg.n):
+        _, g = po.mlp_loss_grad(xo[a], cfg.dims, X[0, a], c[0, a])
+        assert rel_l2(x_gpu[a] - xo[a], -cfg.eta_prime * g) < 1e-5
+
+
+def test_identical_replicas_shared_batches_stay_identical_on_gpu():
+    cfg = si.C1
+    m, xo, xb, hp = make(cfg)
+    m.x.copy_(m.x[0].clone().expand_as(m.x)); m.mean()
+    X, c = si.round_batches(cfg, 0, shared=True)
+    m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
+    for a in range(1, cfg.n):
+        assert torch.equal(m.x[a], m.x[0])
+
+
+def test_bad_label_is_flagged_not_faulted():
+    cfg = si.C1
+    m, *_ = make(cfg)
+    X, c = si.round_batches(cfg, 0)
+    c = c.copy(); c[0, 1, 3] = 99
+    m.round_begin(); m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV)); torch.cuda.synchronize()
+    assert m.status() & pb.FLAG_BAD_LABEL
+
+
+def test_host_buffer_step_matches_device_step():
+    cfg = si.C1
+    X, c = si.round_batches(cfg, 0)
+    res = []
+    for host in (False, True):
+        m, *_ = make(cfg)
+        m.round_begin()
+        if host:
+            Xh, ch = torch.from_numpy(X[0]).pin_memory(), torch.from_numpy(c[0]).pin_memory()
+            lh = torch.zeros(cfg.n).pin_memory()
+            m.inner_step_host(Xh, ch, lh); torch.cuda.synchronize()
+            res.append((m.y.clone(), lh.clone()))
+        else:
+            ld = torch.zeros(cfg.n, device=DEV)
+            m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV), ld); torch.cuda.synchronize()
+            res.append((m.y.clone(), ld.cpu()))
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+
+
+def test_c2_one_round_fp32():
+    run_rounds(si.C2, 1, disp_tol=1e-3)
+
+
+# ------------------------------------------------------------------ bf16 GEMMs (tcgen05)
+def test_small_gradient_bf16():
+    grad_check(si.C1.scaled(name="bf16-small", dims=(64, 128, 72, 10), batch=16, gemm_dtype=1), 2e-2)
+
+
+def test_ragged_tiles_gradient_bf16():
+    # several 128-tiles with tails in every dimension, K tails, last width not a multiple of 8
+    grad_check(si.C1.scaled(name="bf16-ragged", n=2, dims=(200, 328, 136, 101), batch=136, gemm_dtype=1), 2e-2)
+
+
+def test_small_rounds_bf16():
+    run_rounds(si.C1.scaled(name="bf16-small", dims=(64, 128, 72, 10), batch=16, gemm_dtype=1), 2, disp_tol=5e-2)
+
+
+def test_c3_scaled_down_round_bf16():
+    cfg = si.C3.scaled(name="C3/4", n=2, dims=(768, 512, 512, 512, 100), L=5)
+    run_rounds(cfg, 2, disp_tol=5e-2)
+
+
+def test_c3_gradient_full_shape_bf16():
+    grad_check(si.C3.scaled(n=2), 2e-2)
+
+
+def test_c3_full_round_bf16():
+    run_rounds(si.C3, 1, disp_tol=5e-2, use_round_call=True)
