@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the Parle round (arXiv 1707.00424, Section 3) on B200.
+
+A "step" is one whole Parle round over n replicas: round begin, L inner steps
+(forward/backward + Eq. parle_y/parle_z), the outer step (Eq. parle_xa) and the
+replica mean (Eq. parle_x).  The metric is replica-inner-steps per second
+= n * L * rounds / time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
+
+Prints ONE JSON line.  With --impl reference the fp64 CPU oracle is timed on the
+host cores instead (a bounded sample of the same workload per step).
+Multi-GPU (torchrun): every rank holds n replicas; the only exchange is the
+average of the per-rank means once per round (NCCL all-reduce), so the job has
+N*n replicas and scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "parle_replica_inner_steps_per_sec"
+UNIT = "replica-inner-steps/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for nm, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------ workloads
+def make_round_inputs(cfg, sets: int):
+    """`sets` rounds' worth of minibatches: X [sets, L, n, B, d0] fp32, labels [sets, L, n, B] int32."""
+    Xs, cs = [], []
+    for r in range(sets):
+        X, c = si.round_batches(cfg, r)
+        Xs.append(X); cs.append(c)
+    return np.stack(Xs), np.stack(cs)
+
+
+def dense_to_padded(model, cfg, replica_layers):
+    out = np.zeros((cfg.n, model.stride), dtype=np.float32)
+    for a, layers in enumerate(replica_layers):
+        for l, (W, b) in enumerate(layers):
+            w_off, b_off = model.layer_offset(l)
+            out[a, w_off:w_off + W.size] = W.ravel()
+            out[a, b_off:b_off + b.size] = b
+    return out
+
+
+def bytes_per_param_inner_update(cfg) -> int:
+    # read g, y, x, z + write y, z (fp32) [+ bf16 operand copy of y]
+    return 24 + (2 if cfg.gemm_dtype == 1 else 0)
+
+
+# ------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1707_00424_b200 as pb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the Parle library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = si.CONFIGS[args.workload]
+    if world > 1:           # every rank owns its own n replicas (independent streams per rank)
+        cfg = cfg.scaled(seed=cfg.seed + 7919 * rank)
+    model = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, gamma=cfg.gamma, rho=cfg.rho,
+                     alpha=cfg.alpha, eta=cfg.eta, eta_prime=cfg.eta_prime).alloc(dev)
+    model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
+    model.mean()
+    sets = 2
+    Xh, ch = make_round_inputs(cfg, sets)
+    Xd, cd = torch.from_numpy(Xh).to(dev), torch.from_numpy(ch).to(dev)
+    Xp, cp = torch.from_numpy(Xh).pin_memory(), torch.from_numpy(ch).pin_memory()
+    loss_d = torch.zeros(cfg.L, cfg.n, device=dev)
+    loss_p = torch.zeros(cfg.L, cfg.n).pin_memory()
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    def exchange():
+        if world > 1:       # global mean = mean over ranks of the per-rank means (equal replica counts)
+            dist.all_reduce(model.xbar, op=dist.ReduceOp.AVG)
+
+    def round_device(r):
+        model.round(cfg.L, Xd[r % sets], cd[r % sets], loss_d)
+        exchange()
+
+    def round_host(r):
+        model.round_begin()
+        for l in range(cfg.L):
+            model.inner_step_host(Xp[r % sets, l], cp[r % sets, l], loss_p[l])
+        model.outer_step()
+        exchange()
+
+    def timed(fn, warmup, steps, sample_clocks=False):
+        for r in range(warmup):
+            fn(r)
+        sync_all()
+        sampler = ClockSampler(local) if sample_clocks else None
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = model.launch_count
+        e0.record()
+        for r in range(steps):
+            fn(warmup + r)
+        e1.record()
+        sync_all()
+        clocks = sampler.stop() if sampler else None
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, model.launch_count - launches0, clocks
+
+    W, K = max(args.warmup, 0), args.steps
+    # 1. device-resident inputs: the headline value
+    ms, launches, clocks = timed(round_device, W, K, sample_clocks=True)
+    flags = model.status()
+    value = world * cfg.n * cfg.L * K / (ms * 1e-3)
+    # 2. per-kernel-class device time over the same K rounds (events around every launch)
+    model.profile_enable(True)
+    for r in range(K):
+        round_device(W + r)
+    prof, dropped = model.profile_read()
+    model.profile_enable(False)
+    # 3. end to end: host (pinned) inputs copied in and per-step losses copied out inside the timed region
+    ms_e2e, _, _ = timed(round_host, min(W, 2), K)
+    e2e_value = world * cfg.n * cfg.L * K / (ms_e2e * 1e-3)
+    h2d = cfg.L * (cfg.n * cfg.batch * cfg.dims[0] * 4 + cfg.n * cfg.batch * 4)
+    d2h = cfg.L * cfg.n * 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    total_ms = sum(v[0] for v in prof.values()) or 1.0
+    shares = {k: {"ms_per_round": v[0] / K, "launches_per_round": v[1] / K, "share": v[0] / total_ms} for k, v in prof.items()}
+    dom = max(prof, key=lambda k: prof[k][0])
+    roofline = None
+    if dom == "inner_update":
+        per_launch_ms = prof[dom][0] / prof[dom][1]
+        # steady-state launches move 24 (+2) B per element; the first of each round (reset folded in) 8 B less
+        bpp = bytes_per_param_inner_update(cfg)
+        bytes_per_launch = cfg.n * model.stride * (bpp - 8.0 / cfg.L)
+        ach = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "bytes_per_launch": bytes_per_launch, "ms_per_launch": per_launch_ms}
+    else:
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": None, "traffic": None, "peak_source": peaks["source"]}
+    cpu = cpu_baseline(cfg, budget_s=15.0)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.gemm_dtype == 1 else "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: n={cfg.n} replicas/GPU, MLP {'-'.join(map(str, cfg.dims))}, batch {cfg.batch}, L={cfg.L}, "
+                               f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else 'fp32'}",
+                   "step": "one Parle round (L inner steps + outer step + replica mean)",
+                   "l2": "state + gradients per round >> 126 MB L2 (no flush needed)" if cfg.n * model.stride * 16 > 4e8 else "working set may be L2 resident",
+                   "parallelism": f"{world} x {cfg.n} replicas, one all-reduce of xbar per round" if world > 1 else "single GPU"},
+        "gpu_launches": launches, "device_flags": flags, "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e / K},
+        "roofline": roofline, "kernel_shares": shares, "profile_dropped": dropped,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------ oracle timing (CPU)
+def _blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(cfg, inner_steps: int, rnd: int = 0):
+    """Time the oracle on `inner_steps` inner steps of one round (all n replicas) + outer step + mean."""
+    from oracle import parle_oracle as po
+    sub = cfg.scaled(L=inner_steps)
+    X, c = si.round_batches(sub, rnd)
+    x0 = np.stack([po.pack(si.init_replica(cfg, a)) for a in range(cfg.n)])
+    hp = po.Hyper(cfg.eta, cfg.eta_prime, cfg.alpha, cfg.gamma, cfg.rho)
+    t0 = time.perf_counter()
+    po.parle_round(x0, x0.mean(axis=0), po.mlp_grad_fn(cfg.dims, X, c), inner_steps, hp)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, budget_s: float):
+    """The oracle as it stands, on the host cores, on a bounded sample of the workload."""
+    t1 = oracle_sample(cfg, 1)
+    steps = int(max(1, min(cfg.L, budget_s / max(t1, 1e-3))))
+    t = oracle_sample(cfg, steps) if steps > 1 else t1
+    return {"value": cfg.n * steps / t, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+            "sample": f"{steps} of {cfg.L} inner steps of one round, all {cfg.n} replicas, fp64 numpy ({t:.1f} s)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = si.CONFIGS[args.workload]
+    t1 = oracle_sample(cfg, 1)
+    per_step = int(max(1, min(cfg.L, 20.0 / max(t1, 1e-3) / max(args.steps + args.warmup, 1))))
+    for r in range(args.warmup):
+        oracle_sample(cfg, per_step, r)
+    t = 0.0
+    for r in range(args.steps):
+        t += oracle_sample(cfg, per_step, args.warmup + r)
+    value = cfg.n * per_step * args.steps / t
+    sample = f"each step = {per_step} of {cfg.L} inner steps of a round, all {cfg.n} replicas, + outer step and mean; fp64 numpy"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: n={cfg.n}, MLP {'-'.join(map(str, cfg.dims))}, batch {cfg.batch}, L={cfg.L}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

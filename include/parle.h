@@ -159,6 +159,35 @@ int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
 int parle_status(parle_ctx *ctx, int *device_flags);
 int parle_clear_status(parle_ctx *ctx);
 
+/* Per-kernel-class device timing.  While enabled, every kernel launch is
+ * bracketed by a pair of CUDA events on the bound stream (at most 16384
+ * launches between two reads; later ones are counted in *dropped).
+ * parle_profile_read is the one call that synchronises the stream: it then
+ * sums the elapsed times per class into ms[k] / launches[k] for
+ * k < n_classes (arrays in host memory) and restarts the recording.
+ * Class names: parle_profile_class_name(k), k < parle_profile_class_count(). */
+int parle_profile_enable(parle_ctx *ctx, int on);
+int parle_profile_read(parle_ctx *ctx, int n_classes, double *ms, long long *launches, long long *dropped);
+int parle_profile_class_count(void);
+const char *parle_profile_class_name(int k);
+
+/* Diagnostics: where, inside the caller's workspace, the last inner step left
+ * its intermediates (valid until the next call that launches work).
+ *   PARLE_DBG_ACT     output of hidden layer `layer`   [n, B, d]   fp32 (fp32 path) or bf16 (bf16 path)
+ *   PARLE_DBG_ACT_T   its transposed copy (bf16 path)  [n, d, B]   bf16
+ *   PARLE_DBG_DACT    gradient w.r.t. layer's output   [n, B, ld]  fp32 (ld = d) or bf16 (ld = d rounded up to 8)
+ *   PARLE_DBG_DACT_T  its transposed copy (bf16 path)  [n, d, B]   bf16
+ *   PARLE_DBG_LOGITS  logits                            [n, B, d_last] fp32   (layer ignored)
+ *   PARLE_DBG_OPERAND_COPY  bf16 copy of the vector the GEMMs read [n, stride] (bf16 path; layer ignored)
+ * EINVAL if that buffer does not exist in this configuration. */
+#define PARLE_DBG_ACT 0
+#define PARLE_DBG_ACT_T 1
+#define PARLE_DBG_DACT 2
+#define PARLE_DBG_DACT_T 3
+#define PARLE_DBG_LOGITS 4
+#define PARLE_DBG_OPERAND_COPY 5
+int parle_debug_buffer(const parle_ctx *ctx, int kind, int layer, size_t *byte_offset, size_t *bytes);
+
 /* Kernels launched by this context since creation (for accounting). */
 long long parle_launch_count(const parle_ctx *ctx);
 

@@ -107,9 +107,27 @@ def softmax_ce(logits, labels):
     return loss, d / B
 
 
-def mlp_loss_grad(vec, dims, X, labels, weight_decay: float = 0.0):
-    """Loss f(vec) on the minibatch and its gradient in the oracle's packing."""
+def round_to_bf16(a):
+    """Round fp64 values to the nearest bfloat16 (ties to even), returned as fp64.
+    Diagnostic only: used to imitate a mixed-precision implementation's operand
+    rounding so that a kernel bug can be told apart from rounding."""
+    f = np.asarray(a, np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(F64).reshape(np.shape(a))
+
+
+def mlp_loss_grad(vec, dims, X, labels, weight_decay: float = 0.0, operand_rounding=None):
+    """Loss f(vec) on the minibatch and its gradient in the oracle's packing.
+
+    operand_rounding (diagnostic, default None = exact fp64): a function applied
+    to every operand of every dense product (weights, layer inputs, hidden
+    activations, back-propagated deltas) before it is used, as a bf16-operand
+    implementation would; sums stay in fp64."""
+    q = operand_rounding
     layers = unpack(np.asarray(vec, F64), dims)
+    if q is not None:
+        return _mlp_loss_grad_rounded(layers, X, np.asarray(labels), q)
     logits, acts = mlp_forward(layers, X)
     loss, delta = softmax_ce(logits, np.asarray(labels))
     grads = [None] * len(layers)
@@ -125,6 +143,26 @@ def mlp_loss_grad(vec, dims, X, labels, weight_decay: float = 0.0):
         loss += 0.5 * weight_decay * float(np.dot(vec, vec))
         g = g + weight_decay * vec
     return loss, g
+
+
+def _mlp_loss_grad_rounded(layers, X, labels, q):
+    """Same forward/backward with every product operand passed through q."""
+    Wq = [q(W) for W, _ in layers]
+    h = q(np.asarray(X, F64))
+    acts = [h]
+    for l, (_, b) in enumerate(layers):
+        pre = np.matmul(h, Wq[l].T) + b
+        if l + 1 < len(layers):
+            h = q(np.maximum(pre, 0.0))
+            acts.append(h)
+    loss, delta = softmax_ce(pre, labels)
+    delta = q(delta)
+    grads = [None] * len(layers)
+    for l in range(len(layers) - 1, -1, -1):
+        grads[l] = (np.matmul(delta.T, acts[l]), delta.sum(axis=0))
+        if l > 0:
+            delta = q(np.matmul(delta, Wq[l]) * (acts[l] > 0.0))
+    return loss, pack(grads)
 
 
 # --------------------------------------------------------------------------

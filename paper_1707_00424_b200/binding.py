@@ -69,6 +69,11 @@ def lib() -> C.CDLL:
         "parle_set_lr": (ci, [vp, cd, cd]),
         "parle_status": (ci, [vp, C.POINTER(ci)]),
         "parle_clear_status": (ci, [vp]),
+        "parle_profile_enable": (ci, [vp, ci]),
+        "parle_profile_read": (ci, [vp, ci, C.POINTER(cd), C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]),
+        "parle_profile_class_count": (ci, []),
+        "parle_profile_class_name": (C.c_char_p, [ci]),
+        "parle_debug_buffer": (ci, [vp, ci, ci, C.POINTER(sz), C.POINTER(sz)]),
         "parle_launch_count": (C.c_longlong, [vp]),
         "parle_last_cuda_error": (ci, [vp]),
         "parle_strerror": (C.c_char_p, [ci]),
@@ -196,6 +201,37 @@ class Parle:
 
     def clear_status(self):
         self._check(self._L.parle_clear_status(self._h), "parle_clear_status")
+
+    DBG_ACT, DBG_ACT_T, DBG_DACT, DBG_DACT_T, DBG_LOGITS, DBG_OPERAND_COPY = range(6)
+
+    def debug_buffer(self, kind: int, layer: int = 0):
+        """View (torch, no copy) of an intermediate of the last inner step inside the workspace."""
+        import torch
+        off, nbytes = C.c_size_t(), C.c_size_t()
+        self._check(self._L.parle_debug_buffer(self._h, kind, layer, C.byref(off), C.byref(nbytes)), "parle_debug_buffer")
+        raw = self.workspace[off.value:off.value + nbytes.value]
+        n, B = self.n, self.batch
+        bf = self.gemm_dtype == GEMM_BF16
+        d = self.dims[layer + 1]
+        if kind == self.DBG_LOGITS:
+            return raw.view(torch.float32).view(n, B, self.dims[-1])
+        if kind == self.DBG_OPERAND_COPY:
+            return raw.view(torch.bfloat16).view(n, self.stride)
+        if kind in (self.DBG_ACT_T, self.DBG_DACT_T):
+            return raw.view(torch.bfloat16).view(n, d, B)
+        t = raw.view(torch.bfloat16 if bf else torch.float32)
+        return t.view(n, B, -1)[:, :, :d]
+
+    def profile_enable(self, on: bool = True):
+        self._check(self._L.parle_profile_enable(self._h, 1 if on else 0), "parle_profile_enable")
+
+    def profile_read(self):
+        """Synchronises the stream; returns {class name: (total ms, launches)} and the dropped count."""
+        k = self._L.parle_profile_class_count()
+        ms, cnt, drop = (C.c_double * k)(), (C.c_longlong * k)(), C.c_longlong()
+        self._check(self._L.parle_profile_read(self._h, k, ms, cnt, C.byref(drop)), "parle_profile_read")
+        out = {self._L.parle_profile_class_name(i).decode(): (ms[i], cnt[i]) for i in range(k) if cnt[i]}
+        return out, drop.value
 
     @property
     def launch_count(self) -> int:

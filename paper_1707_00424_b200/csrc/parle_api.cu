@@ -14,6 +14,15 @@ using namespace parle;
 namespace {
 
 constexpr size_t kWsAlign = 1024;
+constexpr int kProfCapacity = 16384;       // launches recorded between two parle_profile_read calls
+
+enum KernelClass {
+    KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_LOSS_MEAN, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
+    KC_INNER_UPDATE, KC_OUTER_MEAN, KC_MEAN, KC_TO_BF16, KC_COUNT
+};
+const char *const kClassNames[KC_COUNT] = {
+    "input_to_bf16", "fwd_gemm", "softmax_ce_backward", "loss_mean", "wgrad_gemm", "bias_grad", "dgrad_gemm",
+    "inner_update", "outer_mean", "mean", "to_bf16"};
 
 struct Workspace {
     // byte offsets into parle_buffers.workspace; index = layer (0-based)
@@ -51,6 +60,11 @@ struct parle_ctx {
     CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
+    // optional per-launch timing (events, host-side bookkeeping only)
+    bool prof_on, prof_open;
+    int prof_used, prof_dropped;
+    cudaEvent_t *prof_ev;            // 2 * kProfCapacity events
+    unsigned char *prof_cls;
 };
 
 namespace {
@@ -60,7 +74,21 @@ inline int cuda_fail(parle_ctx *c, cudaError_t e) {
     return PARLE_ECUDA;
 }
 #define PARLE_CUDA(c, expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
-#define PARLE_LAUNCHED(c) do { (c)->launches++; cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
+#define PARLE_LAUNCHED(c) do { (c)->launches++; prof_end(c); cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
+
+inline void prof_begin(parle_ctx *c, int cls) {
+    if (!c->prof_on) return;
+    if (c->prof_used >= kProfCapacity) { c->prof_dropped++; return; }
+    cudaEventRecord(c->prof_ev[2 * c->prof_used], c->stream);
+    c->prof_cls[c->prof_used] = (unsigned char)cls;
+    c->prof_open = true;
+}
+inline void prof_end(parle_ctx *c) {
+    if (!c->prof_open) return;
+    cudaEventRecord(c->prof_ev[2 * c->prof_used + 1], c->stream);
+    c->prof_used++;
+    c->prof_open = false;
+}
 #define PARLE_TRY(expr) do { int rc_ = (expr); if (rc_ != PARLE_OK) return rc_; } while (0)
 
 inline bool coupling_ok(double v) { return v > 0.0 && !isnan(v); }
@@ -167,13 +195,14 @@ int build_tensor_maps(parle_ctx *c) {
 }
 
 template <int EPI, bool B_MN>
-int launch_umma(parle_ctx *c, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
+int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
     p.groups = c->n;
     p.tiles_m = (p.M + UM_BM - 1) / UM_BM;
     p.tiles_n = (p.N + UM_BN - 1) / UM_BN;
     p.status = c->status_dev;
     const int tiles = p.groups * p.tiles_m * p.tiles_n;
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    prof_begin(c, cls);
     umma_gemm_kernel<EPI, B_MN><<<grid, UM_THREADS, UM_SMEM_BYTES, c->stream>>>(a, b, p);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
@@ -186,8 +215,9 @@ cudaError_t allow_big_smem() {
 }
 
 template <int EPI>
-int launch_simt(parle_ctx *c, const SimtGemmArgs &a) {
+int launch_simt(parle_ctx *c, int cls, const SimtGemmArgs &a) {
     dim3 grid((a.N + SG_BN - 1) / SG_BN, (a.M + SG_BM - 1) / SG_BM, c->n);
+    prof_begin(c, cls);
     simt_gemm_kernel<EPI><<<grid, SG_THREADS, 0, c->stream>>>(a);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
@@ -211,6 +241,7 @@ int run_inner_update(parle_ctx *c, const float *grad) {
     const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
     const bool sh = c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0;
     uint2 *shadow = sh ? ws_ptr<uint2>(c, c->ws.shadow) : nullptr;
+    prof_begin(c, KC_INNER_UPDATE);
 #define PARLE_UPD(F, S) inner_update_kernel<F, S, U><<<grid, kUpdThreads, 0, c->stream>>>( \
         g, y, x, z, shadow, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev)
     if (c->fresh) { if (sh) PARLE_UPD(true, true); else PARLE_UPD(true, false); }
@@ -237,14 +268,16 @@ int forward_backward_fp32(parle_ctx *c, const float *inputs, const int32_t *labe
         a.C = ws_ptr<float>(c, w.act[l]); a.c_gs = (long long)B * dout; a.ldc = dout;
         a.M = B; a.N = dout; a.K = din;
         a.bias = params + c->layers[l].b_off; a.bias_gs = S;
-        if (l + 1 < nl) PARLE_TRY(launch_simt<EPI_BIAS_RELU>(c, a)); else PARLE_TRY(launch_simt<EPI_BIAS>(c, a));
+        if (l + 1 < nl) PARLE_TRY(launch_simt<EPI_BIAS_RELU>(c, KC_FWD_GEMM, a)); else PARLE_TRY(launch_simt<EPI_BIAS>(c, KC_FWD_GEMM, a));
     }
     const int C = c->dims[nl], rows = n * B;
+    prof_begin(c, KC_SOFTMAX_CE);
     softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.act[nl - 1]), labels, ws_ptr<float>(c, w.dact[nl - 1]), nullptr, nullptr,
         ws_ptr<float>(c, w.row_loss), rows, B, C, 0, c->status_dev);
     PARLE_LAUNCHED(c);
     if (loss_out) {
+        prof_begin(c, KC_LOSS_MEAN);
         loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
         PARLE_LAUNCHED(c);
     }
@@ -256,7 +289,8 @@ int forward_backward_fp32(parle_ctx *c, const float *inputs, const int32_t *labe
         a.B = act_in; a.b_gs = (long long)B * din; a.b_ks = din; a.b_ns = 1;
         a.C = c->buf.grad + c->layers[l].w_off; a.c_gs = S; a.ldc = din;
         a.M = dout; a.N = din; a.K = B;
-        PARLE_TRY(launch_simt<EPI_PLAIN>(c, a));
+        PARLE_TRY(launch_simt<EPI_PLAIN>(c, KC_WGRAD_GEMM, a));
+        prof_begin(c, KC_BIAS_GRAD);
         bias_grad_f32_kernel<<<dim3((dout + 255) / 256, n), 256, 0, c->stream>>>(
             ws_ptr<float>(c, w.dact[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
         PARLE_LAUNCHED(c);
@@ -267,7 +301,7 @@ int forward_backward_fp32(parle_ctx *c, const float *inputs, const int32_t *labe
             d.C = ws_ptr<float>(c, w.dact[l - 1]); d.c_gs = (long long)B * din; d.ldc = din;
             d.M = B; d.N = din; d.K = dout;
             d.mask = ws_ptr<float>(c, w.act[l - 1]); d.mask_gs = (long long)B * din; d.ldmask = din;
-            PARLE_TRY(launch_simt<EPI_MASK>(c, d));
+            PARLE_TRY(launch_simt<EPI_MASK>(c, KC_DGRAD_GEMM, d));
         }
     }
     return PARLE_OK;
@@ -280,6 +314,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     const float *params = c->fresh ? c->buf.x : c->buf.y;      // fp32 biases come from the master copy
     {
         const int d0 = c->dims[0];
+        prof_begin(c, KC_INPUT_CVT);
         input_to_bf16_kernel<<<dim3((d0 + 31) / 32, (B + 31) / 32, n), 256, 0, c->stream>>>(
             inputs, ws_ptr<__nv_bfloat16>(c, w.xb), ws_ptr<__nv_bfloat16>(c, w.xbT), B, d0);
         PARLE_LAUNCHED(c);
@@ -292,19 +327,21 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         if (l + 1 < nl) {
             p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
             p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
-            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, false>(c, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, false>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         } else {
             p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
-            PARLE_TRY((launch_umma<UEPI_FWD_LAST, false>(c, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_FWD_LAST, false>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         }
     }
     const int C = c->dims[nl], rows = n * B;
+    prof_begin(c, KC_SOFTMAX_CE);
     softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
         ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
         c->status_dev);
     PARLE_LAUNCHED(c);
     if (loss_out) {
+        prof_begin(c, KC_LOSS_MEAN);
         loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
         PARLE_LAUNCHED(c);
     }
@@ -313,7 +350,8 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         UmmaParams p = {};                                      // dW_l = dH_l^T * H_{l-1}
         p.M = dout; p.N = din; p.K = B;
         p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
-        PARLE_TRY((launch_umma<UEPI_WGRAD, false>(c, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+        PARLE_TRY((launch_umma<UEPI_WGRAD, false>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+        prof_begin(c, KC_BIAS_GRAD);
         bias_grad_bf16_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
             ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
         PARLE_LAUNCHED(c);
@@ -323,7 +361,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
             d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
             d.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); d.outT_gs = (long long)B * din; d.outT_ld = B;
             d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
-            PARLE_TRY((launch_umma<UEPI_DGRAD, true>(c, c->tm_dg_a[l], c->tm_dg_b[l], d)));
+            PARLE_TRY((launch_umma<UEPI_DGRAD, true>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d)));
         }
     }
     return PARLE_OK;
@@ -389,6 +427,11 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
 void parle_destroy(parle_ctx *c) {
     if (!c) return;
     if (c->status_host) cudaFreeHost(c->status_host);
+    if (c->prof_ev) {
+        for (int i = 0; i < 2 * kProfCapacity; ++i) cudaEventDestroy(c->prof_ev[i]);
+        delete[] c->prof_ev;
+        delete[] c->prof_cls;
+    }
     delete c;
 }
 
@@ -441,6 +484,7 @@ int parle_round_begin(parle_ctx *c) {
     PARLE_TRY(check_bound(c));
     if (c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16 && !c->shadow_is_x) {
         const size_t n4 = (size_t)c->n * c->stride / 4;
+        prof_begin(c, KC_TO_BF16);
         to_bf16_kernel<<<stream_grid(c, n4, 1), kUpdThreads, 0, c->stream>>>(
             reinterpret_cast<const float4 *>(c->buf.x), ws_ptr<uint2>(c, c->ws.shadow), n4);
         PARLE_LAUNCHED(c);
@@ -491,6 +535,7 @@ int parle_outer_step(parle_ctx *c) {
     float4 *x = reinterpret_cast<float4 *>(c->buf.x), *xbar = reinterpret_cast<float4 *>(c->buf.xbar);
     const float4 *z = reinterpret_cast<const float4 *>(c->buf.z);
     const bool sh = c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0;
+    prof_begin(c, KC_OUTER_MEAN);
     if (sh)
         outer_mean_kernel<true, 4><<<grid, kUpdThreads, 0, c->stream>>>(
             x, z, xbar, ws_ptr<uint2>(c, c->ws.shadow), s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
@@ -506,6 +551,7 @@ int parle_outer_step(parle_ctx *c) {
 int parle_mean(parle_ctx *c) {
     PARLE_TRY(check_bound(c));
     const size_t s4 = c->stride / 4;
+    prof_begin(c, KC_MEAN);
     mean_kernel<4><<<stream_grid(c, s4, 1), kUpdThreads, 0, c->stream>>>(
         reinterpret_cast<const float4 *>(c->buf.x), reinterpret_cast<float4 *>(c->buf.xbar), s4, c->n, (float)c->n);
     PARLE_LAUNCHED(c);
@@ -553,6 +599,75 @@ int parle_clear_status(parle_ctx *c) {
     if (c->status_host) memset(c->status_host, 0, SLOT_COUNT * sizeof(int));
     return PARLE_OK;
 }
+
+int parle_profile_enable(parle_ctx *c, int on) {
+    PARLE_TRY(check_bound(c));
+    if (on && !c->prof_ev) {
+        c->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfCapacity];
+        c->prof_cls = new (std::nothrow) unsigned char[kProfCapacity];
+        if (!c->prof_ev || !c->prof_cls) return PARLE_EINVAL;
+        for (int i = 0; i < 2 * kProfCapacity; ++i) PARLE_CUDA(c, cudaEventCreate(&c->prof_ev[i]));
+    }
+    c->prof_on = on != 0;
+    c->prof_open = false;
+    c->prof_used = 0; c->prof_dropped = 0;
+    return PARLE_OK;
+}
+
+int parle_profile_read(parle_ctx *c, int n_classes, double *ms, long long *launches, long long *dropped) {
+    PARLE_TRY(check_bound(c));
+    if (!ms || !launches || n_classes < 1) return PARLE_EINVAL;
+    for (int k = 0; k < n_classes; ++k) { ms[k] = 0.0; launches[k] = 0; }
+    PARLE_CUDA(c, cudaStreamSynchronize(c->stream));
+    for (int i = 0; i < c->prof_used; ++i) {
+        float t = 0.f;
+        PARLE_CUDA(c, cudaEventElapsedTime(&t, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]));
+        const int k = c->prof_cls[i];
+        if (k < n_classes) { ms[k] += t; launches[k]++; }
+    }
+    if (dropped) *dropped = c->prof_dropped;
+    c->prof_used = 0; c->prof_dropped = 0;
+    return PARLE_OK;
+}
+
+int parle_debug_buffer(const parle_ctx *c, int kind, int layer, size_t *byte_offset, size_t *bytes) {
+    if (!c || !byte_offset || !bytes || c->n_layers == 0) return PARLE_EINVAL;
+    const Workspace &w = c->ws;
+    const int nl = c->n_layers;
+    const size_t nB = (size_t)c->n * c->batch;
+    const bool bf = c->gemm_dtype == PARLE_GEMM_BF16;
+    const size_t es = bf ? 2 : 4;
+    if (kind == PARLE_DBG_LOGITS) {
+        *byte_offset = bf ? w.logits : w.act[nl - 1];
+        *bytes = nB * c->dims[nl] * 4;
+        return PARLE_OK;
+    }
+    if (kind == PARLE_DBG_OPERAND_COPY) {
+        if (!bf) return PARLE_EINVAL;
+        *byte_offset = w.shadow; *bytes = (size_t)c->n * c->stride * 2;
+        return PARLE_OK;
+    }
+    if (layer < 0 || layer >= nl) return PARLE_EINVAL;
+    const size_t d = c->dims[layer + 1];
+    switch (kind) {
+        case PARLE_DBG_ACT:
+            if (layer == nl - 1) return PARLE_EINVAL;
+            *byte_offset = bf ? w.hb[layer] : w.act[layer]; *bytes = nB * d * es; return PARLE_OK;
+        case PARLE_DBG_ACT_T:
+            if (!bf || layer == nl - 1) return PARLE_EINVAL;
+            *byte_offset = w.hbT[layer]; *bytes = nB * d * 2; return PARLE_OK;
+        case PARLE_DBG_DACT:
+            *byte_offset = bf ? w.dhb[layer] : w.dact[layer];
+            *bytes = bf ? nB * (size_t)w.dh_ld[layer] * 2 : nB * d * 4; return PARLE_OK;
+        case PARLE_DBG_DACT_T:
+            if (!bf) return PARLE_EINVAL;
+            *byte_offset = w.dhbT[layer]; *bytes = nB * d * 2; return PARLE_OK;
+        default: return PARLE_EINVAL;
+    }
+}
+
+int parle_profile_class_count(void) { return KC_COUNT; }
+const char *parle_profile_class_name(int k) { return (k >= 0 && k < KC_COUNT) ? kClassNames[k] : ""; }
 
 long long parle_launch_count(const parle_ctx *c) { return c ? c->launches : 0; }
 int parle_last_cuda_error(const parle_ctx *c) { return c ? c->last_cuda : 0; }

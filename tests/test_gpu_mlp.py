@@ -70,7 +70,8 @@ def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False):
         disp = rel_l2(x_gpu - xo, out["x"] - xo)
         if disp_tol is not None:
             assert disp <= disp_tol, disp
-        np.testing.assert_allclose(loss.cpu().numpy(), out["loss"], rtol=50 * tol, atol=1e-5)
+        np.testing.assert_allclose(loss[0].cpu().numpy(), out["loss"][0], rtol=50 * tol, atol=1e-5)
+        np.testing.assert_allclose(loss.cpu().numpy(), out["loss"], rtol=0.05, atol=1e-4)
         assert torch.all(m.x[:, pad] == 0) and torch.all(m.xbar[pad] == 0)
         # invariant of Section 3.1: xbar is the mean of the current replicas
         np.testing.assert_allclose(xb_gpu, x_gpu.mean(axis=0), rtol=1e-5, atol=1e-6)
@@ -78,8 +79,18 @@ def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False):
     return m
 
 
-def grad_check(cfg, tol):
-    """One inner step: the gradient buffer against the oracle's gradient, layer by layer."""
+def grad_check(cfg, tol, loose=None, outliers=0):
+    """One inner step: the gradient buffer against the oracle's gradient, layer by layer.
+
+    bf16 GEMMs: a ReLU unit whose pre-activation lies within operand rounding of
+    zero can switch, and each switched unit changes the layers below by a full
+    term (relative L2 ~ sqrt(fraction switched), several per cent at width 2048),
+    although the parameters after a round stay within 2e-2.  So the tight check
+    (`tol`) is against the oracle with its product operands rounded to bf16
+    where the kernels round theirs, and the exact oracle gets `loose`.
+    fp32 GEMMs at full width: one unit within fp32 rounding of zero (probability
+    ~1e-7 per unit and sample, ~1e6 units per step) switches now and then; up to
+    `outliers` replicas may exceed `tol` and must then stay within 1e-2."""
     m, xo, xb, hp = make(cfg)
     X, c = si.round_batches(cfg.scaled(L=1), 0)
     loss = torch.zeros(cfg.n, device=DEV)
@@ -87,16 +98,26 @@ def grad_check(cfg, tol):
     torch.cuda.synchronize()
     assert m.status() == 0
     g_gpu = to_dense(m, m.grad.cpu().numpy())
+    over = 0
     for a in range(cfg.n):
-        lo, g = po.mlp_loss_grad(xo[a], cfg.dims, X[0, a], c[0, a])
-        assert abs(loss[a].item() - lo) <= 20 * tol * max(1.0, abs(lo)), (a, loss[a].item(), lo)
-        got, want = po.unpack(g_gpu[a], cfg.dims), po.unpack(g, cfg.dims)
-        errs = {}
-        for l, ((gW, gb), (wW, wb)) in enumerate(zip(got, want)):
-            errs[f"dW{l}"] = rel_l2(gW, wW)
-            errs[f"db{l}"] = rel_l2(gb, wb)
-        print(cfg.name, "replica", a, {k: f"{v:.2e}" for k, v in errs.items()})
-        assert max(errs.values()) <= tol, (a, errs)
+        if cfg.gemm_dtype == pb.GEMM_BF16:
+            passes = [(po.round_to_bf16, tol)] + ([(None, loose)] if loose is not None else [])
+        else:
+            passes = [(None, tol)]
+        for rounding, bound in passes:
+            lo, g = po.mlp_loss_grad(xo[a], cfg.dims, X[0, a], c[0, a], operand_rounding=rounding)
+            assert abs(loss[a].item() - lo) <= 20 * bound * max(1.0, abs(lo)), (a, loss[a].item(), lo)
+            got, want = po.unpack(g_gpu[a], cfg.dims), po.unpack(g, cfg.dims)
+            errs = {}
+            for l, ((gW, gb), (wW, wb)) in enumerate(zip(got, want)):
+                errs[f"dW{l}"] = rel_l2(gW, wW)
+                errs[f"db{l}"] = rel_l2(gb, wb)
+            print(cfg.name, "replica", a, "rounded" if rounding else "exact", {k: f"{v:.2e}" for k, v in errs.items()})
+            if outliers and max(errs.values()) > bound:
+                over += 1
+                assert max(errs.values()) <= 1e-2 and over <= outliers, (a, over, errs)
+            else:
+                assert max(errs.values()) <= bound, (a, errs)
     return m
 
 
@@ -172,7 +193,7 @@ def test_host_buffer_step_matches_device_step():
 
 
 def test_c2_gradient_full_shape_fp32():
-    grad_check(si.C2, 1e-5)
+    grad_check(si.C2, 1e-5, outliers=1)
 
 
 def test_c2_one_round_fp32():
@@ -181,12 +202,12 @@ def test_c2_one_round_fp32():
 
 # ------------------------------------------------------------------ bf16 GEMMs (tcgen05)
 def test_small_gradient_bf16():
-    grad_check(si.C1.scaled(name="bf16-small", dims=(64, 128, 72, 10), batch=16, gemm_dtype=1), 4e-2)
+    grad_check(si.C1.scaled(name="bf16-small", dims=(64, 128, 72, 10), batch=16, gemm_dtype=1), 5e-3, loose=0.15)
 
 
 def test_ragged_tiles_gradient_bf16():
     # several 128-tiles with tails in every dimension, K tails, last width not a multiple of 8
-    grad_check(si.C1.scaled(name="bf16-ragged", n=2, dims=(200, 328, 136, 101), batch=136, gemm_dtype=1), 4e-2)
+    grad_check(si.C1.scaled(name="bf16-ragged", n=2, dims=(200, 328, 136, 101), batch=136, gemm_dtype=1), 5e-3, loose=0.15)
 
 
 def test_small_rounds_bf16():
@@ -199,8 +220,70 @@ def test_c3_scaled_down_round_bf16():
 
 
 def test_c3_gradient_full_shape_bf16():
-    grad_check(si.C3.scaled(n=2), 4e-2)
+    grad_check(si.C3.scaled(n=2), 4e-2, loose=0.15)
 
 
 def test_c3_full_round_bf16():
     run_rounds(si.C3, 1, disp_tol=5e-2, use_round_call=True)
+
+
+def _layerwise_bf16(cfg):
+    """Every GEMM of one inner step checked on its own: each layer's result is
+    recomputed in fp64 from the operands the GPU itself used (read back from the
+    workspace), so that ReLU switching cannot accumulate across layers.
+    Allowed differences: a bf16 result one unit in the last place off where the
+    fp32-accumulated value sits on a rounding tie."""
+    m, xo, xb, hp = make(cfg)
+    X, c = si.round_batches(cfg.scaled(L=1), 0)
+    m.round_begin()
+    m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV))
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    q, nl, B = po.round_to_bf16, cfg.n_layers, cfg.batch
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    H = [f64(m.debug_buffer(m.DBG_ACT, l)) for l in range(nl - 1)]
+    HT = [f64(m.debug_buffer(m.DBG_ACT_T, l)) for l in range(nl - 1)]
+    dH = [f64(m.debug_buffer(m.DBG_DACT, l)) for l in range(nl)]
+    dHT = [f64(m.debug_buffer(m.DBG_DACT_T, l)) for l in range(nl)]
+    logits = f64(m.debug_buffer(m.DBG_LOGITS))
+    shadow = f64(m.debug_buffer(m.DBG_OPERAND_COPY))
+    # the operand copy now holds bf16(y) after the update; the step itself used bf16(x)
+    grad = m.grad.cpu().numpy().astype(np.float64)
+
+    def ulp_close(got, want, what):
+        diff = got != want
+        assert diff.mean() < 5e-3, (what, diff.mean())
+        # one bf16 unit in the last place, or (next to zero) the fp32 accumulation error itself
+        slack = 2.0 ** -7 * np.abs(want) + 1e-5 * np.sqrt(np.mean(want ** 2))
+        assert np.all(np.abs(got - want) <= slack), (what, np.max(np.abs(got - want) / slack))
+
+    for a in range(cfg.n):
+        layers = po.unpack(xo[a], cfg.dims)
+        Wq = [q(W) for W, _ in layers]
+        h = q(X[0, a].astype(np.float64))
+        inputs = [h]
+        for l in range(nl - 1):
+            ulp_close(H[l][a], q(np.maximum(h @ Wq[l].T + layers[l][1], 0.0)), f"H{l}")
+            assert np.array_equal(HT[l][a].T, H[l][a])
+            h = H[l][a]
+            inputs.append(h)
+        pre = h @ Wq[-1].T + layers[-1][1]
+        assert rel_l2(logits[a], pre) < 1e-5
+        _, d = po.softmax_ce(logits[a], c[0, a])
+        ulp_close(dH[nl - 1][a], q(d), "dlogits")
+        for l in range(nl - 1, -1, -1):
+            assert np.array_equal(dHT[l][a].T, dH[l][a])
+            w_off, b_off = m.layer_offset(l)
+            dW = grad[a, w_off:w_off + cfg.dims[l + 1] * cfg.dims[l]].reshape(cfg.dims[l + 1], cfg.dims[l])
+            assert rel_l2(dW, dH[l][a].T @ inputs[l]) < 1e-5, ("dW", l)
+            assert rel_l2(grad[a, b_off:b_off + cfg.dims[l + 1]], dH[l][a].sum(axis=0)) < 1e-5, ("db", l)
+            if l > 0:
+                ulp_close(dH[l - 1][a], q((dH[l][a] @ Wq[l]) * (H[l - 1][a] > 0)), f"dH{l - 1}")
+
+
+def test_layerwise_teacher_forced_c3_bf16():
+    _layerwise_bf16(si.C3.scaled(n=2))
+
+
+def test_layerwise_teacher_forced_ragged_bf16():
+    _layerwise_bf16(si.C1.scaled(name="bf16-ragged", n=2, dims=(200, 328, 136, 101), batch=136, gemm_dtype=1))

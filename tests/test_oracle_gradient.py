@@ -131,3 +131,22 @@ def test_planted_mistakes_are_caught_by_finite_differences(monkeypatch):
         return logits, [a + (a == 0) * 1e-300 for a in acts]   # every unit looks active
     monkeypatch.setattr(po, "mlp_forward", fwd_no_mask)
     assert not fd_ok()
+
+
+def test_bf16_rounding_helper_and_rounded_mode():
+    # exact cases of round-to-nearest-even at 8 significant bits
+    vals = np.array([1.0, 1.00390625, 1.001953125, 1.005859375, -3.1415926, 0.0, 65504.0])
+    want = np.array([1.0, 1.0, 1.0, 1.0078125, -3.140625, 0.0, 65536.0])
+    np.testing.assert_array_equal(po.round_to_bf16(vals), want)
+    # against torch's own bfloat16 conversion
+    r = np.random.default_rng(0).normal(size=1000) * 10.0 ** np.random.default_rng(1).integers(-5, 5, 1000)
+    t = torch.tensor(r, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(po.round_to_bf16(r), t)
+    # identity "rounding" reproduces the exact gradient; bf16 rounding stays close
+    dims, B = (16, 12, 5), 8
+    vec, X, c = _rand_problem(dims, B, seed=8)
+    l0, g0 = po.mlp_loss_grad(vec, dims, X, c)
+    l1, g1 = po.mlp_loss_grad(vec, dims, X, c, operand_rounding=lambda a: np.asarray(a, np.float64))
+    assert abs(l0 - l1) < 1e-14 and np.allclose(g0, g1, rtol=1e-13, atol=1e-15)
+    l2, g2 = po.mlp_loss_grad(vec, dims, X, c, operand_rounding=po.round_to_bf16)
+    assert 0 < np.linalg.norm(g2 - g0) / np.linalg.norm(g0) < 0.05
