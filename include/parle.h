@@ -45,6 +45,7 @@ extern "C" {
 #define PARLE_ESTATE       -5   /* call out of order (e.g. inner step before parle_round_begin) */
 #define PARLE_EWORKSPACE   -6   /* workspace smaller than parle_workspace_bytes() */
 #define PARLE_EUNSUPPORTED -7   /* shape not supported by the requested GEMM path */
+#define PARLE_ETOOBIG      -8   /* size beyond the fixed capacity of an allocation-free entry point */
 
 /* bits of the device status word, see parle_status() */
 #define PARLE_FLAG_NONFINITE   1   /* an update kernel produced a NaN or Inf */
@@ -187,6 +188,37 @@ const char *parle_profile_class_name(int k);
 #define PARLE_DBG_LOGITS 4
 #define PARLE_DBG_OPERAND_COPY 5
 int parle_debug_buffer(const parle_ctx *ctx, int kind, int layer, size_t *byte_offset, size_t *bytes);
+
+/* Allocation-free loss step (the paper has no counterpart: this is a packaging
+ * variant of the loss part of parle_inner_step, not a step of the method).
+ *
+ * Who it is for: callers that can neither allocate device memory nor hand the
+ * library a workspace -- a plug-in running inside another framework's fixed
+ * memory pool, a component whose device memory budget was fully assigned at
+ * start-up, code on a path where calling the device allocator is forbidden
+ * (it may synchronise or fail).  Such a caller still owns its inputs and outputs.
+ *
+ * What it does: for n replicas with B rows each, row-wise softmax cross-entropy
+ *   dlogits[r, :] = (softmax(logits[r, :]) - onehot(labels[r])) / B,   loss[a] = mean over replica a's rows,
+ * exactly the kernels parle_inner_step runs after the last layer.
+ *   logits  dev [n*B, C] fp32 (in)     labels dev [n*B] int32 (in)
+ *   dlogits dev [n*B, C] fp32 (out)    loss   dev [n] fp32 (out)
+ *   flags   dev [1] int32 (out) or NULL: non-zero if a label was outside [0, C)
+ * The per-row losses, which parle_inner_step keeps in the caller's workspace,
+ * live here in a fixed array inside the library image: PARLE_STATIC_LOSS_MAX_ROWS
+ * floats + 256 bytes (about 256 KiB), present on every GPU that loads the library
+ * until the process exits.  n*B beyond that limit returns PARLE_ETOOBIG.
+ * The function calls no device allocator of any kind.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current) and keeps it; make that first call before starting any stream
+ * capture.  All calls on a device share the one array: it keeps the previous
+ * call's contents (the flag slots are cleared at the start of every call), and
+ * two calls whose work overlaps on the GPU (different streams, no ordering) race.
+ * Work is enqueued on cuda_stream (cudaStream_t as void*, NULL = default). */
+#define PARLE_STATIC_LOSS_MAX_ROWS 65536
+int parle_softmax_ce_static(const float *logits, const int32_t *labels, int n, int B, int C,
+                            float *dlogits, float *loss, int32_t *flags, void *cuda_stream);
 
 /* Kernels launched by this context since creation (for accounting). */
 long long parle_launch_count(const parle_ctx *ctx);

@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         "parle_profile_class_count": (ci, []),
         "parle_profile_class_name": (C.c_char_p, [ci]),
         "parle_debug_buffer": (ci, [vp, ci, ci, C.POINTER(sz), C.POINTER(sz)]),
+        "parle_softmax_ce_static": (ci, [vp, vp, ci, ci, ci, vp, vp, vp, vp]),
         "parle_launch_count": (C.c_longlong, [vp]),
         "parle_last_cuda_error": (ci, [vp]),
         "parle_strerror": (C.c_char_p, [ci]),
@@ -92,6 +93,22 @@ def _ptr(t) -> int:
     if isinstance(t, int):
         return t
     return t.data_ptr()
+
+
+STATIC_LOSS_MAX_ROWS = 65536
+
+
+def softmax_ce_static(logits, labels, n: int, B: int, C_: int, dlogits, loss, flags=None, stream=None):
+    """Allocation-free loss step (parle_softmax_ce_static): for callers that cannot give the
+    library a workspace.  All arguments are caller-owned device tensors; nothing is allocated."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream(logits.device)
+    with torch.cuda.device(logits.device):
+        rc = lib().parle_softmax_ce_static(_ptr(logits), _ptr(labels), n, B, C_, _ptr(dlogits), _ptr(loss),
+                                           _ptr(flags), C.c_void_p(stream.cuda_stream))
+    if rc != 0:
+        raise ParleError(rc, "parle_softmax_ce_static")
 
 
 class Parle:

@@ -682,6 +682,7 @@ const char *parle_strerror(int code) {
         case PARLE_ESTATE: return "call out of order";
         case PARLE_EWORKSPACE: return "workspace too small";
         case PARLE_EUNSUPPORTED: return "shape or device not supported by this GEMM path";
+        case PARLE_ETOOBIG: return "size exceeds the fixed capacity of this allocation-free entry point";
         default: return "unknown error";
     }
 }
