@@ -150,6 +150,13 @@ int parle_mean(parle_ctx *ctx);
 int parle_round(parle_ctx *ctx, int L, const float *inputs, const int32_t *labels,
                 float *loss_out);
 
+/* bf16 path only.  on (the default): Eq. (parle_y), (parle_z) are applied
+ * inside the weight-gradient GEMM's epilogue, so the weight gradient is never
+ * written and `grad` is left untouched by parle_inner_step.  off: the gradient is
+ * written to `grad` and a separate update kernel follows (same results up to
+ * fp32 rounding).  EUNSUPPORTED on the fp32 path, ESTATE in the middle of a round. */
+int parle_set_fused_update(parle_ctx *ctx, int on);
+
 /* Change gamma, rho (Eq. scoping changes them between rounds) or the step
  * sizes eta, eta' between calls.  +INFINITY allowed for gamma and rho. */
 int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);

@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
         "parle_round": (ci, [vp, ci, vp, vp, vp]),
         "parle_set_coupling": (ci, [vp, cd, cd]),
         "parle_set_lr": (ci, [vp, cd, cd]),
+        "parle_set_fused_update": (ci, [vp, ci]),
         "parle_status": (ci, [vp, C.POINTER(ci)]),
         "parle_clear_status": (ci, [vp]),
         "parle_profile_enable": (ci, [vp, ci]),
@@ -210,6 +211,9 @@ class Parle:
 
     def set_lr(self, eta: float, eta_prime: float):
         self._check(self._L.parle_set_lr(self._h, eta, eta_prime), "parle_set_lr")
+
+    def set_fused_update(self, on: bool):
+        self._check(self._L.parle_set_fused_update(self._h, 1 if on else 0), "parle_set_fused_update")
 
     def status(self) -> int:
         f = C.c_int()

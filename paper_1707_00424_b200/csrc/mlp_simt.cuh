@@ -167,6 +167,48 @@ bias_grad_bf16_kernel(const __nv_bfloat16 *__restrict__ dHT, float *__restrict__
     if (lane == 0) grad[(long long)g * grad_gs + j] = s;
 }
 
+// Everything of a replica's vector that the weight tiles do not cover -- the
+// bias segments and the alignment padding after each segment -- gets its inner
+// update (Eq. parle_y, parle_z) here when the update of the weights is fused into
+// the weight-gradient GEMM.  One warp per element: for a bias element the warp
+// first forms db_j = sum_i dH^T[j, i] (bf16 transposed copy, fp32 sum); padding
+// has gradient 0 and stays 0.
+struct TailPlan {
+    int n_layers, batch;
+    long long begin[PARLE_MAX_LAYERS], b_off[PARLE_MAX_LAYERS], end[PARLE_MAX_LAYERS];   // element ranges in a replica
+    int d_out[PARLE_MAX_LAYERS];
+    const __nv_bfloat16 *dHT[PARLE_MAX_LAYERS];      // [n, d_out, B]
+};
+
+template <bool FIRST>
+__global__ void __launch_bounds__(256)
+tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__ z, const float *__restrict__ x,
+                   __nv_bfloat16 *__restrict__ shadow, long long stride, float eta_p, float inv_gamma,
+                   float alpha, int *status) {
+    const int l = blockIdx.y, g = blockIdx.z;
+    const int lane = threadIdx.x % 32;
+    const long long e = tp.begin[l] + (long long)blockIdx.x * 8 + threadIdx.x / 32;
+    if (e >= tp.end[l]) return;
+    float grad = 0.f;
+    const long long j = e - tp.b_off[l];
+    if (j >= 0 && j < tp.d_out[l]) {
+        const __nv_bfloat16 *p = tp.dHT[l] + ((long long)g * tp.d_out[l] + j) * tp.batch;
+        for (int i = lane; i < tp.batch; i += 32) grad += __bfloat162float(p[i]);
+        for (int o = 16; o > 0; o >>= 1) grad += __shfl_xor_sync(0xffffffffu, grad, o);
+    }
+    if (lane == 0) {
+        const long long i = (long long)g * stride + e;
+        const float xv = x[i];
+        const float yo = FIRST ? xv : y[i], zo = FIRST ? xv : z[i];
+        const float yn = yo - eta_p * fmaf(inv_gamma, yo - xv, grad);
+        const float zn = fmaf(alpha, zo, (1.0f - alpha) * yn);
+        y[i] = yn;
+        z[i] = zn;
+        shadow[i] = __float2bfloat16_rn(yn);
+        if (!(fabsf(yn) <= 3.402823466e+38f)) status[SLOT_NONFINITE] = 1;
+    }
+}
+
 // Minibatch inputs fp32 [n, B, d] -> bf16 [n, B, d] and its transpose [n, d, B]
 // (the K-major operand of the first layer's weight-gradient product).
 __global__ void __launch_bounds__(256)

@@ -18,11 +18,11 @@ constexpr int kProfCapacity = 16384;       // launches recorded between two parl
 
 enum KernelClass {
     KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_LOSS_MEAN, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
-    KC_INNER_UPDATE, KC_OUTER_MEAN, KC_MEAN, KC_TO_BF16, KC_COUNT
+    KC_INNER_UPDATE, KC_OUTER_MEAN, KC_MEAN, KC_TO_BF16, KC_WGRAD_UPDATE, KC_TAIL_UPDATE, KC_COUNT
 };
 const char *const kClassNames[KC_COUNT] = {
     "input_to_bf16", "fwd_gemm", "softmax_ce_backward", "loss_mean", "wgrad_gemm", "bias_grad", "dgrad_gemm",
-    "inner_update", "outer_mean", "mean", "to_bf16"};
+    "inner_update", "outer_mean", "mean", "to_bf16", "wgrad_gemm_fused_update", "tail_update"};
 
 struct Workspace {
     // byte offsets into parle_buffers.workspace; index = layer (0-based)
@@ -53,6 +53,7 @@ struct parle_ctx {
     cudaStream_t stream;
     int *status_host, *status_dev;
     bool round_open, fresh, shadow_is_x;
+    bool fused_update;               // bf16 path: apply Eq. (parle_y)/(parle_z) inside the weight-gradient GEMM
     int steps_in_round;
     long long launches;
     int last_cuda;
@@ -180,9 +181,10 @@ int build_tensor_maps(parle_ctx *c) {
         // forward: A = layer input [B, din], B = W [dout, din], both K-major (K = din)
         PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_a[l], a_in, din, B, n, din, B * din, UM_BK, UM_BM));
         PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_b[l], W, din, dout, n, din, c->stride, UM_BK, UM_BN));
-        // weight gradient: A = dH^T [dout, B], B = input^T [din, B], both K-major (K = batch)
-        PARLE_TRY(encode_bf16_map(c, &c->tm_wg_a[l], ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), B, dout, n, B, dout * B, UM_BK, UM_BM));
-        PARLE_TRY(encode_bf16_map(c, &c->tm_wg_b[l], a_inT, B, din, n, B, din * B, UM_BK, UM_BN));
+        // weight gradient, computed transposed (dW^T = input^T dH): A = input^T [din, B], B = dH^T [dout, B],
+        // both K-major (K = batch)
+        PARLE_TRY(encode_bf16_map(c, &c->tm_wg_a[l], a_inT, B, din, n, B, din * B, UM_BK, UM_BM));
+        PARLE_TRY(encode_bf16_map(c, &c->tm_wg_b[l], ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), B, dout, n, B, dout * B, UM_BK, UM_BN));
         if (l > 0) {
             // data gradient: A = dH [B, dout] K-major (K = dout); B = W [dout (K), din (N)] MN-major,
             // fetched as 64 k-rows x 64 n-columns boxes
@@ -203,7 +205,7 @@ int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &
     const int tiles = p.groups * p.tiles_m * p.tiles_n;
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     prof_begin(c, cls);
-    umma_gemm_kernel<EPI, B_MN><<<grid, UM_THREADS, UM_SMEM_BYTES, c->stream>>>(a, b, p);
+    umma_gemm_kernel<EPI, B_MN><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
@@ -345,25 +347,65 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
         PARLE_LAUNCHED(c);
     }
+    auto dgrad = [&](int l) -> int {                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        UmmaParams d = {};
+        d.M = B; d.N = din; d.K = dout;
+        d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
+        d.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); d.outT_gs = (long long)B * din; d.outT_ld = B;
+        d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
+        return launch_umma<UEPI_DGRAD, true>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d);
+    };
+    if (!c->fused_update) {
+        for (int l = nl - 1; l >= 0; --l) {
+            const int din = c->dims[l], dout = c->dims[l + 1];
+            UmmaParams p = {};                                  // dW_l^T = H_{l-1}^T * dH_l
+            p.M = din; p.N = dout; p.K = B;
+            p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
+            PARLE_TRY((launch_umma<UEPI_WGRAD, false>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+            prof_begin(c, KC_BIAS_GRAD);
+            bias_grad_bf16_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
+                ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
+            PARLE_LAUNCHED(c);
+            if (l > 0) PARLE_TRY(dgrad(l));
+        }
+        return PARLE_OK;
+    }
+    // Fused: the weight gradient never reaches memory.  dgrad(l) must read W_l before the fused
+    // kernel of layer l overwrites its bf16 copy, so it goes first.
+    __nv_bfloat16 *shadow = ws_ptr<__nv_bfloat16>(c, w.shadow);
     for (int l = nl - 1; l >= 0; --l) {
         const int din = c->dims[l], dout = c->dims[l + 1];
-        UmmaParams p = {};                                      // dW_l = dH_l^T * H_{l-1}
-        p.M = dout; p.N = din; p.K = B;
-        p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
-        PARLE_TRY((launch_umma<UEPI_WGRAD, false>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
-        prof_begin(c, KC_BIAS_GRAD);
-        bias_grad_bf16_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
-            ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
-        PARLE_LAUNCHED(c);
-        if (l > 0) {                                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
-            UmmaParams d = {};
-            d.M = B; d.N = din; d.K = dout;
-            d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
-            d.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); d.outT_gs = (long long)B * din; d.outT_ld = B;
-            d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
-            PARLE_TRY((launch_umma<UEPI_DGRAD, true>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d)));
-        }
+        if (l > 0) PARLE_TRY(dgrad(l));
+        UmmaParams p = {};
+        p.M = din; p.N = dout; p.K = B;
+        const size_t wo = c->layers[l].w_off;
+        p.upd_y = c->buf.y + wo; p.upd_z = c->buf.z + wo; p.upd_x = c->buf.x + wo; p.upd_shadow = shadow + wo;
+        p.upd_gs = S; p.upd_ld = din;
+        p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha;
+        if (c->fresh) PARLE_TRY((launch_umma<UEPI_WGRAD_UPDATE_FIRST, false>(c, KC_WGRAD_UPDATE, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+        else PARLE_TRY((launch_umma<UEPI_WGRAD_UPDATE, false>(c, KC_WGRAD_UPDATE, c->tm_wg_a[l], c->tm_wg_b[l], p)));
     }
+    TailPlan tp = {};
+    tp.n_layers = nl; tp.batch = B;
+    long long longest = 0;
+    for (int l = 0; l < nl; ++l) {
+        tp.begin[l] = (long long)c->layers[l].w_off + (long long)c->dims[l] * c->dims[l + 1];
+        tp.b_off[l] = (long long)c->layers[l].b_off;
+        tp.end[l] = l + 1 < nl ? (long long)c->layers[l + 1].w_off : (long long)c->stride;
+        tp.d_out[l] = c->dims[l + 1];
+        tp.dHT[l] = ws_ptr<__nv_bfloat16>(c, w.dhbT[l]);
+        if (tp.end[l] - tp.begin[l] > longest) longest = tp.end[l] - tp.begin[l];
+    }
+    const dim3 tgrid((unsigned)((longest + 7) / 8), nl, n);
+    prof_begin(c, KC_TAIL_UPDATE);
+    if (c->fresh)
+        tail_update_kernel<true><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, shadow, S,
+                                                               c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+    else
+        tail_update_kernel<false><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, shadow, S,
+                                                                c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+    PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
 
@@ -419,6 +461,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         }
     }
     c->P = P; c->stride = off;
+    c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
     plan_workspace(c);
     *out = c;
     return PARLE_OK;
@@ -472,6 +515,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, false>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD_UPDATE, false>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD_UPDATE_FIRST, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, true>()));
         PARLE_TRY(build_tensor_maps(c));
     }
@@ -498,8 +543,15 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
     PARLE_TRY(check_bound(c));
     if (c->n_layers == 0 || !inputs || !labels) return PARLE_EINVAL;
     if (!c->round_open) return PARLE_ESTATE;
-    if (c->gemm_dtype == PARLE_GEMM_BF16) PARLE_TRY(forward_backward_bf16(c, inputs, labels, loss_out));
-    else PARLE_TRY(forward_backward_fp32(c, inputs, labels, loss_out));
+    if (c->gemm_dtype == PARLE_GEMM_BF16) {
+        PARLE_TRY(forward_backward_bf16(c, inputs, labels, loss_out));
+        if (c->fused_update) {            // y, z and the operand copy were updated by the backward kernels
+            c->fresh = false; c->shadow_is_x = false; c->steps_in_round++;
+            return PARLE_OK;
+        }
+    } else {
+        PARLE_TRY(forward_backward_fp32(c, inputs, labels, loss_out));
+    }
     return run_inner_update(c, c->buf.grad);
 }
 
@@ -572,6 +624,14 @@ int parle_round(parle_ctx *c, int L, const float *inputs, const int32_t *labels,
 int parle_set_coupling(parle_ctx *c, double gamma, double rho) {
     if (!c || !coupling_ok(gamma) || !coupling_ok(rho)) return PARLE_EINVAL;
     c->inv_gamma = inverse_or_zero(gamma); c->inv_rho = inverse_or_zero(rho);
+    return PARLE_OK;
+}
+
+int parle_set_fused_update(parle_ctx *c, int on) {
+    if (!c) return PARLE_EINVAL;
+    if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
+    if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
+    c->fused_update = on != 0;
     return PARLE_OK;
 }
 

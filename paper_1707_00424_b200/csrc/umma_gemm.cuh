@@ -2,7 +2,9 @@
 // forward / backward (Section 1.1 / 2.1: the minibatch gradient of f):
 //   forward      H_l      = act(H_{l-1} W_l^T + b_l)           A=[B,d_in]   K-major, B=W [d_out,d_in] K-major
 //   data grad    dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]        A=[B,d_out]  K-major, B=W [d_out(K), d_in(N)] MN-major
-//   weight grad  dW_l     = dH_l^T H_{l-1}                     A=dH^T [d_out,B] K-major, B=H^T [d_in,B] K-major
+//   weight grad  dW_l^T   = H_{l-1}^T dH_l                     A=H^T [d_in,B] K-major, B=dH^T [d_out,B] K-major
+//                (computed transposed: accumulator rows = d_in, the contiguous direction of W in memory,
+//                 so the 32 lanes of an epilogue warp touch 32 consecutive floats of one W row)
 // One persistent CTA per SM walks (replica, m-tile, n-tile) work items.
 // Warp 0 stages 128x64 operand tiles with TMA (128-byte swizzle) through a ring
 // of shared-memory buffers, warp 1 issues tcgen05.mma (M=128, N=128, K=16,
@@ -21,7 +23,11 @@ constexpr int UM_STAGES = 6;
 constexpr int UM_A_BYTES = UM_BM * UM_BK * 2;              // 16 KiB
 constexpr int UM_B_BYTES = UM_BN * UM_BK * 2;              // 16 KiB
 constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
-constexpr int UM_THREADS = 192;
+// Epilogue warps: 4 (one per 32-lane quarter of tensor memory) for the GEMMs whose epilogue is small;
+// 16 (four per quarter, each taking every fourth 16-column chunk) for the weight-gradient kernel with the
+// fused update, whose epilogue streams 22 bytes per element and needs many loads in flight.
+__host__ __device__ constexpr int umma_epi_warps(int epi) { return epi >= 4 ? 16 : 4; }
+__host__ __device__ constexpr int umma_threads(int epi) { return 64 + 32 * umma_epi_warps(epi); }
 constexpr int UM_TMEM_COLS = 256;                          // two 128-column accumulators
 constexpr size_t UM_SMEM_BYTES = (size_t)UM_STAGES * UM_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long UM_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
@@ -30,7 +36,9 @@ enum UmmaEpilogue {
     UEPI_FWD_HIDDEN = 0,   // + bias[n], ReLU, bf16 out [M,ld] and transposed out [N,ldT]
     UEPI_FWD_LAST = 1,     // + bias[n], fp32 out [M,ld]
     UEPI_DGRAD = 2,        // * (mask[m,n] > 0), bf16 out and transposed out
-    UEPI_WGRAD = 3         // fp32 out [M,ld]
+    UEPI_WGRAD = 3,        // fp32 out, transposed: element (m, n) -> outf[n * ld + m]
+    UEPI_WGRAD_UPDATE = 4, // no gradient store: Eq. (parle_y)/(parle_z) applied in place to y, z (+ bf16 copy)
+    UEPI_WGRAD_UPDATE_FIRST = 5   // same on the first step of a round (y = z = x read from x)
 };
 
 struct UmmaParams {
@@ -41,6 +49,10 @@ struct UmmaParams {
     __nv_bfloat16 *outT; long long outT_gs; int outT_ld;
     float *outf; long long outf_gs; int outf_ld;
     const __nv_bfloat16 *mask; long long mask_gs; int mask_ld;
+    // fused inner update (UEPI_WGRAD_UPDATE*): the W_l segment of every replica, row pitch upd_ld, replica pitch upd_gs
+    float *upd_y; float *upd_z; const float *upd_x; __nv_bfloat16 *upd_shadow;
+    long long upd_gs; int upd_ld;
+    float eta_p, inv_gamma, alpha;
     int *status;
 };
 
@@ -115,6 +127,14 @@ __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tc_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a 128-byte-swizzled operand tile.
@@ -147,7 +167,7 @@ __device__ __forceinline__ void tile_coords(const UmmaParams &p, int t, int &g, 
 }
 
 template <int EPI, bool B_MN>
-__global__ void __launch_bounds__(UM_THREADS, 1)
+__global__ void __launch_bounds__(umma_threads(EPI), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -166,7 +186,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < UM_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, umma_epi_warps(EPI)); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -254,6 +274,54 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tc_fence_after();
             const int m = m0 + q * 32 + lane;                // output row of this thread
             const bool m_ok = m < p.M;
+            if constexpr (EPI == UEPI_WGRAD_UPDATE || EPI == UEPI_WGRAD_UPDATE_FIRST) {
+                // accumulator row m = column of W (contiguous in memory), accumulator column = row of W:
+                // for each j the 32 lanes touch 32 consecutive elements of W row nb + j in y, x, z.
+                constexpr bool FIRST = (EPI == UEPI_WGRAD_UPDATE_FIRST);
+                constexpr int CW = 16;
+                const int cg = (warp - 2) >> 2;
+                const float one_m_alpha = 1.0f - p.alpha;
+                bool fin = true;
+#pragma unroll 1
+                for (int c = cg; c < UM_BN / CW; c += umma_epi_warps(EPI) / 4) {
+                    const int nb = n0 + c * CW;
+                    if (nb >= p.N) break;                    // warp-uniform
+                    const long long e0 = (long long)g * p.upd_gs + (long long)nb * p.upd_ld + m;
+                    const float *xp = p.upd_x + e0;
+                    float *yp = p.upd_y + e0, *zp = p.upd_z + e0;
+                    __nv_bfloat16 *sp = p.upd_shadow + e0;
+                    float xv[CW], yv[CW], zv[CW];
+                    if (m_ok) {
+#pragma unroll
+                        for (int j = 0; j < CW; ++j) {
+                            if (nb + j < p.N) {
+                                const long long o = (long long)j * p.upd_ld;
+                                xv[j] = __ldcs(xp + o);
+                                if (!FIRST) { yv[j] = __ldcs(yp + o); zv[j] = __ldcs(zp + o); }
+                            }
+                        }
+                    }
+                    uint32_t r[CW];
+                    tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * UM_BN + c * CW), r);
+                    tc_wait_ld();
+                    if (m_ok) {
+#pragma unroll
+                        for (int j = 0; j < CW; ++j) {
+                            if (nb + j < p.N) {
+                                const long long o = (long long)j * p.upd_ld;
+                                const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
+                                const float yn = yo - p.eta_p * fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j]));
+                                const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
+                                fin &= (fabsf(yn) <= 3.402823466e+38f);
+                                __stcs(yp + o, yn);
+                                __stcs(zp + o, zn);
+                                sp[o] = __float2bfloat16_rn(yn);
+                            }
+                        }
+                    }
+                }
+                if (!fin) p.status[SLOT_NONFINITE] = 1;
+            } else {
 #pragma unroll 1
             for (int c = 0; c < UM_BN / 32; ++c) {
                 const int nb = n0 + c * 32;
@@ -312,21 +380,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             if (nb + j < p.N) oT[(long long)(nb + j) * p.outT_ld] = __float2bfloat16_rn(v[j]);
                     }
                 }
-                if (EPI == UEPI_FWD_LAST || EPI == UEPI_WGRAD) {
+                if (EPI == UEPI_FWD_LAST) {
                     if (m_ok) {
                         float *o = p.outf + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
-                        if (EPI == UEPI_WGRAD) {             // N % 8 == 0 and ld % 8 == 0: 16-byte stores
 #pragma unroll
-                            for (int j4 = 0; j4 < 32; j4 += 4)
-                                if (nb + j4 < p.N)
-                                    *reinterpret_cast<float4 *>(o + j4) = make_float4(v[j4], v[j4 + 1], v[j4 + 2], v[j4 + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (nb + j < p.N) o[j] = v[j];
-                        }
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N) o[j] = v[j];
                     }
                 }
+                if (EPI == UEPI_WGRAD) {
+                    // accumulator row m = column of W, accumulator column = row of W: for each j the
+                    // 32 lanes store 32 consecutive floats of W row nb + j
+                    if (m_ok) {
+                        float *o = p.outf + (long long)g * p.outf_gs + (long long)nb * p.outf_ld + m;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N) o[(long long)j * p.outf_ld] = v[j];
+                    }
+                }
+            }
             }
             tc_fence_before();
             __syncwarp();

@@ -25,10 +25,14 @@ DEV = "cuda:0"
 TOL = {pb.GEMM_FP32: 1e-4, pb.GEMM_BF16: 2e-2}
 
 
-def make(cfg, **over):
+def make(cfg, fused=None, **over):
+    """fused: None = library default (on for bf16 GEMMs); False = write the gradient to `grad`
+    and run the separate update kernel (needed by the tests that read the gradient)."""
     hyper = dict(gamma=cfg.gamma, rho=cfg.rho, alpha=cfg.alpha, eta=cfg.eta, eta_prime=cfg.eta_prime)
     hyper.update(over)
     m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, **hyper).alloc(DEV)
+    if fused is not None and cfg.gemm_dtype == pb.GEMM_BF16:
+        m.set_fused_update(fused)
     x0 = np.stack([po.pack(si.init_replica(cfg, a)) for a in range(cfg.n)])
     m.x.copy_(torch.from_numpy(to_padded(m, x0)))
     m.mean(); torch.cuda.synchronize()
@@ -36,8 +40,8 @@ def make(cfg, **over):
     return m, x0, xbar0, po.Hyper(hyper["eta"], hyper["eta_prime"], hyper["alpha"], hyper["gamma"], hyper["rho"])
 
 
-def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False):
-    m, xo, xb, hp = make(cfg)
+def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False, fused=None):
+    m, xo, xb, hp = make(cfg, fused=fused)
     tol = TOL[cfg.gemm_dtype]
     pad = torch.from_numpy(padding_mask(m)).to(DEV)
     for r in range(rounds):
@@ -91,7 +95,7 @@ def grad_check(cfg, tol, loose=None, outliers=0):
     fp32 GEMMs at full width: one unit within fp32 rounding of zero (probability
     ~1e-7 per unit and sample, ~1e6 units per step) switches now and then; up to
     `outliers` replicas may exceed `tol` and must then stay within 1e-2."""
-    m, xo, xb, hp = make(cfg)
+    m, xo, xb, hp = make(cfg, fused=False)
     X, c = si.round_batches(cfg.scaled(L=1), 0)
     loss = torch.zeros(cfg.n, device=DEV)
     m.round_begin(); m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV), loss)
@@ -211,12 +215,39 @@ def test_ragged_tiles_gradient_bf16():
 
 
 def test_small_rounds_bf16():
-    run_rounds(si.C1.scaled(name="bf16-small", dims=(64, 128, 72, 10), batch=16, gemm_dtype=1), 2, disp_tol=5e-2)
+    cfg = si.C1.scaled(name="bf16-small", dims=(64, 128, 72, 10), batch=16, gemm_dtype=1)
+    run_rounds(cfg, 2, disp_tol=5e-2)
+    run_rounds(cfg, 2, disp_tol=5e-2, fused=False)
+
+
+@pytest.mark.parametrize("dims,batch,n", [((64, 128, 72, 10), 16, 3), ((200, 328, 136, 101), 136, 2),
+                                          ((3072, 2048, 2048, 2048, 100), 128, 2)])
+def test_fused_update_equals_separate_update_bf16(dims, batch, n):
+    """Update applied inside the weight-gradient GEMM == gradient written out + update kernel:
+    the accumulators are the same, so y, z and the bf16 operand copy must agree bit for bit,
+    on the first step of a round (reset folded in) and on a later one, padding included."""
+    cfg = si.C1.scaled(name="fused", n=n, dims=dims, batch=batch, gemm_dtype=1, L=2)
+    X, c = si.round_batches(cfg, 0)
+    res = []
+    for fused in (True, False):
+        m, *_ = make(cfg, fused=fused)
+        m.y.fill_(7.0); m.z.fill_(-3.0)            # stale contents must not survive the folded reset
+        m.round_begin()
+        for l in range(cfg.L):
+            m.inner_step(torch.from_numpy(X[l]).to(DEV), torch.from_numpy(c[l]).to(DEV))
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        res.append((m.y.clone(), m.z.clone(), m.debug_buffer(m.DBG_OPERAND_COPY).clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+    pad = torch.from_numpy(padding_mask(m)).to(DEV)
+    assert torch.all(res[0][0][:, pad] == 0) and torch.all(res[0][1][:, pad] == 0)
 
 
 def test_c3_scaled_down_round_bf16():
     cfg = si.C3.scaled(name="C3/4", n=2, dims=(768, 512, 512, 512, 100), L=5)
     run_rounds(cfg, 2, disp_tol=5e-2)
+    run_rounds(cfg, 1, disp_tol=5e-2, fused=False)
 
 
 def test_c3_gradient_full_shape_bf16():
@@ -233,7 +264,7 @@ def _layerwise_bf16(cfg):
     workspace), so that ReLU switching cannot accumulate across layers.
     Allowed differences: a bf16 result one unit in the last place off where the
     fp32-accumulated value sits on a rounding tie."""
-    m, xo, xb, hp = make(cfg)
+    m, xo, xb, hp = make(cfg, fused=False)
     X, c = si.round_batches(cfg.scaled(L=1), 0)
     m.round_begin()
     m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV))
