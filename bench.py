@@ -113,8 +113,7 @@ def dense_to_padded(model, cfg, replica_layers):
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture
 # (profiles/ncu_full_inner_update_and_gemms_C3.md), valid only while the kernel source is unchanged.
-NCU_TRAFFIC = {("C3", "inner_update"): {"bytes": 1.906072e9 + 1.139100e9, "source_sha256_16": "d8f450f3c97c7a57",
-                                        "source": "paper_1707_00424_b200/csrc/update_kernels.cuh"}}
+NCU_TRAFFIC = {}
 
 
 def ncu_traffic(workload: str, kernel: str):
@@ -128,9 +127,26 @@ def ncu_traffic(workload: str, kernel: str):
     return rec["bytes"]
 
 
-def bytes_per_param_inner_update(cfg) -> int:
-    # read g, y, x, z + write y, z (fp32) [+ bf16 operand copy of y]
-    return 24 + (2 if cfg.gemm_dtype == 1 else 0)
+def algorithmic_bytes_per_round(cfg, stride):
+    """Bytes each kernel class has to move per Parle round (all n replicas), from the data it must
+    touch once: parameter-state vectors at 4 B (fp32) or 2 B (bf16 copy) per element, plus GEMM operands."""
+    n, B, L, dims = cfg.n, cfg.batch, cfg.L, cfg.dims
+    nl = len(dims) - 1
+    Pw = sum(dims[l] * dims[l + 1] for l in range(nl))
+    bf = cfg.gemm_dtype == 1
+    act = lambda l: B * dims[l]                          # elements of one replica's activation at level l
+    out = {}
+    # separate update: read g, y, x, z, write y, z (+2 B bf16 copy); first step of a round reads x for y and z
+    out["inner_update"] = n * stride * ((24 + (2 if bf else 0)) * L - 8)
+    out["outer_mean"] = stride * ((12 + (2 if bf else 0)) * n + 8)
+    if bf:
+        opnd = sum(2 * (act(l) + act(l + 1)) for l in range(nl))             # dH^T and H^T, bf16
+        # fused: read y, x, z (12 B), write y, z, bf16 copy (10 B); first step reads only x
+        out["wgrad_gemm_fused_update"] = n * (Pw * (22 * (L - 1) + 14) + opnd * L)
+        out["wgrad_gemm"] = n * L * (4 * Pw + opnd)
+        out["fwd_gemm"] = n * L * (2 * Pw + sum(2 * act(l) + 4 * act(l + 1) for l in range(nl)))
+        out["dgrad_gemm"] = n * L * sum(2 * dims[l] * dims[l + 1] + 2 * act(l + 1) + 6 * act(l) for l in range(1, nl))
+    return out
 
 
 # ------------------------------------------------------------------ our arm
@@ -178,10 +194,7 @@ def run_ours(args):
         exchange()
 
     def round_host(r):
-        model.round_begin()
-        for l in range(cfg.L):
-            model.inner_step_host(Xp[r % sets, l], cp[r % sets, l], loss_p[l])
-        model.outer_step()
+        model.round_host(cfg.L, Xp[r % sets], cp[r % sets], loss_p)
         exchange()
 
     def timed(fn, warmup, steps, sample_clocks=False):
@@ -231,19 +244,18 @@ def run_ours(args):
     total_ms = sum(v[0] for v in prof.values()) or 1.0
     shares = {k: {"ms_per_round": v[0] / K, "launches_per_round": v[1] / K, "share": v[0] / total_ms} for k, v in prof.items()}
     dom = max(prof, key=lambda k: prof[k][0])
-    roofline = None
-    if dom == "inner_update":
-        per_launch_ms = prof[dom][0] / prof[dom][1]
-        # steady-state launches move 24 (+2) B per element; the first of each round (reset folded in) 8 B less
-        bpp = bytes_per_param_inner_update(cfg)
-        bytes_per_launch = cfg.n * model.stride * (bpp - 8.0 / cfg.L)
-        ach = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
-        roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, dom), "peak_source": peaks["source"],
-                    "bytes_per_launch": bytes_per_launch, "ms_per_launch": per_launch_ms}
-    else:
-        roofline = {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": None, "traffic": None, "peak_source": peaks["source"]}
+    alg = algorithmic_bytes_per_round(cfg, model.stride)
+    rooflines = {}
+    for k, (ms_k, cnt_k) in prof.items():
+        if k not in alg:
+            continue
+        ach = alg[k] * K / (ms_k * 1e-3) / 1e9          # bytes of K rounds / device time of the class over K rounds
+        rooflines[k] = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, k),
+                        "peak_source": peaks["source"], "bytes_per_launch": alg[k] * K / cnt_k,
+                        "ms_per_launch": ms_k / cnt_k, "launches_per_round": cnt_k / K}
+    roofline = rooflines.get(dom, {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": None, "traffic": None, "peak_source": peaks["source"]})
     cpu = cpu_baseline(cfg, budget_s=15.0)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -257,7 +269,8 @@ def run_ours(args):
         "gpu_launches": launches, "device_flags": flags, "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / K},
-        "roofline": roofline, "kernel_shares": shares, "profile_dropped": dropped,
+        "roofline": roofline, "roofline_other_kernels": {k: v for k, v in rooflines.items() if k != dom},
+        "kernel_shares": shares, "profile_dropped": dropped,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))

@@ -150,6 +150,16 @@ int parle_mean(parle_ctx *ctx);
 int parle_round(parle_ctx *ctx, int L, const float *inputs, const int32_t *labels,
                 float *loss_out);
 
+/* A whole round from host buffers: inputs host [L, n, B, d_0], labels host
+ * [L, n, B], loss_out host [L, n] or NULL.  The minibatch of step l+1 is uploaded
+ * on a second stream into a second staging buffer while step l computes, so with
+ * pinned host memory the copies hide behind the kernels.  The first call creates
+ * that stream and four events (no device memory).  Results (and loss_out) are
+ * valid once the bound stream has been synchronised; the host buffers must stay
+ * untouched until then. */
+int parle_round_host(parle_ctx *ctx, int L, const float *inputs_host, const int32_t *labels_host,
+                     float *loss_out_host);
+
 /* bf16 path only.  on (the default): Eq. (parle_y), (parle_z) are applied
  * inside the weight-gradient GEMM's epilogue, so the weight gradient is never
  * written and `grad` is left untouched by parle_inner_step.  off: the gradient is

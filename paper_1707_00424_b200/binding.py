@@ -65,6 +65,7 @@ def lib() -> C.CDLL:
         "parle_outer_step": (ci, [vp]),
         "parle_mean": (ci, [vp]),
         "parle_round": (ci, [vp, ci, vp, vp, vp]),
+        "parle_round_host": (ci, [vp, ci, vp, vp, vp]),
         "parle_set_coupling": (ci, [vp, cd, cd]),
         "parle_set_lr": (ci, [vp, cd, cd]),
         "parle_set_fused_update": (ci, [vp, ci]),
@@ -205,6 +206,10 @@ class Parle:
 
     def round(self, L: int, inputs, labels, loss_out=None):
         self._check(self._L.parle_round(self._h, L, _ptr(inputs), _ptr(labels), _ptr(loss_out)), "parle_round")
+
+    def round_host(self, L: int, inputs_host, labels_host, loss_out_host=None):
+        self._check(self._L.parle_round_host(self._h, L, _ptr(inputs_host), _ptr(labels_host), _ptr(loss_out_host)),
+                    "parle_round_host")
 
     def set_coupling(self, gamma: float, rho: float):
         self._check(self._L.parle_set_coupling(self._h, gamma, rho), "parle_set_coupling")

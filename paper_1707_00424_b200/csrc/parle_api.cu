@@ -35,7 +35,7 @@ struct Workspace {
     size_t dhb[PARLE_MAX_LAYERS], dhbT[PARLE_MAX_LAYERS];    // their gradients, both layouts
     int dh_ld[PARLE_MAX_LAYERS];       // row pitch of dhb[l] (d_{l+1} rounded up to 8)
     size_t row_loss;                   // [n,B] fp32
-    size_t stage_in, stage_lab, stage_loss;   // staging for the host-buffer entry point
+    size_t stage_in[2], stage_lab[2], stage_loss[2];   // double-buffered staging for the host-buffer entry points
     size_t total;
 };
 
@@ -61,6 +61,10 @@ struct parle_ctx {
     CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
+    // host-buffer rounds: a second stream uploads the next minibatch while the current step runs
+    cudaStream_t copy_stream;
+    cudaEvent_t ev_copied[2], ev_consumed[2];
+    bool copy_ready;
     // optional per-launch timing (events, host-side bookkeeping only)
     bool prof_on, prof_open;
     int prof_used, prof_dropped;
@@ -123,9 +127,11 @@ void plan_workspace(parle_ctx *c) {
         }
     }
     w.row_loss = take(n * B * sizeof(float));
-    w.stage_in = take(n * B * c->dims[0] * sizeof(float));
-    w.stage_lab = take(n * B * sizeof(int32_t));
-    w.stage_loss = take(n * sizeof(float));
+    for (int b = 0; b < 2; ++b) {
+        w.stage_in[b] = take(n * B * c->dims[0] * sizeof(float));
+        w.stage_lab[b] = take(n * B * sizeof(int32_t));
+        w.stage_loss[b] = take(n * sizeof(float));
+    }
     w.total = off;
 }
 
@@ -470,6 +476,10 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
 void parle_destroy(parle_ctx *c) {
     if (!c) return;
     if (c->status_host) cudaFreeHost(c->status_host);
+    if (c->copy_ready) {
+        cudaStreamDestroy(c->copy_stream);
+        for (int b = 0; b < 2; ++b) { cudaEventDestroy(c->ev_copied[b]); cudaEventDestroy(c->ev_consumed[b]); }
+    }
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfCapacity; ++i) cudaEventDestroy(c->prof_ev[i]);
         delete[] c->prof_ev;
@@ -560,9 +570,11 @@ int parle_inner_step_host(parle_ctx *c, const float *inputs_host, const int32_t 
     if (c->n_layers == 0 || !inputs_host || !labels_host) return PARLE_EINVAL;
     if (!c->round_open) return PARLE_ESTATE;
     const size_t nb = (size_t)c->n * c->batch;
-    float *din = ws_ptr<float>(c, c->ws.stage_in);
-    int32_t *dlab = ws_ptr<int32_t>(c, c->ws.stage_lab);
-    float *dloss = ws_ptr<float>(c, c->ws.stage_loss);
+    float *din = ws_ptr<float>(c, c->ws.stage_in[0]);
+    int32_t *dlab = ws_ptr<int32_t>(c, c->ws.stage_lab[0]);
+    float *dloss = ws_ptr<float>(c, c->ws.stage_loss[0]);
+    if (c->copy_ready)      // the pipelined entry point may still own the staging buffer
+        PARLE_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_consumed[0], 0));
     PARLE_CUDA(c, cudaMemcpyAsync(din, inputs_host, nb * c->dims[0] * sizeof(float), cudaMemcpyHostToDevice, c->stream));
     PARLE_CUDA(c, cudaMemcpyAsync(dlab, labels_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
     PARLE_TRY(parle_inner_step(c, din, dlab, loss_out_host ? dloss : nullptr));
@@ -618,6 +630,48 @@ int parle_round(parle_ctx *c, int L, const float *inputs, const int32_t *labels,
     for (int l = 0; l < L; ++l)
         PARLE_TRY(parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
                                    loss_out ? loss_out + (size_t)l * c->n : nullptr));
+    return parle_outer_step(c);
+}
+
+int parle_round_host(parle_ctx *c, int L, const float *inputs_host, const int32_t *labels_host, float *loss_out_host) {
+    PARLE_TRY(check_bound(c));
+    if (L < 1 || c->n_layers == 0 || !inputs_host || !labels_host) return PARLE_EINVAL;
+    if (!c->copy_ready) {
+        PARLE_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; ++b) {
+            PARLE_CUDA(c, cudaEventCreateWithFlags(&c->ev_copied[b], cudaEventDisableTiming));
+            PARLE_CUDA(c, cudaEventCreateWithFlags(&c->ev_consumed[b], cudaEventDisableTiming));
+        }
+        c->copy_ready = true;
+    }
+    const size_t nb = (size_t)c->n * c->batch, in_elems = nb * c->dims[0];
+    auto upload = [&](int l) -> int {       // minibatch l -> staging buffer l % 2, on the copy stream
+        const int b = l & 1;
+        PARLE_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_consumed[b], 0));   // its previous user is done
+        PARLE_CUDA(c, cudaMemcpyAsync(ws_ptr<float>(c, c->ws.stage_in[b]), inputs_host + (size_t)l * in_elems,
+                                      in_elems * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+        PARLE_CUDA(c, cudaMemcpyAsync(ws_ptr<int32_t>(c, c->ws.stage_lab[b]), labels_host + (size_t)l * nb,
+                                      nb * sizeof(int32_t), cudaMemcpyHostToDevice, c->copy_stream));
+        PARLE_CUDA(c, cudaEventRecord(c->ev_copied[b], c->copy_stream));
+        return PARLE_OK;
+    };
+    // everything enqueued on the bound stream so far (earlier users of the staging buffers) comes first
+    PARLE_CUDA(c, cudaEventRecord(c->ev_consumed[0], c->stream));
+    PARLE_CUDA(c, cudaEventRecord(c->ev_consumed[1], c->stream));
+    PARLE_TRY(parle_round_begin(c));
+    PARLE_TRY(upload(0));
+    for (int l = 0; l < L; ++l) {
+        const int b = l & 1;
+        if (l + 1 < L) PARLE_TRY(upload(l + 1));
+        PARLE_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
+        float *dloss = ws_ptr<float>(c, c->ws.stage_loss[b]);
+        PARLE_TRY(parle_inner_step(c, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
+                                   loss_out_host ? dloss : nullptr));
+        if (loss_out_host)
+            PARLE_CUDA(c, cudaMemcpyAsync(loss_out_host + (size_t)l * c->n, dloss, c->n * sizeof(float),
+                                          cudaMemcpyDeviceToHost, c->stream));
+        PARLE_CUDA(c, cudaEventRecord(c->ev_consumed[b], c->stream));
+    }
     return parle_outer_step(c);
 }
 

@@ -196,6 +196,35 @@ def test_host_buffer_step_matches_device_step():
     assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
 
 
+@pytest.mark.parametrize("dtype_dims", [(0, (64, 32, 10)), (1, (64, 128, 72, 10))])
+def test_host_buffer_round_matches_device_round(dtype_dims):
+    """parle_round_host (pipelined uploads) == parle_round on device-resident inputs, twice in a row,
+    interleaved with the single-step host entry point (they share the staging buffers)."""
+    gd, dims = dtype_dims
+    cfg = si.C1.scaled(dims=dims, gemm_dtype=gd, L=5)
+    a, *_ = make(cfg)
+    b, *_ = make(cfg)
+    for r in range(2):
+        X, c = si.round_batches(cfg, r)
+        la = torch.zeros(cfg.L, cfg.n, device=DEV)
+        a.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV), la)
+        Xh, ch = torch.from_numpy(X).pin_memory(), torch.from_numpy(c).pin_memory()
+        lb = torch.zeros(cfg.L, cfg.n).pin_memory()
+        b.round_host(cfg.L, Xh, ch, lb)
+        torch.cuda.synchronize()
+        assert torch.equal(a.x, b.x) and torch.equal(a.xbar, b.xbar) and torch.equal(la.cpu(), lb)
+        # a single host-buffer step right after (reuses staging buffer 0)
+        for m in (a, b):
+            m.round_begin()
+        l1 = torch.zeros(cfg.n).pin_memory()
+        a.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV))
+        b.inner_step_host(Xh[0], ch[0], l1)
+        for m in (a, b):
+            m.outer_step()
+        torch.cuda.synchronize()
+        assert torch.equal(a.x, b.x)
+
+
 def test_c2_gradient_full_shape_fp32():
     grad_check(si.C2, 1e-5, outliers=1)
 

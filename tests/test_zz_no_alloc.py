@@ -8,6 +8,8 @@ losses of a regular inner step are read back and the new entry point is run on
 those logits, twice in a row with different data (the array is shared between
 calls and keeps old contents, so the second call checks that nothing stale
 leaks through)."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -45,10 +47,12 @@ def test_static_loss_matches_inner_step_twice_in_a_row():
         got_d = torch.full_like(want_d.contiguous(), float("nan"))
         got_loss = torch.full((cfg.n,), float("nan"), device=DEV)
         flags = torch.full((1,), -1, dtype=torch.int32, device=DEV)
+        logits = logits.contiguous()
+        gc.collect(); torch.cuda.synchronize()               # drop the finished model's tensors first
         before = torch.cuda.memory_allocated()
-        pb.softmax_ce_static(logits.contiguous(), labels, cfg.n, cfg.batch, C, got_d, got_loss, flags)
+        pb.softmax_ce_static(logits, labels, cfg.n, cfg.batch, C, got_d, got_loss, flags)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.memory_allocated() == before       # torch's allocator was not touched
         # same kernels, same inputs: equal to rounding (the tolerance of the fp32 element-wise tests)
         np.testing.assert_allclose(got_d.cpu().numpy(), want_d.cpu().numpy(), rtol=1e-6, atol=1e-7)
         np.testing.assert_allclose(got_loss.cpu().numpy(), want_loss.cpu().numpy(), rtol=1e-6, atol=1e-7)
