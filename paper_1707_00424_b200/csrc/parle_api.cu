@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "mlp_simt.cuh"
 #include "umma_gemm.cuh"
+#include "umma_wgrad_update.cuh"
 #include "update_kernels.cuh"
 
 using namespace parle;
@@ -61,6 +62,7 @@ struct parle_ctx {
     CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
+    CUtensorMap tm_sx[PARLE_MAX_LAYERS], tm_sy[PARLE_MAX_LAYERS], tm_sz[PARLE_MAX_LAYERS];   // fp32 W_l segments of x, y, z
     // host-buffer rounds: a second stream uploads the next minibatch while the current step runs
     cudaStream_t copy_stream;
     cudaEvent_t ev_copied[2], ev_consumed[2];
@@ -175,6 +177,22 @@ int encode_bf16_map(parle_ctx *c, CUtensorMap *tm, const void *base, size_t cols
     return PARLE_OK;
 }
 
+// fp32 tensor [groups][rows][cols], no swizzle (boxes are read back word by word, lane = column).
+int encode_f32_map(parle_ctx *c, CUtensorMap *tm, const void *base, size_t cols, size_t rows, size_t groups,
+                   size_t row_pitch, size_t group_pitch, unsigned box_cols, unsigned box_rows) {
+    EncodeTiledFn enc;
+    PARLE_TRY(get_encoder(c, &enc));
+    cuuint64_t dims[3] = {cols, rows, groups};
+    cuuint64_t strides[2] = {row_pitch * 4, group_pitch * 4};
+    cuuint32_t box[3] = {box_cols, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
+    return PARLE_OK;
+}
+
 int build_tensor_maps(parle_ctx *c) {
     const Workspace &w = c->ws;
     const size_t n = c->n, B = c->batch;
@@ -191,6 +209,11 @@ int build_tensor_maps(parle_ctx *c) {
         // both K-major (K = batch)
         PARLE_TRY(encode_bf16_map(c, &c->tm_wg_a[l], a_inT, B, din, n, B, din * B, UM_BK, UM_BM));
         PARLE_TRY(encode_bf16_map(c, &c->tm_wg_b[l], ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), B, dout, n, B, dout * B, UM_BK, UM_BN));
+        // fused update: the W_l segments of x, y, z as [n][dout][din] fp32, fetched in 16-row x 128-column boxes
+        const size_t wo = c->layers[l].w_off;
+        PARLE_TRY(encode_f32_map(c, &c->tm_sx[l], c->buf.x + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
+        PARLE_TRY(encode_f32_map(c, &c->tm_sy[l], c->buf.y + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
+        PARLE_TRY(encode_f32_map(c, &c->tm_sz[l], c->buf.z + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
         if (l > 0) {
             // data gradient: A = dH [B, dout] K-major (K = dout); B = W [dout (K), din (N)] MN-major,
             // fetched as 64 k-rows x 64 n-columns boxes
@@ -383,14 +406,24 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     for (int l = nl - 1; l >= 0; --l) {
         const int din = c->dims[l], dout = c->dims[l + 1];
         if (l > 0) PARLE_TRY(dgrad(l));
-        UmmaParams p = {};
+        WgradUpdateParams p = {};
         p.M = din; p.N = dout; p.K = B;
+        p.groups = n; p.tiles_m = (din + UM_BM - 1) / UM_BM; p.tiles_n = (dout + UM_BN - 1) / UM_BN;
         const size_t wo = c->layers[l].w_off;
-        p.upd_y = c->buf.y + wo; p.upd_z = c->buf.z + wo; p.upd_x = c->buf.x + wo; p.upd_shadow = shadow + wo;
-        p.upd_gs = S; p.upd_ld = din;
+        p.y = c->buf.y + wo; p.z = c->buf.z + wo; p.shadow = shadow + wo;
+        p.gs = S; p.ld = din;
         p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha;
-        if (c->fresh) PARLE_TRY((launch_umma<UEPI_WGRAD_UPDATE_FIRST, false>(c, KC_WGRAD_UPDATE, c->tm_wg_a[l], c->tm_wg_b[l], p)));
-        else PARLE_TRY((launch_umma<UEPI_WGRAD_UPDATE, false>(c, KC_WGRAD_UPDATE, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+        p.status = c->status_dev;
+        const int tiles = p.groups * p.tiles_m * p.tiles_n;
+        const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+        prof_begin(c, KC_WGRAD_UPDATE);
+        if (c->fresh)
+            umma_wgrad_update_kernel<true><<<grid, WU_THREADS, WU_SMEM_BYTES, c->stream>>>(
+                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], p);
+        else
+            umma_wgrad_update_kernel<false><<<grid, WU_THREADS, WU_SMEM_BYTES, c->stream>>>(
+                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], p);
+        PARLE_LAUNCHED(c);
     }
     TailPlan tp = {};
     tp.n_layers = nl; tp.batch = B;
@@ -525,8 +558,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, false>()));
-        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD_UPDATE, false>()));
-        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD_UPDATE_FIRST, false>()));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WU_SMEM_BYTES));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WU_SMEM_BYTES));
         PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, true>()));
         PARLE_TRY(build_tensor_maps(c));
     }

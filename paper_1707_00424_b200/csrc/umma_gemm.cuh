@@ -23,10 +23,8 @@ constexpr int UM_STAGES = 6;
 constexpr int UM_A_BYTES = UM_BM * UM_BK * 2;              // 16 KiB
 constexpr int UM_B_BYTES = UM_BN * UM_BK * 2;              // 16 KiB
 constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
-// Epilogue warps: 4 (one per 32-lane quarter of tensor memory) for the GEMMs whose epilogue is small;
-// 16 (four per quarter, each taking every fourth 16-column chunk) for the weight-gradient kernel with the
-// fused update, whose epilogue streams 22 bytes per element and needs many loads in flight.
-__host__ __device__ constexpr int umma_epi_warps(int epi) { return epi >= 4 ? 16 : 4; }
+// Epilogue warps: one per 32-lane quarter of tensor memory.
+__host__ __device__ constexpr int umma_epi_warps(int) { return 4; }
 __host__ __device__ constexpr int umma_threads(int epi) { return 64 + 32 * umma_epi_warps(epi); }
 constexpr int UM_TMEM_COLS = 256;                          // two 128-column accumulators
 constexpr size_t UM_SMEM_BYTES = (size_t)UM_STAGES * UM_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -36,9 +34,7 @@ enum UmmaEpilogue {
     UEPI_FWD_HIDDEN = 0,   // + bias[n], ReLU, bf16 out [M,ld] and transposed out [N,ldT]
     UEPI_FWD_LAST = 1,     // + bias[n], fp32 out [M,ld]
     UEPI_DGRAD = 2,        // * (mask[m,n] > 0), bf16 out and transposed out
-    UEPI_WGRAD = 3,        // fp32 out, transposed: element (m, n) -> outf[n * ld + m]
-    UEPI_WGRAD_UPDATE = 4, // no gradient store: Eq. (parle_y)/(parle_z) applied in place to y, z (+ bf16 copy)
-    UEPI_WGRAD_UPDATE_FIRST = 5   // same on the first step of a round (y = z = x read from x)
+    UEPI_WGRAD = 3         // fp32 out, transposed: element (m, n) -> outf[n * ld + m]
 };
 
 struct UmmaParams {
@@ -49,10 +45,6 @@ struct UmmaParams {
     __nv_bfloat16 *outT; long long outT_gs; int outT_ld;
     float *outf; long long outf_gs; int outf_ld;
     const __nv_bfloat16 *mask; long long mask_gs; int mask_ld;
-    // fused inner update (UEPI_WGRAD_UPDATE*): the W_l segment of every replica, row pitch upd_ld, replica pitch upd_gs
-    float *upd_y; float *upd_z; const float *upd_x; __nv_bfloat16 *upd_shadow;
-    long long upd_gs; int upd_ld;
-    float eta_p, inv_gamma, alpha;
     int *status;
 };
 
@@ -134,6 +126,10 @@ __device__ __forceinline__ void tc_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_ld_32x4(uint32_t taddr, uint32_t (&r)[4]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -274,54 +270,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tc_fence_after();
             const int m = m0 + q * 32 + lane;                // output row of this thread
             const bool m_ok = m < p.M;
-            if constexpr (EPI == UEPI_WGRAD_UPDATE || EPI == UEPI_WGRAD_UPDATE_FIRST) {
-                // accumulator row m = column of W (contiguous in memory), accumulator column = row of W:
-                // for each j the 32 lanes touch 32 consecutive elements of W row nb + j in y, x, z.
-                constexpr bool FIRST = (EPI == UEPI_WGRAD_UPDATE_FIRST);
-                constexpr int CW = 16;
-                const int cg = (warp - 2) >> 2;
-                const float one_m_alpha = 1.0f - p.alpha;
-                bool fin = true;
-#pragma unroll 1
-                for (int c = cg; c < UM_BN / CW; c += umma_epi_warps(EPI) / 4) {
-                    const int nb = n0 + c * CW;
-                    if (nb >= p.N) break;                    // warp-uniform
-                    const long long e0 = (long long)g * p.upd_gs + (long long)nb * p.upd_ld + m;
-                    const float *xp = p.upd_x + e0;
-                    float *yp = p.upd_y + e0, *zp = p.upd_z + e0;
-                    __nv_bfloat16 *sp = p.upd_shadow + e0;
-                    float xv[CW], yv[CW], zv[CW];
-                    if (m_ok) {
-#pragma unroll
-                        for (int j = 0; j < CW; ++j) {
-                            if (nb + j < p.N) {
-                                const long long o = (long long)j * p.upd_ld;
-                                xv[j] = __ldcs(xp + o);
-                                if (!FIRST) { yv[j] = __ldcs(yp + o); zv[j] = __ldcs(zp + o); }
-                            }
-                        }
-                    }
-                    uint32_t r[CW];
-                    tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * UM_BN + c * CW), r);
-                    tc_wait_ld();
-                    if (m_ok) {
-#pragma unroll
-                        for (int j = 0; j < CW; ++j) {
-                            if (nb + j < p.N) {
-                                const long long o = (long long)j * p.upd_ld;
-                                const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
-                                const float yn = yo - p.eta_p * fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j]));
-                                const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
-                                fin &= (fabsf(yn) <= 3.402823466e+38f);
-                                __stcs(yp + o, yn);
-                                __stcs(zp + o, zn);
-                                sp[o] = __float2bfloat16_rn(yn);
-                            }
-                        }
-                    }
-                }
-                if (!fin) p.status[SLOT_NONFINITE] = 1;
-            } else {
+            {
 #pragma unroll 1
             for (int c = 0; c < UM_BN / 32; ++c) {
                 const int nb = n0 + c * 32;

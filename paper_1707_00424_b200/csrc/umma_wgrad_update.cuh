@@ -1,0 +1,263 @@
+// Weight-gradient GEMM with the inner update fused into its epilogue
+// (Section 2.1 gradient; Eq. parle_y, parle_z applied in place):
+//     G^T  = H_{l-1}^T dH_l                (tcgen05.mma, bf16 operands, fp32 accumulators in tensor memory)
+//     y   <- y - eta' (G + (y - x)/gamma)
+//     z   <- alpha z + (1 - alpha) y,     operand copy <- bf16(y)
+// for the W_l segment of every replica.  The gradient never reaches memory.
+//
+// The accumulator is the *transposed* gradient: its 128 rows (tensor-memory
+// lanes) run along d_in, the contiguous direction of W in memory, so a warp's
+// 32 lanes always touch 32 consecutive elements of one W row.
+//
+// This is a streaming kernel with a small GEMM inside (K = batch): 22 bytes per
+// weight go through the epilogue.  To keep enough bytes in flight, x, y and z
+// tiles are not loaded through registers: a loader warp brings 16-row x 128-col
+// fp32 boxes of x, y, z into a ring of shared-memory stages with TMA, running
+// several stages ahead of the epilogue warps, which read them conflict-free
+// (consecutive lanes -> consecutive words), combine them with the accumulator
+// chunk from tensor memory and store y, z and the bf16 copy straight from
+// registers (coalesced 128-byte / 64-byte warp stores).
+//
+// Roles: warp 0 operand TMA producer, warp 1 MMA issuer, warp 2 state loader,
+// warps 3.. epilogue: G groups of 4 warps (the four 32-lane quarters of tensor
+// memory).  Every epilogue warp consumes every chunk, in order -- group g takes
+// rows 4g .. 4g+3 of the chunk's 16 -- so each stage barrier sees all its
+// consumers in every phase and no waiter can fall a phase behind.
+// All waits are bounded.
+#pragma once
+
+#include "umma_gemm.cuh"
+
+namespace parle {
+
+constexpr int WU_CHUNK_ROWS = 16;                              // W rows (accumulator columns) per epilogue chunk
+constexpr int WU_CHUNKS = UM_BN / WU_CHUNK_ROWS;               // 8 per 128x128 tile
+constexpr int WU_OP_STAGES = 2;                                // operand ring (K = batch is short)
+constexpr int WU_ARRAY_BYTES = WU_CHUNK_ROWS * UM_BM * 4;      // 8 KiB: one fp32 box of x, y or z
+constexpr int WU_STATE_BYTES = 3 * WU_ARRAY_BYTES;             // x | y | z
+constexpr int WU_STATE_STAGES = 6;
+constexpr int WU_GROUPS = 4;                                   // epilogue warp groups
+constexpr int WU_THREADS = 96 + 128 * WU_GROUPS;
+constexpr size_t WU_SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)WU_STATE_STAGES * WU_STATE_BYTES +
+                                 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct WgradUpdateParams {
+    int M, N, K;                 // M = d_in (tile rows), N = d_out (tile columns), K = batch
+    int groups, tiles_m, tiles_n;
+    float *y, *z;                // W_l segment of replica 0; element (replica g, W row r, W col c) at g*gs + r*ld + c
+    __nv_bfloat16 *shadow;
+    long long gs; int ld;
+    float eta_p, inv_gamma, alpha;
+    int *status;
+};
+
+template <bool FIRST>
+__global__ void __launch_bounds__(WU_THREADS, 1)
+umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
+                         const __grid_constant__ CUtensorMap tmZ, const WgradUpdateParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t op_base = (raw + 1023u) & ~1023u;
+    const uint32_t st_base = op_base + WU_OP_STAGES * UM_STAGE_BYTES;
+    uint8_t *st_ptr = smem_raw + (st_base - raw);
+    uint8_t *ctl = st_ptr + (size_t)WU_STATE_STAGES * WU_STATE_BYTES;
+    // barriers: op_full[2], op_empty[2], tfull[2], tempty[2], st_full[S], st_empty[S]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);
+    constexpr int NBARS = 2 * WU_OP_STAGES + 4 + 2 * WU_STATE_STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * NBARS);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * WU_OP_STAGES;
+    const uint32_t bar_tfull = bar_empty + 8 * WU_OP_STAGES, bar_tempty = bar_tfull + 16;
+    const uint32_t bar_sfull = bar_tempty + 16, bar_sempty = bar_sfull + 8 * WU_STATE_STAGES;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int num_kb = (p.K + UM_BK - 1) / UM_BK;
+    const int per_g = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < WU_OP_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, 4 * WU_GROUPS); }
+        for (int s = 0; s < WU_STATE_STAGES; ++s) { mbar_init(bar_sfull + 8 * s, 1); mbar_init(bar_sempty + 8 * s, 4 * WU_GROUPS); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)UM_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto coords = [&](int t, int &g, int &m0, int &n0) {
+        g = t / per_g;
+        const int r = t - g * per_g;
+        m0 = (r % p.tiles_m) * UM_BM;
+        n0 = (r / p.tiles_m) * UM_BN;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------ operand producer (A = H^T tile, B = dH^T tile)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int g, m0, n0; coords(t, g, m0, n0);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = op_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
+                    const uint32_t fb = bar_full + 8 * stage;
+                    mbar_expect_tx(fb, UM_STAGE_BYTES);
+                    tma_load_3d(sa, &tmA, fb, kb * UM_BK, m0, g);
+                    tma_load_3d(sb, &tmB, fb, kb * UM_BK, n0, g);
+                    if (++stage == WU_OP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                for (int s = 0; s < WU_OP_STAGES; ++s) {
+                    const uint32_t armed_parity = (s < stage) ? phase : (phase ^ 1u);
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(false, false);
+            int stage = 0; uint32_t phase = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * UM_BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = op_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
+                    const uint64_t adesc = make_smem_desc(sa, 16, 1024), bdesc = make_smem_desc(sb, 16, 1024);
+#pragma unroll
+                    for (int k = 0; k < UM_BK / 16; ++k)
+                        tc_mma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                    tc_commit(bar_empty + 8 * stage);
+                    if (++stage == WU_OP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(bar_tfull + 8 * acc);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------ state loader: x (, y, z) boxes, chunk by chunk
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int g, m0, n0; coords(t, g, m0, n0);
+                for (int c = 0; c < WU_CHUNKS; ++c) {
+                    const int nb = n0 + c * WU_CHUNK_ROWS;
+                    if (nb >= p.N) break;
+                    if (!mbar_wait(bar_sempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = st_base + stage * WU_STATE_BYTES;
+                    const uint32_t fb = bar_sfull + 8 * stage;
+                    mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES);
+                    tma_load_3d(dst, &tmX, fb, m0, nb, g);
+                    if (!FIRST) {
+                        tma_load_3d(dst + WU_ARRAY_BYTES, &tmY, fb, m0, nb, g);
+                        tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &tmZ, fb, m0, nb, g);
+                    }
+                    if (++stage == WU_STATE_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                for (int s = 0; s < WU_STATE_STAGES; ++s) {
+                    const uint32_t armed_parity = (s < stage) ? phase : (phase ^ 1u);
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_sfull + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue groups
+        const int q = warp & 3;                              // tensor-memory lane quarter of this warp
+        const int grp = (warp - 3) >> 2;                     // rows grp*RPG .. of every chunk
+        constexpr int RPG = WU_CHUNK_ROWS / WU_GROUPS;       // rows per group and chunk
+        static_assert(RPG == 4, "tcgen05.ld shape below reads 4 columns");
+        const float one_m_alpha = 1.0f - p.alpha;
+        int acc = 0; uint32_t acc_phase = 0;
+        int stage = 0; uint32_t sphase = 0;                  // state ring position: every warp walks every chunk
+        bool fin = true, ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            int g, m0, n0; coords(t, g, m0, n0);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const int col = q * 32 + lane;                   // tile column along d_in
+            const int m = m0 + col;
+            const bool m_ok = m < p.M;
+#pragma unroll 1
+            for (int c = 0; c < WU_CHUNKS; ++c) {
+                const int nb0 = n0 + c * WU_CHUNK_ROWS;
+                if (nb0 >= p.N) break;                       // same rule as the loader
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
+                if (!ok) break;
+                const int nb = nb0 + grp * RPG;
+                const float *sx = reinterpret_cast<const float *>(st_ptr + (size_t)stage * WU_STATE_BYTES) +
+                                  grp * RPG * UM_BM + col;
+                float xv[RPG], yv[RPG], zv[RPG];
+#pragma unroll
+                for (int j = 0; j < RPG; ++j) {
+                    xv[j] = sx[j * UM_BM];
+                    if (!FIRST) {
+                        yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
+                        zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
+                    }
+                }
+                uint32_t r[RPG];
+                tc_ld_32x4(tmem_base + ((uint32_t)(q * 32) << 16) +
+                           (uint32_t)(acc * UM_BN + c * WU_CHUNK_ROWS + grp * RPG), r);
+                tc_wait_ld();
+                // the values are in registers: hand the stage back to the loader
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
+                if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
+                if (m_ok) {
+                    const long long e0 = (long long)g * p.gs + (long long)nb * p.ld + m;
+                    float *yp = p.y + e0, *zp = p.z + e0;
+                    __nv_bfloat16 *sp = p.shadow + e0;
+#pragma unroll
+                    for (int j = 0; j < RPG; ++j) {
+                        if (nb + j < p.N) {
+                            const long long o = (long long)j * p.ld;
+                            const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
+                            const float yn = yo - p.eta_p * fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j]));
+                            const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
+                            fin &= (fabsf(yn) <= 3.402823466e+38f);
+                            __stcs(yp + o, yn);
+                            __stcs(zp + o, zn);
+                            sp[o] = __float2bfloat16_rn(yn);
+                        }
+                    }
+                }
+            }
+            if (!ok) break;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (!fin) p.status[SLOT_NONFINITE] = 1;
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) p.status[SLOT_WAIT_LIMIT] = 1;
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)UM_TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace parle
