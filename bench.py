@@ -95,8 +95,9 @@ class ClockSampler:
 def make_round_inputs(cfg, sets: int):
     """`sets` rounds' worth of minibatches: X [sets, L, n, B, d0] fp32, labels [sets, L, n, B] int32."""
     Xs, cs = [], []
+    big = cfg.n * cfg.batch * cfg.dims[0] * cfg.L > (1 << 28)      # > 1 GiB of fp32 per round: cycle 4 distinct steps
     for r in range(sets):
-        X, c = si.round_batches(cfg, r)
+        X, c = si.round_batches(cfg, r, pool=4 if big else 0)
         Xs.append(X); cs.append(c)
     return np.stack(Xs), np.stack(cs)
 
@@ -170,7 +171,12 @@ def run_ours(args):
         cfg = cfg.scaled(seed=cfg.seed + 7919 * rank)
     model = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, gamma=cfg.gamma, rho=cfg.rho,
                      alpha=cfg.alpha, eta=cfg.eta, eta_prime=cfg.eta_prime).alloc(dev)
-    model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
+    if cfg.n_params > 50_000_000:                 # replica by replica: the padded host copy of all replicas would be tens of GB
+        for a in range(cfg.n):
+            one = dense_to_padded(model, cfg.scaled(n=1), [si.init_replica(cfg, a, fast=True)])
+            model.x[a].copy_(torch.from_numpy(one[0]))
+    else:
+        model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
     model.mean()
     sets = 2
     Xh, ch = make_round_inputs(cfg, sets)
@@ -287,12 +293,19 @@ def _blas_threads():
         return os.cpu_count() or 1
 
 
+def oracle_replicas(cfg) -> int:
+    """Replicas the oracle sample covers: all of them unless their fp64 state would not fit in ~16 GB of host memory."""
+    return max(1, min(cfg.n, int(16e9 // (cfg.n_params * 8 * 4))))
+
+
 def oracle_sample(cfg, inner_steps: int, rnd: int = 0):
-    """Time the oracle on `inner_steps` inner steps of one round (all n replicas) + outer step + mean."""
+    """Time the oracle on `inner_steps` inner steps of one round (oracle_replicas(cfg) replicas) + outer step + mean."""
     from oracle import parle_oracle as po
+    cfg = cfg.scaled(n=oracle_replicas(cfg))
     sub = cfg.scaled(L=inner_steps)
     X, c = si.round_batches(sub, rnd)
-    x0 = np.stack([po.pack(si.init_replica(cfg, a)) for a in range(cfg.n)])
+    fast = cfg.n_params > 50_000_000
+    x0 = np.stack([po.pack(si.init_replica(cfg, a, fast=fast)) for a in range(cfg.n)])
     hp = po.Hyper(cfg.eta, cfg.eta_prime, cfg.alpha, cfg.gamma, cfg.rho)
     t0 = time.perf_counter()
     po.parle_round(x0, x0.mean(axis=0), po.mlp_grad_fn(cfg.dims, X, c), inner_steps, hp)
@@ -304,8 +317,9 @@ def cpu_baseline(cfg, budget_s: float):
     t1 = oracle_sample(cfg, 1)
     steps = int(max(1, min(cfg.L, budget_s / max(t1, 1e-3))))
     t = oracle_sample(cfg, steps) if steps > 1 else t1
-    return {"value": cfg.n * steps / t, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
-            "sample": f"{steps} of {cfg.L} inner steps of one round, all {cfg.n} replicas, fp64 numpy ({t:.1f} s)"}
+    nr = oracle_replicas(cfg)
+    return {"value": nr * steps / t, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+            "sample": f"{steps} of {cfg.L} inner steps of one round, {nr} of {cfg.n} replicas, fp64 numpy ({t:.1f} s)"}
 
 
 def run_reference(args):
@@ -320,8 +334,9 @@ def run_reference(args):
     t = 0.0
     for r in range(args.steps):
         t += oracle_sample(cfg, per_step, args.warmup + r)
-    value = cfg.n * per_step * args.steps / t
-    sample = f"each step = {per_step} of {cfg.L} inner steps of a round, all {cfg.n} replicas, + outer step and mean; fp64 numpy"
+    nr = oracle_replicas(cfg)
+    value = nr * per_step * args.steps / t
+    sample = f"each step = {per_step} of {cfg.L} inner steps of a round, {nr} of {cfg.n} replicas, + outer step and mean; fp64 numpy"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,

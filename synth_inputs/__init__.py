@@ -151,17 +151,25 @@ SWEEP_N = (3, 8, 16)
 # Parameters, minibatches, labels
 # --------------------------------------------------------------------------
 
-def init_layer(cfg: ParleConfig, replica: int, layer: int) -> Tuple[np.ndarray, np.ndarray]:
-    """Initial W_l ~ N(0, 1/fan_in) as [d_l, d_{l-1}] fp32 and b_l = 0."""
+def init_layer(cfg: ParleConfig, replica: int, layer: int, fast: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+    """Initial W_l ~ N(0, 1/fan_in) as [d_l, d_{l-1}] fp32 and b_l = 0.
+
+    fast=True draws the same distribution from numpy's Philox bit generator keyed by the
+    same stream key (about 20x quicker; for the 243 M-parameter workload)."""
     d_in, d_out = cfg.dims[layer], cfg.dims[layer + 1]
     key = stream_key(cfg.seed, TAG_PARAM_W, replica, layer)
-    W = normal_f32(key, (d_out, d_in), std=d_in ** -0.5)
+    if fast:
+        rng = np.random.Generator(np.random.Philox(key=key))
+        W = rng.standard_normal((d_out, d_in), dtype=np.float32)
+        W *= np.float32(d_in ** -0.5)
+    else:
+        W = normal_f32(key, (d_out, d_in), std=d_in ** -0.5)
     b = np.zeros(d_out, dtype=np.float32)
     return W, b
 
 
-def init_replica(cfg: ParleConfig, replica: int) -> List[Tuple[np.ndarray, np.ndarray]]:
-    return [init_layer(cfg, replica, l) for l in range(cfg.n_layers)]
+def init_replica(cfg: ParleConfig, replica: int, fast: bool = False) -> List[Tuple[np.ndarray, np.ndarray]]:
+    return [init_layer(cfg, replica, l, fast) for l in range(cfg.n_layers)]
 
 
 def _teacher_weights(cfg: ParleConfig) -> List[np.ndarray]:
@@ -201,11 +209,17 @@ def minibatch(cfg: ParleConfig, replica: int, rnd: int, step: int,
     return X, teacher_labels(cfg, X)
 
 
-def round_batches(cfg: ParleConfig, rnd: int, shared: bool = False):
-    """X [L, n, batch, d_0] fp32 and labels [L, n, batch] int32 for one round."""
+def round_batches(cfg: ParleConfig, rnd: int, shared: bool = False, pool: int = 0):
+    """X [L, n, batch, d_0] fp32 and labels [L, n, batch] int32 for one round.
+
+    pool > 0: only `pool` distinct inner steps are drawn and cycled through the L steps
+    (for the largest workload, where a round of fresh minibatches is gigabytes)."""
     X = np.empty((cfg.L, cfg.n, cfg.batch, cfg.dims[0]), dtype=np.float32)
     c = np.empty((cfg.L, cfg.n, cfg.batch), dtype=np.int32)
     for l in range(cfg.L):
+        if pool and l >= pool:
+            X[l], c[l] = X[l % pool], c[l % pool]
+            continue
         for a in range(cfg.n):
             X[l, a], c[l, a] = minibatch(cfg, a, rnd, l, shared)
     return X, c
