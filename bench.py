@@ -57,7 +57,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.index)],
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i", str(self.index)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -148,6 +148,16 @@ def algorithmic_bytes_per_round(cfg, stride):
         out["fwd_gemm"] = n * L * (2 * Pw + sum(2 * act(l) + 4 * act(l + 1) for l in range(nl)))
         out["dgrad_gemm"] = n * L * sum(2 * dims[l] * dims[l + 1] + 2 * act(l + 1) + 6 * act(l) for l in range(1, nl))
     return out
+
+
+def gemm_flops_per_round(cfg):
+    """Floating-point operations of the forward / data-gradient / weight-gradient products per round (all replicas)."""
+    n, B, L, dims = cfg.n, cfg.batch, cfg.L, cfg.dims
+    nl = len(dims) - 1
+    Pw = sum(dims[l] * dims[l + 1] for l in range(nl))
+    f = {"fwd_gemm": 2 * B * Pw, "dgrad_gemm": 2 * B * (Pw - dims[0] * dims[1]), "wgrad_gemm": 2 * B * Pw,
+         "wgrad_gemm_fused_update": 2 * B * Pw}
+    return {k: v * n * L for k, v in f.items()}
 
 
 # ------------------------------------------------------------------ our arm
@@ -260,6 +270,13 @@ def run_ours(args):
                         "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, k),
                         "peak_source": peaks["source"], "bytes_per_launch": alg[k] * K / cnt_k,
                         "ms_per_launch": ms_k / cnt_k, "launches_per_round": cnt_k / K}
+    flops = gemm_flops_per_round(cfg)
+    for k, f in flops.items():
+        if k in prof and k in rooflines:
+            tf = f * K / (prof[k][0] * 1e-3) / 1e12
+            rooflines[k]["tensor_tflops"] = tf
+            rooflines[k]["tensor_frac_of_burst_peak"] = tf / peaks["bf16_tflops"]
+            rooflines[k]["tensor_frac_of_sustained_peak"] = tf / peaks["bf16_tflops_sustained"]
     roofline = rooflines.get(dom, {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": None, "traffic": None, "peak_source": peaks["source"]})
     cpu = cpu_baseline(cfg, budget_s=15.0)
@@ -352,7 +369,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))

@@ -418,10 +418,10 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         const int grid = tiles < c->sm_count ? tiles : c->sm_count;
         prof_begin(c, KC_WGRAD_UPDATE);
         if (c->fresh)
-            umma_wgrad_update_kernel<true><<<grid, WU_THREADS, WU_SMEM_BYTES, c->stream>>>(
+            umma_wgrad_update_kernel<true, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
                 c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], p);
         else
-            umma_wgrad_update_kernel<false><<<grid, WU_THREADS, WU_SMEM_BYTES, c->stream>>>(
+            umma_wgrad_update_kernel<false, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
                 c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], p);
         PARLE_LAUNCHED(c);
     }
@@ -558,8 +558,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, false>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, false>()));
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WU_SMEM_BYTES));
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WU_SMEM_BYTES));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
         PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, true>()));
         PARLE_TRY(build_tensor_maps(c));
     }

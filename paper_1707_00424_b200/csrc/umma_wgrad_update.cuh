@@ -11,7 +11,7 @@
 //
 // This is a streaming kernel with a small GEMM inside (K = batch): 22 bytes per
 // weight go through the epilogue.  To keep enough bytes in flight, x, y and z
-// tiles are not loaded through registers: a loader warp brings 16-row x 128-col
+// tiles are not loaded through registers: a loader warp brings 32-row x 128-col
 // fp32 boxes of x, y, z into a ring of shared-memory stages with TMA, running
 // several stages ahead of the epilogue warps, which read them conflict-free
 // (consecutive lanes -> consecutive words), combine them with the accumulator
@@ -21,7 +21,7 @@
 // Roles: warp 0 operand TMA producer, warp 1 MMA issuer, warp 2 state loader,
 // warps 3.. epilogue: G groups of 4 warps (the four 32-lane quarters of tensor
 // memory).  Every epilogue warp consumes every chunk, in order -- group g takes
-// rows 4g .. 4g+3 of the chunk's 16 -- so each stage barrier sees all its
+// its own slice of the chunk's rows -- so each stage barrier sees all its
 // consumers in every phase and no waiter can fall a phase behind.
 // All waits are bounded.
 #pragma once
@@ -30,16 +30,35 @@
 
 namespace parle {
 
-constexpr int WU_CHUNK_ROWS = 16;                              // W rows (accumulator columns) per epilogue chunk
-constexpr int WU_CHUNKS = UM_BN / WU_CHUNK_ROWS;               // 8 per 128x128 tile
 constexpr int WU_OP_STAGES = 2;                                // operand ring (K = batch is short)
-constexpr int WU_ARRAY_BYTES = WU_CHUNK_ROWS * UM_BM * 4;      // 8 KiB: one fp32 box of x, y or z
-constexpr int WU_STATE_BYTES = 3 * WU_ARRAY_BYTES;             // x | y | z
-constexpr int WU_STATE_STAGES = 6;
-constexpr int WU_GROUPS = 4;                                   // epilogue warp groups
-constexpr int WU_THREADS = 96 + 128 * WU_GROUPS;
-constexpr size_t WU_SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)WU_STATE_STAGES * WU_STATE_BYTES +
-                                 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int WU_STATE_RING_BYTES = 144 * 1024;                // shared memory given to the x/y/z stages
+
+// Shape of the epilogue: G groups of 4 warps share chunks of CR W-rows (accumulator columns);
+// every thread owns CR / G rows of one column.
+template <int G, int CR>
+struct WuShape {
+    static constexpr int GROUPS = G, CHUNK_ROWS = CR, RPG = CR / G;
+    static constexpr int CHUNKS = UM_BN / CR;
+    static constexpr int ARRAY_BYTES = CR * UM_BM * 4;          // one fp32 box of x, y or z
+    static constexpr int STATE_BYTES = 3 * ARRAY_BYTES;         // x | y | z
+    static constexpr int STAGES = WU_STATE_RING_BYTES / STATE_BYTES;
+    static constexpr int THREADS = 96 + 128 * G;
+    static constexpr size_t SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)STAGES * STATE_BYTES +
+                                         1024 /*alignment slack*/ + 256 /*barriers*/;
+    static_assert(RPG == 4 || RPG == 8 || RPG == 16, "rows per thread must match a tcgen05.ld shape");
+    static_assert(STAGES >= 2 && 2 * WU_OP_STAGES + 4 + 2 * STAGES <= 30, "stage count");
+};
+using WuDefault = WuShape<4, 32>;
+constexpr int WU_CHUNK_ROWS = WuDefault::CHUNK_ROWS;           // TMA box height of the x/y/z tensor maps
+
+template <int N> __device__ __forceinline__ void tc_ld_cols(uint32_t taddr, uint32_t (&r)[N]);
+template <> __device__ __forceinline__ void tc_ld_cols<4>(uint32_t taddr, uint32_t (&r)[4]) { tc_ld_32x4(taddr, r); }
+template <> __device__ __forceinline__ void tc_ld_cols<8>(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+template <> __device__ __forceinline__ void tc_ld_cols<16>(uint32_t taddr, uint32_t (&r)[16]) { tc_ld_32x16(taddr, r); }
 
 struct WgradUpdateParams {
     int M, N, K;                 // M = d_in (tile rows), N = d_out (tile columns), K = batch
@@ -51,11 +70,14 @@ struct WgradUpdateParams {
     int *status;
 };
 
-template <bool FIRST>
-__global__ void __launch_bounds__(WU_THREADS, 1)
+template <bool FIRST, class SH>
+__global__ void __launch_bounds__(SH::THREADS, 1)
 umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
                          const __grid_constant__ CUtensorMap tmZ, const WgradUpdateParams p) {
+    constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
+    constexpr int WU_STATE_BYTES = SH::STATE_BYTES, WU_STATE_STAGES = SH::STAGES, RPG = SH::RPG;
+    constexpr int WU_CHUNK_ROWS = SH::CHUNK_ROWS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t op_base = (raw + 1023u) & ~1023u;
@@ -183,12 +205,12 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // ------------------------------------------------ epilogue groups
         const int q = warp & 3;                              // tensor-memory lane quarter of this warp
         const int grp = (warp - 3) >> 2;                     // rows grp*RPG .. of every chunk
-        constexpr int RPG = WU_CHUNK_ROWS / WU_GROUPS;       // rows per group and chunk
-        static_assert(RPG == 4, "tcgen05.ld shape below reads 4 columns");
         const float one_m_alpha = 1.0f - p.alpha;
+        const float neg_eta_p = -p.eta_p;
         int acc = 0; uint32_t acc_phase = 0;
         int stage = 0; uint32_t sphase = 0;                  // state ring position: every warp walks every chunk
-        bool fin = true, ok = true;
+        float chk = 0.f;                                     // 0 * y summed: turns NaN as soon as a y is NaN or Inf
+        bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             int g, m0, n0; coords(t, g, m0, n0);
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
@@ -197,8 +219,12 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             const int col = q * 32 + lane;                   // tile column along d_in
             const int m = m0 + col;
             const bool m_ok = m < p.M;
+            const long long tile_e0 = (long long)g * p.gs + (long long)(n0 + grp * RPG) * p.ld + m;
+            const long long chunk_step = (long long)WU_CHUNK_ROWS * p.ld;
+            float *yp = p.y + tile_e0, *zp = p.z + tile_e0;
+            __nv_bfloat16 *sp = p.shadow + tile_e0;
 #pragma unroll 1
-            for (int c = 0; c < WU_CHUNKS; ++c) {
+            for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += chunk_step) {
                 const int nb0 = n0 + c * WU_CHUNK_ROWS;
                 if (nb0 >= p.N) break;                       // same rule as the loader
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
@@ -216,28 +242,38 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     }
                 }
                 uint32_t r[RPG];
-                tc_ld_32x4(tmem_base + ((uint32_t)(q * 32) << 16) +
-                           (uint32_t)(acc * UM_BN + c * WU_CHUNK_ROWS + grp * RPG), r);
+                tc_ld_cols<RPG>(tmem_base + ((uint32_t)(q * 32) << 16) +
+                                (uint32_t)(acc * UM_BN + c * WU_CHUNK_ROWS + grp * RPG), r);
                 tc_wait_ld();
                 // the values are in registers: hand the stage back to the loader
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
                 if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
-                if (m_ok) {
-                    const long long e0 = (long long)g * p.gs + (long long)nb * p.ld + m;
-                    float *yp = p.y + e0, *zp = p.z + e0;
-                    __nv_bfloat16 *sp = p.shadow + e0;
+                const int rows = m_ok ? (p.N - nb) : 0;      // rows of this thread that exist
+                float *yr = yp, *zr = zp;
+                __nv_bfloat16 *sr = sp;
+                if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j) {
-                        if (nb + j < p.N) {
-                            const long long o = (long long)j * p.ld;
+                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += p.ld) {
+                        const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
+                        const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j])), yo);
+                        const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
+                        chk = fmaf(yn, 0.f, chk);
+                        *yr = yn;
+                        *zr = zn;
+                        *sr = __float2bfloat16_rn(yn);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += p.ld) {
+                        if (j < rows) {
                             const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
-                            const float yn = yo - p.eta_p * fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j]));
+                            const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j])), yo);
                             const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
-                            fin &= (fabsf(yn) <= 3.402823466e+38f);
-                            __stcs(yp + o, yn);
-                            __stcs(zp + o, zn);
-                            sp[o] = __float2bfloat16_rn(yn);
+                            chk = fmaf(yn, 0.f, chk);
+                            *yr = yn;
+                            *zr = zn;
+                            *sr = __float2bfloat16_rn(yn);
                         }
                     }
                 }
@@ -248,7 +284,7 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
-        if (!fin) p.status[SLOT_NONFINITE] = 1;
+        if (chk != 0.f) p.status[SLOT_NONFINITE] = 1;        // NaN != 0 is true
     }
 
     tc_fence_before();
