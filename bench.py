@@ -165,6 +165,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     import paper_1707_00424_b200 as pb
+    from paper_1707_00424_b200.parallel import allreduce_mean_
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -203,7 +204,7 @@ def run_ours(args):
 
     def exchange():
         if world > 1:       # global mean = mean over ranks of the per-rank means (equal replica counts)
-            dist.all_reduce(model.xbar, op=dist.ReduceOp.AVG)
+            allreduce_mean_(model.xbar)
 
     def round_device(r):
         model.round(cfg.L, Xd[r % sets], cd[r % sets], loss_d)

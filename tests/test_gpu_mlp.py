@@ -347,3 +347,63 @@ def test_layerwise_teacher_forced_c3_bf16():
 
 def test_layerwise_teacher_forced_ragged_bf16():
     _layerwise_bf16(si.C1.scaled(name="bf16-ragged", n=2, dims=(200, 328, 136, 101), batch=136, gemm_dtype=1))
+
+
+# ------------------------------------------------------------------ the 243 M-parameter shape
+def test_c5_widths_div8_round_bf16():
+    """Same depth, replica count and batch as the largest workload, widths / 8 (a full fp64 round at
+    full width is ~1e17 flop): whole-round parity, fused update."""
+    cfg = si.C5.scaled(name="C5/8", dims=(512, 1024, 1024, 1024, 1024, 125), L=5)
+    run_rounds(cfg, 1, disp_tol=5e-2, use_round_call=True)
+
+
+def test_c5_full_shape_sampled_outputs_bf16():
+    """Full width, batch 256 (two M-tiles per weight tile, 64 x 64 weight tiles per layer), one replica:
+    sampled entries of every GEMM output of one inner step are recomputed in fp64 from the operands the
+    GPU used; plus the fused path against the separate update on the whole 243 M-element vector."""
+    cfg = si.C5.scaled(n=1, L=1)
+    rng = np.random.default_rng(5)
+    q = po.round_to_bf16
+    X, c = si.round_batches(cfg, 0)
+    Xd, cd = torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV)
+    layers = si.init_replica(cfg, 0, fast=True)
+    states = []
+    for fused in (False, True):
+        m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype).alloc(DEV)
+        m.set_fused_update(fused)
+        for l, (W, b) in enumerate(layers):
+            w_off, b_off = m.layer_offset(l)
+            m.x[0, w_off:w_off + W.size].copy_(torch.from_numpy(W.ravel()))
+        m.mean(); m.round_begin(); m.inner_step(Xd, cd); torch.cuda.synchronize()
+        assert m.status() == 0
+        states.append((m.y.clone(), m.z.clone()))
+        if fused:
+            break
+        nl, B = cfg.n_layers, cfg.batch
+        f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+        H = [q(X[0, 0].astype(np.float64))] + [f64(m.debug_buffer(m.DBG_ACT, l))[0] for l in range(nl - 1)]
+        dH = [f64(m.debug_buffer(m.DBG_DACT, l))[0] for l in range(nl)]
+        logits = f64(m.debug_buffer(m.DBG_LOGITS))[0]
+        grad = m.grad[0].cpu().numpy().astype(np.float64)
+        for l in range(nl):
+            din, dout = cfg.dims[l], cfg.dims[l + 1]
+            Wq = q(layers[l][0].astype(np.float64))
+            i = rng.integers(0, B, 64); j = rng.integers(0, dout, 64); k = rng.integers(0, din, 64)
+            pre = np.einsum("sk,sk->s", H[l][i], Wq[j])          # forward entries (i, j)
+            if l + 1 < nl:
+                want, got = q(np.maximum(pre, 0.0)), H[l + 1][i, j]
+                assert np.all(np.abs(got - want) <= 2.0 ** -7 * np.abs(want) + 1e-5 * np.sqrt(np.mean(H[l + 1] ** 2))), ("H", l)
+            else:
+                assert np.allclose(logits[i, j], pre, rtol=1e-4, atol=1e-5), "logits"
+            w_off, _ = m.layer_offset(l)
+            dW = grad[w_off:w_off + dout * din].reshape(dout, din)
+            want = np.einsum("bs,bs->s", dH[l][:, j], H[l][:, k])  # weight-gradient entries (j, k)
+            assert np.allclose(dW[j, k], want, rtol=1e-4, atol=1e-9), ("dW", l)
+            if l > 0:
+                want = q(np.einsum("sj,js->s", dH[l][i], Wq[:, k]) * (H[l][i, k] > 0))   # data-gradient entries (i, k)
+                got = dH[l - 1][i, k]
+                assert np.all(np.abs(got - want) <= 2.0 ** -7 * np.abs(want) + 1e-5 * np.sqrt(np.mean(dH[l - 1] ** 2))), ("dH", l)
+        del m
+        torch.cuda.empty_cache()
+    for a, b in zip(*states):
+        assert torch.equal(a, b)
