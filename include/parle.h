@@ -196,7 +196,8 @@ const char *parle_profile_class_name(int k);
  *   PARLE_DBG_DACT    gradient w.r.t. layer's output   [n, B, ld]  fp32 (ld = d) or bf16 (ld = d rounded up to 8)
  *   PARLE_DBG_DACT_T  its transposed copy (bf16 path)  [n, d, B]   bf16
  *   PARLE_DBG_LOGITS  logits                            [n, B, d_last] fp32   (layer ignored)
- *   PARLE_DBG_OPERAND_COPY  bf16 copy of the vector the GEMMs read [n, stride] (bf16 path; layer ignored)
+ *   PARLE_DBG_OPERAND_COPY  bf16 copy of the weights the GEMMs read, stored per layer in 128-row x 64-column
+ *                           blocks (row-block major), [n, bytes/(2n)] (bf16 path; layer ignored)
  * EINVAL if that buffer does not exist in this configuration. */
 #define PARLE_DBG_ACT 0
 #define PARLE_DBG_ACT_T 1

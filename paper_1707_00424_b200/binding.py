@@ -242,7 +242,7 @@ class Parle:
         if kind == self.DBG_LOGITS:
             return raw.view(torch.float32).view(n, B, self.dims[-1])
         if kind == self.DBG_OPERAND_COPY:
-            return raw.view(torch.bfloat16).view(n, self.stride)
+            return raw.view(torch.bfloat16).view(n, -1)
         if kind in (self.DBG_ACT_T, self.DBG_DACT_T):
             return raw.view(torch.bfloat16).view(n, d, B)
         t = raw.view(torch.bfloat16 if bf else torch.float32)

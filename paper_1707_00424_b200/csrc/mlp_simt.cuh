@@ -183,8 +183,7 @@ struct TailPlan {
 template <bool FIRST>
 __global__ void __launch_bounds__(256)
 tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__ z, const float *__restrict__ x,
-                   __nv_bfloat16 *__restrict__ shadow, long long stride, float eta_p, float inv_gamma,
-                   float alpha, int *status) {
+                   long long stride, float eta_p, float inv_gamma, float alpha, int *status) {
     const int l = blockIdx.y, g = blockIdx.z;
     const int lane = threadIdx.x % 32;
     const long long e = tp.begin[l] + (long long)blockIdx.x * 8 + threadIdx.x / 32;
@@ -204,8 +203,41 @@ tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__
         const float zn = fmaf(alpha, zo, (1.0f - alpha) * yn);
         y[i] = yn;
         z[i] = zn;
-        shadow[i] = __float2bfloat16_rn(yn);
         if (!(fabsf(yn) <= 3.402823466e+38f)) status[SLOT_NONFINITE] = 1;
+    }
+}
+
+// bf16 operand copy of the weights in blocked layout: W_l [d_out, d_in] row-major fp32 ->
+// blocks of 128 rows x 64 columns (16 KiB of bf16 each), row-block major; element (r, c) of layer l at
+//   sh_off[l] + ((r/128) * cb[l] + c/64) * 8192 + (r%128) * 64 + c%64.
+// One CTA per block; rows and columns beyond the matrix are never written (they stay zero).
+struct BlockedPlan {
+    int n_layers;
+    long long w_off[PARLE_MAX_LAYERS], sh_off[PARLE_MAX_LAYERS];
+    int d_in[PARLE_MAX_LAYERS], d_out[PARLE_MAX_LAYERS], cb[PARLE_MAX_LAYERS], first_block[PARLE_MAX_LAYERS + 1];
+};
+
+__global__ void __launch_bounds__(256)
+blocked_bf16_kernel(const BlockedPlan bp, const float *__restrict__ src, long long stride,
+                    __nv_bfloat16 *__restrict__ dst, long long sh_stride) {
+    const int g = blockIdx.y;
+    int l = 0;
+    while (l + 1 < bp.n_layers && (int)blockIdx.x >= bp.first_block[l + 1]) ++l;
+    const int blk = blockIdx.x - bp.first_block[l];
+    const int rb = blk / bp.cb[l], cb = blk % bp.cb[l];
+    const float *W = src + (long long)g * stride + bp.w_off[l];
+    __nv_bfloat16 *out = dst + (long long)g * sh_stride + bp.sh_off[l] + (long long)blk * 8192;
+    const int c4 = (threadIdx.x % 16) * 4;                   // 16 threads x 4 columns = one 64-column row of the block
+    const int col = cb * 64 + c4;
+    for (int r = threadIdx.x / 16; r < 128; r += 16) {
+        const int row = rb * 128 + r;
+        if (row < bp.d_out[l] && col < bp.d_in[l]) {          // d_in % 8 == 0: the 4 columns are all inside
+            const float4 v = *reinterpret_cast<const float4 *>(W + (long long)row * bp.d_in[l] + col);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t *>(&lo); pk.y = *reinterpret_cast<uint32_t *>(&hi);
+            *reinterpret_cast<uint2 *>(out + r * 64 + c4) = pk;
+        }
     }
 }
 

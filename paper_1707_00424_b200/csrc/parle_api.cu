@@ -30,7 +30,7 @@ struct Workspace {
     size_t act[PARLE_MAX_LAYERS];      // fp32 mode: output of layer l  [n,B,d_{l+1}] fp32 (last = logits)
     size_t dact[PARLE_MAX_LAYERS];     // fp32 mode: gradient w.r.t. layer l's output [n,B,d_{l+1}] fp32
     size_t logits;                     // bf16 mode: fp32 logits [n,B,C]
-    size_t shadow;                     // bf16 mode: bf16 copy of the GEMM operand vector [n,stride]
+    size_t shadow;                     // bf16 mode: blocked bf16 copy of the weights [n, sh_stride]
     size_t xb, xbT;                    // bf16 mode: inputs [n,B,d_0] and transposed [n,d_0,B]
     size_t hb[PARLE_MAX_LAYERS], hbT[PARLE_MAX_LAYERS];      // hidden activations, both layouts
     size_t dhb[PARLE_MAX_LAYERS], dhbT[PARLE_MAX_LAYERS];    // their gradients, both layouts
@@ -47,6 +47,8 @@ struct parle_ctx {
     int dims[PARLE_MAX_LAYERS + 1];
     float inv_gamma, inv_rho, alpha, eta, eta_prime;
     size_t P, stride;
+    size_t sh_stride;                // bf16 path: elements of one replica's blocked weight copy
+    size_t sh_off[PARLE_MAX_LAYERS]; int sh_cb[PARLE_MAX_LAYERS], sh_rb[PARLE_MAX_LAYERS];   // per layer: offset, column / row blocks
     LayerPlan layers[PARLE_MAX_LAYERS];
     Workspace ws;
     bool bound;
@@ -114,7 +116,7 @@ void plan_workspace(parle_ctx *c) {
         for (int l = 0; l < nl; ++l) w.act[l] = take(n * B * c->dims[l + 1] * sizeof(float));
         for (int l = 0; l < nl; ++l) w.dact[l] = take(n * B * c->dims[l + 1] * sizeof(float));
     } else {
-        w.shadow = take(n * c->stride * 2);
+        w.shadow = take(n * c->sh_stride * 2);
         w.xb = take(n * B * c->dims[0] * 2);
         w.xbT = take(n * B * c->dims[0] * 2);
         for (int l = 0; l + 1 < nl; ++l) {
@@ -193,6 +195,23 @@ int encode_f32_map(parle_ctx *c, CUtensorMap *tm, const void *base, size_t cols,
     return PARLE_OK;
 }
 
+// Blocked bf16 weight copy of one layer as a 5-D tensor (column in block, row in block, column block,
+// row block, replica); box = box_rows x 64 columns of one block, 128-byte swizzle, zero fill outside.
+int encode_blocked_map(parle_ctx *c, CUtensorMap *tm, const void *base, int cb, int rb, size_t groups,
+                       size_t group_pitch, unsigned box_rows) {
+    EncodeTiledFn enc;
+    PARLE_TRY(get_encoder(c, &enc));
+    cuuint64_t dims[5] = {64, 128, (cuuint64_t)cb, (cuuint64_t)rb, groups};
+    cuuint64_t strides[4] = {128, 16384, (cuuint64_t)cb * 16384, group_pitch * 2};
+    cuuint32_t box[5] = {64, box_rows, 1, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
+    return PARLE_OK;
+}
+
 int build_tensor_maps(parle_ctx *c) {
     const Workspace &w = c->ws;
     const size_t n = c->n, B = c->batch;
@@ -201,10 +220,10 @@ int build_tensor_maps(parle_ctx *c) {
         const size_t din = c->dims[l], dout = c->dims[l + 1];
         const __nv_bfloat16 *a_in = l == 0 ? ws_ptr<__nv_bfloat16>(c, w.xb) : ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]);
         const __nv_bfloat16 *a_inT = l == 0 ? ws_ptr<__nv_bfloat16>(c, w.xbT) : ws_ptr<__nv_bfloat16>(c, w.hbT[l - 1]);
-        const __nv_bfloat16 *W = shadow + c->layers[l].w_off;
+        const __nv_bfloat16 *W = shadow + c->sh_off[l];
         // forward: A = layer input [B, din], B = W [dout, din], both K-major (K = din)
         PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_a[l], a_in, din, B, n, din, B * din, UM_BK, UM_BM));
-        PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_b[l], W, din, dout, n, din, c->stride, UM_BK, UM_BN));
+        PARLE_TRY(encode_blocked_map(c, &c->tm_fwd_b[l], W, c->sh_cb[l], c->sh_rb[l], n, c->sh_stride, 128));
         // weight gradient, computed transposed (dW^T = input^T dH): A = input^T [din, B], B = dH^T [dout, B],
         // both K-major (K = batch)
         PARLE_TRY(encode_bf16_map(c, &c->tm_wg_a[l], a_inT, B, din, n, B, din * B, UM_BK, UM_BM));
@@ -219,13 +238,13 @@ int build_tensor_maps(parle_ctx *c) {
             // fetched as 64 k-rows x 64 n-columns boxes
             PARLE_TRY(encode_bf16_map(c, &c->tm_dg_a[l], ws_ptr<__nv_bfloat16>(c, w.dhb[l]), dout, B, n,
                                       w.dh_ld[l], B * (size_t)w.dh_ld[l], UM_BK, UM_BM));
-            PARLE_TRY(encode_bf16_map(c, &c->tm_dg_b[l], W, din, dout, n, din, c->stride, 64, UM_BK));
+            PARLE_TRY(encode_blocked_map(c, &c->tm_dg_b[l], W, c->sh_cb[l], c->sh_rb[l], n, c->sh_stride, 64));
         }
     }
     return PARLE_OK;
 }
 
-template <int EPI, bool B_MN>
+template <int EPI, int BKIND>
 int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
     p.groups = c->n;
     p.tiles_m = (p.M + UM_BM - 1) / UM_BM;
@@ -234,14 +253,14 @@ int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &
     const int tiles = p.groups * p.tiles_m * p.tiles_n;
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     prof_begin(c, cls);
-    umma_gemm_kernel<EPI, B_MN><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
+    umma_gemm_kernel<EPI, BKIND><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
 
-template <int EPI, bool B_MN>
+template <int EPI, int BKIND>
 cudaError_t allow_big_smem() {
-    return cudaFuncSetAttribute(umma_gemm_kernel<EPI, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(umma_gemm_kernel<EPI, BKIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)UM_SMEM_BYTES);
 }
 
@@ -263,6 +282,26 @@ inline int stream_grid(const parle_ctx *c, size_t items, int per_thread) {
 }
 
 // ---------------------------------------------------------------- the steps
+// Refresh the blocked bf16 weight copy from an fp32 vector (x at the start of a round; y after a
+// separate update step).
+int run_blocked_copy(parle_ctx *c, const float *src) {
+    BlockedPlan bp = {};
+    bp.n_layers = c->n_layers;
+    int blocks = 0;
+    for (int l = 0; l < c->n_layers; ++l) {
+        bp.w_off[l] = (long long)c->layers[l].w_off; bp.sh_off[l] = (long long)c->sh_off[l];
+        bp.d_in[l] = c->dims[l]; bp.d_out[l] = c->dims[l + 1]; bp.cb[l] = c->sh_cb[l];
+        bp.first_block[l] = blocks;
+        blocks += c->sh_rb[l] * c->sh_cb[l];
+    }
+    bp.first_block[c->n_layers] = blocks;
+    prof_begin(c, KC_TO_BF16);
+    blocked_bf16_kernel<<<dim3(blocks, c->n), 256, 0, c->stream>>>(
+        bp, src, (long long)c->stride, ws_ptr<__nv_bfloat16>(c, c->ws.shadow), (long long)c->sh_stride);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+
 int run_inner_update(parle_ctx *c, const float *grad) {
     const size_t n4 = (size_t)c->n * c->stride / 4;
     constexpr int U = 2;
@@ -270,18 +309,16 @@ int run_inner_update(parle_ctx *c, const float *grad) {
     const float4 *g = reinterpret_cast<const float4 *>(grad);
     float4 *y = reinterpret_cast<float4 *>(c->buf.y), *z = reinterpret_cast<float4 *>(c->buf.z);
     const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
-    const bool sh = c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0;
-    uint2 *shadow = sh ? ws_ptr<uint2>(c, c->ws.shadow) : nullptr;
     prof_begin(c, KC_INNER_UPDATE);
-#define PARLE_UPD(F, S) inner_update_kernel<F, S, U><<<grid, kUpdThreads, 0, c->stream>>>( \
-        g, y, x, z, shadow, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev)
-    if (c->fresh) { if (sh) PARLE_UPD(true, true); else PARLE_UPD(true, false); }
-    else          { if (sh) PARLE_UPD(false, true); else PARLE_UPD(false, false); }
-#undef PARLE_UPD
+    if (c->fresh)
+        inner_update_kernel<true, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+    else
+        inner_update_kernel<false, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
     PARLE_LAUNCHED(c);
     c->fresh = false;
     c->shadow_is_x = false;
     c->steps_in_round++;
+    if (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0) PARLE_TRY(run_blocked_copy(c, c->buf.y));
     return PARLE_OK;
 }
 
@@ -358,10 +395,10 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         if (l + 1 < nl) {
             p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
             p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
-            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, false>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         } else {
             p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
-            PARLE_TRY((launch_umma<UEPI_FWD_LAST, false>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_FWD_LAST, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         }
     }
     const int C = c->dims[nl], rows = n * B;
@@ -383,7 +420,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
         d.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); d.outT_gs = (long long)B * din; d.outT_ld = B;
         d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
-        return launch_umma<UEPI_DGRAD, true>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d);
+        return launch_umma<UEPI_DGRAD, UB_BLOCKED_MN>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d);
     };
     if (!c->fused_update) {
         for (int l = nl - 1; l >= 0; --l) {
@@ -391,7 +428,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
             UmmaParams p = {};                                  // dW_l^T = H_{l-1}^T * dH_l
             p.M = din; p.N = dout; p.K = B;
             p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
-            PARLE_TRY((launch_umma<UEPI_WGRAD, false>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_WGRAD, UB_ROWMAJOR_K>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
             prof_begin(c, KC_BIAS_GRAD);
             bias_grad_bf16_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
                 ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
@@ -410,7 +447,8 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         p.M = din; p.N = dout; p.K = B;
         p.groups = n; p.tiles_m = (din + UM_BM - 1) / UM_BM; p.tiles_n = (dout + UM_BN - 1) / UM_BN;
         const size_t wo = c->layers[l].w_off;
-        p.y = c->buf.y + wo; p.z = c->buf.z + wo; p.shadow = shadow + wo;
+        p.y = c->buf.y + wo; p.z = c->buf.z + wo;
+        p.shadow = shadow + c->sh_off[l]; p.shadow_gs = (long long)c->sh_stride; p.shadow_cb = c->sh_cb[l];
         p.gs = S; p.ld = din;
         p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha;
         p.status = c->status_dev;
@@ -439,10 +477,10 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     const dim3 tgrid((unsigned)((longest + 7) / 8), nl, n);
     prof_begin(c, KC_TAIL_UPDATE);
     if (c->fresh)
-        tail_update_kernel<true><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, shadow, S,
+        tail_update_kernel<true><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
                                                                c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
     else
-        tail_update_kernel<false><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, shadow, S,
+        tail_update_kernel<false><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
                                                                 c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
@@ -500,6 +538,12 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         }
     }
     c->P = P; c->stride = off;
+    for (int l = 0; l < c->n_layers; ++l) {      // blocked bf16 weight copy: 128 x 64 blocks, row-block major
+        c->sh_off[l] = c->sh_stride;
+        c->sh_rb[l] = (c->dims[l + 1] + 127) / 128;
+        c->sh_cb[l] = (c->dims[l] + 63) / 64;
+        c->sh_stride += (size_t)c->sh_rb[l] * c->sh_cb[l] * 8192;
+    }
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
     plan_workspace(c);
     *out = c;
@@ -555,13 +599,15 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         int major = 0;
         PARLE_CUDA(c, cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
         if (major != 10) return PARLE_EUNSUPPORTED;             // tcgen05 kernels need sm_100
-        PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, false>()));
-        PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, false>()));
-        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, false>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, UB_BLOCKED_K>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, UB_BLOCKED_K>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, UB_ROWMAJOR_K>()));
         PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
         PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
-        PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, true>()));
+        PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, UB_BLOCKED_MN>()));
         PARLE_TRY(build_tensor_maps(c));
+        // rows / columns of the blocked weight copy beyond the matrices are never written: they must read as zero
+        PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.shadow), 0, (size_t)c->n * c->sh_stride * 2, c->stream));
     }
     c->bound = true;
     c->round_open = false; c->fresh = false; c->shadow_is_x = false; c->steps_in_round = 0;
@@ -571,11 +617,7 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
 int parle_round_begin(parle_ctx *c) {
     PARLE_TRY(check_bound(c));
     if (c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16 && !c->shadow_is_x) {
-        const size_t n4 = (size_t)c->n * c->stride / 4;
-        prof_begin(c, KC_TO_BF16);
-        to_bf16_kernel<<<stream_grid(c, n4, 1), kUpdThreads, 0, c->stream>>>(
-            reinterpret_cast<const float4 *>(c->buf.x), ws_ptr<uint2>(c, c->ws.shadow), n4);
-        PARLE_LAUNCHED(c);
+        PARLE_TRY(run_blocked_copy(c, c->buf.x));
         c->shadow_is_x = true;
     }
     c->round_open = true; c->fresh = true; c->steps_in_round = 0;
@@ -631,16 +673,11 @@ int parle_outer_step(parle_ctx *c) {
     const int grid = stream_grid(c, s4, 1);
     float4 *x = reinterpret_cast<float4 *>(c->buf.x), *xbar = reinterpret_cast<float4 *>(c->buf.xbar);
     const float4 *z = reinterpret_cast<const float4 *>(c->buf.z);
-    const bool sh = c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0;
     prof_begin(c, KC_OUTER_MEAN);
-    if (sh)
-        outer_mean_kernel<true, 4><<<grid, kUpdThreads, 0, c->stream>>>(
-            x, z, xbar, ws_ptr<uint2>(c, c->ws.shadow), s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
-    else
-        outer_mean_kernel<false, 4><<<grid, kUpdThreads, 0, c->stream>>>(
-            x, z, xbar, nullptr, s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
+    outer_mean_kernel<4><<<grid, kUpdThreads, 0, c->stream>>>(
+        x, z, xbar, s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
     PARLE_LAUNCHED(c);
-    c->shadow_is_x = sh;
+    c->shadow_is_x = false;
     c->round_open = false; c->fresh = false; c->steps_in_round = 0;
     return PARLE_OK;
 }
@@ -791,7 +828,7 @@ int parle_debug_buffer(const parle_ctx *c, int kind, int layer, size_t *byte_off
     }
     if (kind == PARLE_DBG_OPERAND_COPY) {
         if (!bf) return PARLE_EINVAL;
-        *byte_offset = w.shadow; *bytes = (size_t)c->n * c->stride * 2;
+        *byte_offset = w.shadow; *bytes = (size_t)c->n * c->sh_stride * 2;
         return PARLE_OK;
     }
     if (layer < 0 || layer >= nl) return PARLE_EINVAL;

@@ -2,12 +2,14 @@
 // forward / backward (Section 1.1 / 2.1: the minibatch gradient of f):
 //   forward      H_l      = act(H_{l-1} W_l^T + b_l)           A=[B,d_in]   K-major, B=W [d_out,d_in] K-major
 //   data grad    dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]        A=[B,d_out]  K-major, B=W [d_out(K), d_in(N)] MN-major
+//                (W is read from its bf16 operand copy, which is stored in 128-row x 64-column blocks of 16 KiB
+//                 so that every TMA box of either product is one contiguous run of memory)
 //   weight grad  dW_l^T   = H_{l-1}^T dH_l                     A=H^T [d_in,B] K-major, B=dH^T [d_out,B] K-major
 //                (computed transposed: accumulator rows = d_in, the contiguous direction of W in memory,
 //                 so the 32 lanes of an epilogue warp touch 32 consecutive floats of one W row)
 // One persistent CTA per SM walks (replica, m-tile, n-tile) work items.
-// Warp 0 stages 128x64 operand tiles with TMA (128-byte swizzle) through a ring
-// of shared-memory buffers, warp 1 issues tcgen05.mma (M=128, N=128, K=16,
+// Two producer warps stage 128x64 operand tiles with TMA (128-byte swizzle) through
+// two rings of shared-memory buffers (one per operand), warp 1 issues tcgen05.mma (M=128, N=128, K=16,
 // fp32 accumulators in tensor memory, two accumulator buffers), warps 2-5 read
 // the accumulators back with tcgen05.ld and run the fused epilogue.
 // Every wait is bounded: on a time-out the CTA records it in the status block,
@@ -19,16 +21,29 @@
 namespace parle {
 
 constexpr int UM_BM = 128, UM_BN = 128, UM_BK = 64;
-constexpr int UM_STAGES = 6;
 constexpr int UM_A_BYTES = UM_BM * UM_BK * 2;              // 16 KiB
 constexpr int UM_B_BYTES = UM_BN * UM_BK * 2;              // 16 KiB
-constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;
-// Epilogue warps: one per 32-lane quarter of tensor memory.
-__host__ __device__ constexpr int umma_epi_warps(int) { return 4; }
-__host__ __device__ constexpr int umma_threads(int epi) { return 64 + 32 * umma_epi_warps(epi); }
+constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;    // one k-block of both operands
+// The two operands have separate rings.  In the forward and data-gradient products the B operand is the
+// replica's weights, which stream from HBM exactly once (about 3 us loaded latency), while the A operand
+// (activations) is shared by all n-tiles of a replica and comes from L2: B gets the deep ring.  With
+// 8 x 16 KiB of weights in flight on every SM the weight stream is not latency-bound.
+constexpr int UM_A_STAGES = 4, UM_B_STAGES = 8;
+// Warps: 0 = B producer, 1 = MMA issuer, 2..9 = epilogue (two per 32-lane quarter of tensor memory, each taking
+// two of the four 32-column chunks of a tile), 10 = A producer.
+__host__ __device__ constexpr int umma_epi_warps(int) { return 8; }
+__host__ __device__ constexpr int umma_threads(int epi) { return 96 + 32 * umma_epi_warps(epi); }
 constexpr int UM_TMEM_COLS = 256;                          // two 128-column accumulators
-constexpr size_t UM_SMEM_BYTES = (size_t)UM_STAGES * UM_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr size_t UM_SMEM_BYTES = (size_t)UM_A_STAGES * UM_A_BYTES + (size_t)UM_B_STAGES * UM_B_BYTES +
+                                 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long UM_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
+
+// How the B operand is fetched.
+enum UmmaBKind {
+    UB_ROWMAJOR_K = 0,     // plain [rows, K] row-major tensor, K-major operand (3-D map: K, row, replica)
+    UB_BLOCKED_K = 1,      // blocked weight copy, K-major operand: box = one whole 128 x 64 block
+    UB_BLOCKED_MN = 2      // blocked weight copy, MN-major operand: boxes = 64 k-rows x 64 n-columns (half blocks)
+};
 
 enum UmmaEpilogue {
     UEPI_FWD_HIDDEN = 0,   // + bias[n], ReLU, bf16 out [M,ld] and transposed out [N,ldT]
@@ -93,6 +108,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *tm, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -162,26 +184,30 @@ __device__ __forceinline__ void tile_coords(const UmmaParams &p, int t, int &g, 
     n0 = (r / p.tiles_m) * UM_BN;
 }
 
-template <int EPI, bool B_MN>
+template <int EPI, int BKIND>
 __global__ void __launch_bounds__(umma_threads(EPI), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // 1024-byte aligned (swizzle atom)
-    uint8_t *ctl = smem_raw + (tiles_base - raw) + (size_t)UM_STAGES * UM_STAGE_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);                  // full[S], empty[S], tfull[2], tempty[2]
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * (2 * UM_STAGES + 4));
+    const uint32_t a_base = tiles_base, b_base = tiles_base + UM_A_STAGES * UM_A_BYTES;
+    uint8_t *ctl = smem_raw + (tiles_base - raw) + (size_t)UM_A_STAGES * UM_A_BYTES + (size_t)UM_B_STAGES * UM_B_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);   // a_full[SA], a_empty[SA], b_full[SB], b_empty[SB], tfull[2], tempty[2]
+    constexpr int NBARS = 2 * UM_A_STAGES + 2 * UM_B_STAGES + 4;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * NBARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * UM_STAGES;
-    const uint32_t bar_tfull = bar_empty + 8 * UM_STAGES, bar_tempty = bar_tfull + 16;
+    const uint32_t bar_afull = smem_u32(bars), bar_aempty = bar_afull + 8 * UM_A_STAGES;
+    const uint32_t bar_bfull = bar_aempty + 8 * UM_A_STAGES, bar_bempty = bar_bfull + 8 * UM_B_STAGES;
+    const uint32_t bar_tfull = bar_bempty + 8 * UM_B_STAGES, bar_tempty = bar_tfull + 16;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.groups * p.tiles_m * p.tiles_n;
     const int num_kb = (p.K + UM_BK - 1) / UM_BK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < UM_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < UM_A_STAGES; ++s) { mbar_init(bar_afull + 8 * s, 1); mbar_init(bar_aempty + 8 * s, 1); }
+        for (int s = 0; s < UM_B_STAGES; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, umma_epi_warps(EPI)); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -198,49 +224,76 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------ TMA producer
+        // ------------------------------------------------ TMA producer of the B operand (deep ring)
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 int g, m0, n0; tile_coords(p, t, g, m0, n0);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t sa = tiles_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
-                    const uint32_t fb = bar_full + 8 * stage;
-                    mbar_expect_tx(fb, UM_STAGE_BYTES);
-                    tma_load_3d(sa, &tmA, fb, kb * UM_BK, m0, g);
-                    if (!B_MN) {
+                    if (!mbar_wait(bar_bempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sb = b_base + stage * UM_B_BYTES;
+                    const uint32_t fb = bar_bfull + 8 * stage;
+                    mbar_expect_tx(fb, UM_B_BYTES);
+                    if (BKIND == UB_ROWMAJOR_K) {
                         tma_load_3d(sb, &tmB, fb, kb * UM_BK, n0, g);
+                    } else if (BKIND == UB_BLOCKED_K) {
+                        // block (row block n0/128, column block kb) of the blocked weight copy
+                        tma_load_5d(sb, &tmB, fb, 0, 0, kb, n0 / UM_BN, g);
                     } else {
-                        tma_load_3d(sb, &tmB, fb, n0, kb * UM_BK, g);
-                        tma_load_3d(sb + UM_B_BYTES / 2, &tmB, fb, n0 + 64, kb * UM_BK, g);
+                        // k-rows kb*64 .. +63 = half of row block kb/2; n-columns n0 .. n0+127 = column blocks n0/64, n0/64+1
+                        tma_load_5d(sb, &tmB, fb, 0, (kb & 1) * 64, n0 / 64, kb >> 1, g);
+                        tma_load_5d(sb + UM_B_BYTES / 2, &tmB, fb, 0, (kb & 1) * 64, n0 / 64 + 1, kb >> 1, g);
                     }
-                    if (++stage == UM_STAGES) { stage = 0; phase ^= 1u; }
+                    if (++stage == UM_B_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
             if (!ok) {
                 // gave up: let the copies already issued land before the CTA exits
                 // (slots below `stage` were armed in this pass of the ring, the others in the previous one)
-                for (int s = 0; s < UM_STAGES; ++s) {
+                for (int s = 0; s < UM_B_STAGES; ++s) {
                     const uint32_t armed_parity = (s < stage) ? phase : (phase ^ 1u);
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar_full + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
+                    while (!mbar_try_wait(bar_bfull + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 2 + umma_epi_warps(EPI)) {
+        // ------------------------------------------------ TMA producer of the A operand
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int g, m0, n0; tile_coords(p, t, g, m0, n0);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(bar_aempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = bar_afull + 8 * stage;
+                    mbar_expect_tx(fb, UM_A_BYTES);
+                    tma_load_3d(a_base + stage * UM_A_BYTES, &tmA, fb, kb * UM_BK, m0, g);
+                    if (++stage == UM_A_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                for (int s = 0; s < UM_A_STAGES; ++s) {
+                    const uint32_t armed_parity = (s < stage) ? phase : (phase ^ 1u);
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_afull + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
+            constexpr bool B_MN = (BKIND == UB_BLOCKED_MN);
             constexpr uint32_t idesc = make_idesc(false, B_MN);
-            int stage = 0; uint32_t phase = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
+            int sa_i = 0, sb_i = 0; uint32_t pa = 0, pb = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * UM_BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_afull + 8 * sa_i, pa, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_bfull + 8 * sb_i, pb, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = tiles_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
+                    const uint32_t sa = a_base + sa_i * UM_A_BYTES, sb = b_base + sb_i * UM_B_BYTES;
                     const uint64_t adesc = make_smem_desc(sa, 16, 1024);
                     const uint64_t bdesc = B_MN ? make_smem_desc(sb, UM_B_BYTES / 2, 1024)
                                                 : make_smem_desc(sb, 16, 1024);
@@ -251,28 +304,55 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const uint64_t b_k = bdesc + (uint64_t)(B_MN ? k * 128 : k * 2);
                         tc_mma_bf16(d_tmem, a_k, b_k, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    tc_commit(bar_empty + 8 * stage);        // frees the smem slot when these MMAs retire
-                    if (++stage == UM_STAGES) { stage = 0; phase ^= 1u; }
+                    tc_commit(bar_aempty + 8 * sa_i);        // both slots are free once these MMAs retire
+                    tc_commit(bar_bempty + 8 * sb_i);
+                    if (++sa_i == UM_A_STAGES) { sa_i = 0; pa ^= 1u; }
+                    if (++sb_i == UM_B_STAGES) { sb_i = 0; pb ^= 1u; }
                 }
                 if (!ok) break;
                 tc_commit(bar_tfull + 8 * acc);              // accumulator complete
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
-    } else {
-        // ------------------------------------------------ epilogue (warps 2..5)
+    } else if (warp < 2 + umma_epi_warps(EPI)) {
+        // ------------------------------------------------ epilogue (warps 2..9)
         const int q = warp & 3;                              // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                    // chunks 2*half, 2*half + 1 of every tile
         int acc = 0; uint32_t acc_phase = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             int g, m0, n0; tile_coords(p, t, g, m0, n0);
+            const int m = m0 + q * 32 + lane;                // output row of this thread
+            const bool m_ok = m < p.M;
+            // what the epilogue needs besides the accumulator is fetched before the accumulator is awaited
+            float bias_lane[2] = {0.f, 0.f};                 // bias[nb + lane] of this warp's two chunks
+            uint4 mk[2][4];                                  // ReLU mask source: 32 bf16 of row m per chunk
+            if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_FWD_LAST) {
+                const float *bias = p.bias + (long long)g * p.bias_gs;
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int col = n0 + (2 * half + cc) * 32 + lane;
+                    if (col < p.N) bias_lane[cc] = __ldg(bias + col);
+                }
+            }
+            if (EPI == UEPI_DGRAD) {
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int nb = n0 + (2 * half + cc) * 32;
+                    const __nv_bfloat16 *mkp = p.mask + (long long)g * p.mask_gs + (long long)m * p.mask_ld + nb;
+#pragma unroll
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        mk[cc][j8] = make_uint4(0u, 0u, 0u, 0u);
+                        if (m_ok && nb + j8 * 8 < p.N) mk[cc][j8] = *reinterpret_cast<const uint4 *>(mkp + j8 * 8);
+                    }
+                }
+            }
             const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            const int m = m0 + q * 32 + lane;                // output row of this thread
-            const bool m_ok = m < p.M;
             {
-#pragma unroll 1
-            for (int c = 0; c < UM_BN / 32; ++c) {
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+                const int c = 2 * half + cc;
                 const int nb = n0 + c * 32;
                 if (nb >= p.N) break;                        // warp-uniform
                 uint32_t r[32];
@@ -282,27 +362,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
                 if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_FWD_LAST) {
-                    const float *bias = p.bias + (long long)g * p.bias_gs;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const float b = (nb + j < p.N) ? __ldg(bias + nb + j) : 0.f;
-                        v[j] += b;
+                        v[j] += __shfl_sync(0xffffffffu, bias_lane[cc], j);
                         if (EPI == UEPI_FWD_HIDDEN) v[j] = fmaxf(v[j], 0.f);
                     }
                 }
                 if (EPI == UEPI_DGRAD) {
-                    if (m_ok) {
-                        const __nv_bfloat16 *mk = p.mask + (long long)g * p.mask_gs + (long long)m * p.mask_ld + nb;
 #pragma unroll
-                        for (int j8 = 0; j8 < 32; j8 += 8) {
-                            if (nb + j8 < p.N) {             // N % 8 == 0: whole group in range
-                                const uint4 raw4 = *reinterpret_cast<const uint4 *>(mk + j8);
-                                const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&raw4);
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&mk[cc][j8]);
 #pragma unroll
-                                for (int j = 0; j < 8; ++j)
-                                    if (!(__bfloat162float(h[j]) > 0.f)) v[j8 + j] = 0.f;
-                            }
-                        }
+                        for (int j = 0; j < 8; ++j)
+                            if (!(__bfloat162float(h[j]) > 0.f)) v[j8 * 8 + j] = 0.f;
                     }
                 }
                 if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_DGRAD) {

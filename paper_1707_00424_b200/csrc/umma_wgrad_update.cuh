@@ -64,7 +64,8 @@ struct WgradUpdateParams {
     int M, N, K;                 // M = d_in (tile rows), N = d_out (tile columns), K = batch
     int groups, tiles_m, tiles_n;
     float *y, *z;                // W_l segment of replica 0; element (replica g, W row r, W col c) at g*gs + r*ld + c
-    __nv_bfloat16 *shadow;
+    __nv_bfloat16 *shadow;       // blocked bf16 copy of W_l of replica 0 (128 x 64 blocks, row-block major)
+    long long shadow_gs; int shadow_cb;   // replica pitch (elements) and column blocks per row block
     long long gs; int ld;
     float eta_p, inv_gamma, alpha;
     int *status;
@@ -222,9 +223,12 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             const long long tile_e0 = (long long)g * p.gs + (long long)(n0 + grp * RPG) * p.ld + m;
             const long long chunk_step = (long long)WU_CHUNK_ROWS * p.ld;
             float *yp = p.y + tile_e0, *zp = p.z + tile_e0;
-            __nv_bfloat16 *sp = p.shadow + tile_e0;
+            // blocked copy: W row r, column m live in block (r/128, m/64) at (r%128)*64 + m%64; n0 % 128 == 0
+            __nv_bfloat16 *sp = p.shadow + (long long)g * p.shadow_gs +
+                                ((long long)(n0 / UM_BN) * p.shadow_cb + (m >> 6)) * (UM_BN * 64) +
+                                (grp * RPG) * 64 + (m & 63);
 #pragma unroll 1
-            for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += chunk_step) {
+            for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
                 const int nb0 = n0 + c * WU_CHUNK_ROWS;
                 if (nb0 >= p.N) break;                       // same rule as the loader
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
@@ -254,7 +258,7 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 __nv_bfloat16 *sr = sp;
                 if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += p.ld) {
+                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
                         const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
                         const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j])), yo);
                         const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
@@ -265,7 +269,7 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += p.ld) {
+                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
                         if (j < rows) {
                             const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
                             const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j])), yo);

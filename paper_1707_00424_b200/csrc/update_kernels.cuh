@@ -1,7 +1,6 @@
 // Streaming kernels of the Parle round: the fused inner update
 // (Eq. parle_y + Eq. parle_z), the fused outer update + replica mean
-// (Eq. parle_xa + Eq. parle_x with eta'' = rho/n), the stand-alone mean and the
-// bf16 shadow conversion.  All are HBM-bound: every vector is touched once,
+// (Eq. parle_xa + Eq. parle_x with eta'' = rho/n) and the stand-alone mean.  All are HBM-bound: every vector is touched once,
 // with 16-byte accesses, consecutive threads on consecutive addresses.
 #pragma once
 
@@ -17,23 +16,13 @@ __device__ __forceinline__ bool finite4(const float4 &v) {
            (fabsf(v.z) <= 3.402823466e+38f) & (fabsf(v.w) <= 3.402823466e+38f);
 }
 
-__device__ __forceinline__ uint2 pack_bf16x4(const float4 &v) {
-    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
-    uint2 r;
-    r.x = *reinterpret_cast<uint32_t *>(&lo);
-    r.y = *reinterpret_cast<uint32_t *>(&hi);
-    return r;
-}
-
 // Eq. (parle_y): y <- y - eta' (g + (y - x)/gamma), Eq. (parle_z): z <- alpha z + (1-alpha) y_new.
 // FIRST: first inner step of a round, where y = z = x (the reset is folded in:
 // x is read in place of y and z, which are only written).
-// SHADOW: also write y_new rounded to bf16 (the GEMM operand copy).
-template <bool FIRST, bool SHADOW, int UNROLL>
+template <bool FIRST, int UNROLL>
 __global__ void __launch_bounds__(kUpdThreads)
 inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const float4 *__restrict__ x,
-                    float4 *__restrict__ z, uint2 *__restrict__ shadow, size_t n4,
+                    float4 *__restrict__ z, size_t n4,
                     float eta_p, float inv_gamma, float alpha, int *status) {
     const size_t tid = (size_t)blockIdx.x * kUpdThreads + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
@@ -71,7 +60,6 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
                 ok &= finite4(yn);
                 y[i] = yn;
                 z[i] = zn;
-                if (SHADOW) shadow[i] = pack_bf16x4(yn);
             }
         }
     }
@@ -81,11 +69,10 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
 // Eq. (parle_xa) for all replicas of a coordinate, then Eq. (parle_x): each
 // thread owns four consecutive coordinates, walks the replica axis in a fixed
 // order (deterministic sum, no atomics) and writes the new mean.
-// SHADOW: also write bf16(x_new), the GEMM operand of the next round's first step.
-template <bool SHADOW, int RCHUNK>
+template <int RCHUNK>
 __global__ void __launch_bounds__(kUpdThreads)
 outer_mean_kernel(float4 *__restrict__ x, const float4 *__restrict__ z, float4 *__restrict__ xbar,
-                  uint2 *__restrict__ shadow, size_t stride4, int n, float eta, float eta_over_rho,
+                  size_t stride4, int n, float eta, float eta_over_rho,
                   float n_as_float, int *status) {
     const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
     bool ok = true;
@@ -113,7 +100,6 @@ outer_mean_kernel(float4 *__restrict__ x, const float4 *__restrict__ z, float4 *
                     xn.w = xv[r].w - eta * (xv[r].w - zv[r].w) - eta_over_rho * (xv[r].w - xb.w);
                     ok &= finite4(xn);
                     x[i] = xn;
-                    if (SHADOW) shadow[i] = pack_bf16x4(xn);
                     acc.x += xn.x; acc.y += xn.y; acc.z += xn.z; acc.w += xn.w;
                 }
             }
@@ -141,14 +127,6 @@ mean_kernel(const float4 *__restrict__ x, float4 *__restrict__ xbar, size_t stri
         }
         xbar[j] = make_float4(acc.x / n_as_float, acc.y / n_as_float, acc.z / n_as_float, acc.w / n_as_float);
     }
-}
-
-// bf16 copy of an fp32 vector (round to nearest even).
-__global__ void __launch_bounds__(kUpdThreads)
-to_bf16_kernel(const float4 *__restrict__ src, uint2 *__restrict__ dst, size_t n4) {
-    const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
-    for (size_t i = (size_t)blockIdx.x * kUpdThreads + threadIdx.x; i < n4; i += nthreads)
-        dst[i] = pack_bf16x4(src[i]);
 }
 
 }  // namespace parle
