@@ -152,27 +152,35 @@ bias_grad_f32_kernel(const float *__restrict__ dH, float *__restrict__ grad, lon
     grad[(long long)g * grad_gs + j] = s;
 }
 
-// db[g, j] = sum_i dH^T[g, j, i] from the bf16 transposed copy [n, d, B] (warp per row).
-__global__ void __launch_bounds__(256)
+// sum_i row[i] over one row of the bf16 transposed copy dH^T (batch % 8 == 0), fp32, in batch order.
+__device__ __forceinline__ float bias_grad_row(const __nv_bfloat16 *row, int batch) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(row);
+    float s = 0.f;
+    for (int i = 0; i < batch / 8; ++i) {
+        const uint4 v = __ldg(p + i);
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { const float2 f = __bfloat1622float2(h[k]); s += f.x; s += f.y; }
+    }
+    return s;
+}
+
+// db[g, j] = sum_i dH^T[g, j, i] from the bf16 transposed copy [n, d, B] (thread per row).
+__global__ void __launch_bounds__(128)
 bias_grad_bf16_kernel(const __nv_bfloat16 *__restrict__ dHT, float *__restrict__ grad,
                       long long grad_gs, int B, int d) {
-    const int j = blockIdx.x * 8 + threadIdx.x / 32;
-    const int lane = threadIdx.x % 32;
+    const int j = blockIdx.x * 128 + threadIdx.x;
     const int g = blockIdx.y;
     if (j >= d) return;
-    const __nv_bfloat16 *p = dHT + ((size_t)g * d + j) * B;
-    float s = 0.f;
-    for (int i = lane; i < B; i += 32) s += __bfloat162float(p[i]);
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) grad[(long long)g * grad_gs + j] = s;
+    grad[(long long)g * grad_gs + j] = bias_grad_row(dHT + ((size_t)g * d + j) * B, B);
 }
 
 // Everything of a replica's vector that the weight tiles do not cover -- the
 // bias segments and the alignment padding after each segment -- gets its inner
 // update (Eq. parle_y, parle_z) here when the update of the weights is fused into
-// the weight-gradient GEMM.  One warp per element: for a bias element the warp
-// first forms db_j = sum_i dH^T[j, i] (bf16 transposed copy, fp32 sum); padding
-// has gradient 0 and stays 0.
+// the weight-gradient GEMM.  One thread per element: for a bias element the thread
+// first forms db_j = sum_i dH^T[j, i] (bf16 transposed copy, fp32 sum in batch order);
+// padding has gradient 0 and stays 0.
 struct TailPlan {
     int n_layers, batch;
     long long begin[PARLE_MAX_LAYERS], b_off[PARLE_MAX_LAYERS], end[PARLE_MAX_LAYERS];   // element ranges in a replica
@@ -181,30 +189,25 @@ struct TailPlan {
 };
 
 template <bool FIRST>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__ z, const float *__restrict__ x,
                    long long stride, float eta_p, float inv_gamma, float alpha, int *status) {
     const int l = blockIdx.y, g = blockIdx.z;
-    const int lane = threadIdx.x % 32;
-    const long long e = tp.begin[l] + (long long)blockIdx.x * 8 + threadIdx.x / 32;
+    const long long e = tp.begin[l] + (long long)blockIdx.x * 128 + threadIdx.x;     // one thread per element
     if (e >= tp.end[l]) return;
     float grad = 0.f;
     const long long j = e - tp.b_off[l];
     if (j >= 0 && j < tp.d_out[l]) {
-        const __nv_bfloat16 *p = tp.dHT[l] + ((long long)g * tp.d_out[l] + j) * tp.batch;
-        for (int i = lane; i < tp.batch; i += 32) grad += __bfloat162float(p[i]);
-        for (int o = 16; o > 0; o >>= 1) grad += __shfl_xor_sync(0xffffffffu, grad, o);
+        grad = bias_grad_row(tp.dHT[l] + ((long long)g * tp.d_out[l] + j) * tp.batch, tp.batch);
     }
-    if (lane == 0) {
-        const long long i = (long long)g * stride + e;
-        const float xv = x[i];
-        const float yo = FIRST ? xv : y[i], zo = FIRST ? xv : z[i];
-        const float yn = yo - eta_p * fmaf(inv_gamma, yo - xv, grad);
-        const float zn = fmaf(alpha, zo, (1.0f - alpha) * yn);
-        y[i] = yn;
-        z[i] = zn;
-        if (!(fabsf(yn) <= 3.402823466e+38f)) status[SLOT_NONFINITE] = 1;
-    }
+    const long long i = (long long)g * stride + e;
+    const float xv = x[i];
+    const float yo = FIRST ? xv : y[i], zo = FIRST ? xv : z[i];
+    const float yn = yo - eta_p * fmaf(inv_gamma, yo - xv, grad);
+    const float zn = fmaf(alpha, zo, (1.0f - alpha) * yn);
+    y[i] = yn;
+    z[i] = zn;
+    if (!(fabsf(yn) <= 3.402823466e+38f)) status[SLOT_NONFINITE] = 1;
 }
 
 // bf16 operand copy of the weights in blocked layout: W_l [d_out, d_in] row-major fp32 ->
@@ -243,26 +246,40 @@ blocked_bf16_kernel(const BlockedPlan bp, const float *__restrict__ src, long lo
 
 // Minibatch inputs fp32 [n, B, d] -> bf16 [n, B, d] and its transpose [n, d, B]
 // (the K-major operand of the first layer's weight-gradient product).
+// 64 x 64 tiles; 16-byte reads, 8-byte row-major writes, 16-byte transposed writes (needs d % 8 == 0, B % 8 == 0).
 __global__ void __launch_bounds__(256)
 input_to_bf16_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ Xb,
                      __nv_bfloat16 *__restrict__ XbT, int B, int d) {
-    __shared__ float tile[32][33];
+    __shared__ __nv_bfloat16 tile[64][64 + 8];
     const int g = blockIdx.z;
-    const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
-    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;   // 32 x 8
-    for (int r = ty; r < 32; r += 8) {
-        const int i = i0 + r, j = j0 + tx;
-        float v = 0.f;
+    const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+    const int c4 = (threadIdx.x % 16) * 4, r0 = threadIdx.x / 16;          // 16 threads x 4 features per batch row
+#pragma unroll
+    for (int r = r0; r < 64; r += 16) {
+        const int i = i0 + r, j = j0 + c4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (i < B && j < d) {
-            v = X[((size_t)g * B + i) * d + j];
-            Xb[((size_t)g * B + i) * d + j] = __float2bfloat16_rn(v);
+            v = __ldcs(reinterpret_cast<const float4 *>(X + ((size_t)g * B + i) * d + j));
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t *>(&lo); pk.y = *reinterpret_cast<uint32_t *>(&hi);
+            *reinterpret_cast<uint2 *>(Xb + ((size_t)g * B + i) * d + j) = pk;
         }
-        tile[r][tx] = v;
+        tile[r][c4 + 0] = __float2bfloat16_rn(v.x); tile[r][c4 + 1] = __float2bfloat16_rn(v.y);
+        tile[r][c4 + 2] = __float2bfloat16_rn(v.z); tile[r][c4 + 3] = __float2bfloat16_rn(v.w);
     }
     __syncthreads();
-    for (int r = ty; r < 32; r += 8) {
-        const int j = j0 + r, i = i0 + tx;
-        if (i < B && j < d) XbT[((size_t)g * d + j) * B + i] = __float2bfloat16_rn(tile[tx][r]);
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        const int item = threadIdx.x + it * 256;          // 64 features x 8 groups of 8 batch rows
+        const int jj = item / 8, i8 = (item % 8) * 8;
+        const int j = j0 + jj, i = i0 + i8;
+        if (j < d && i < B) {
+            __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = tile[i8 + k][jj];
+            *reinterpret_cast<uint4 *>(XbT + ((size_t)g * d + j) * B + i) = *reinterpret_cast<const uint4 *>(o);
+        }
     }
 }
 

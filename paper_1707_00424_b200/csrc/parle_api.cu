@@ -383,7 +383,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     {
         const int d0 = c->dims[0];
         prof_begin(c, KC_INPUT_CVT);
-        input_to_bf16_kernel<<<dim3((d0 + 31) / 32, (B + 31) / 32, n), 256, 0, c->stream>>>(
+        input_to_bf16_kernel<<<dim3((d0 + 63) / 64, (B + 63) / 64, n), 256, 0, c->stream>>>(
             inputs, ws_ptr<__nv_bfloat16>(c, w.xb), ws_ptr<__nv_bfloat16>(c, w.xbT), B, d0);
         PARLE_LAUNCHED(c);
     }
@@ -430,7 +430,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
             p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
             PARLE_TRY((launch_umma<UEPI_WGRAD, UB_ROWMAJOR_K>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
             prof_begin(c, KC_BIAS_GRAD);
-            bias_grad_bf16_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
+            bias_grad_bf16_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(
                 ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
             PARLE_LAUNCHED(c);
             if (l > 0) PARLE_TRY(dgrad(l));
@@ -474,13 +474,13 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         tp.dHT[l] = ws_ptr<__nv_bfloat16>(c, w.dhbT[l]);
         if (tp.end[l] - tp.begin[l] > longest) longest = tp.end[l] - tp.begin[l];
     }
-    const dim3 tgrid((unsigned)((longest + 7) / 8), nl, n);
+    const dim3 tgrid((unsigned)((longest + 127) / 128), nl, n);
     prof_begin(c, KC_TAIL_UPDATE);
     if (c->fresh)
-        tail_update_kernel<true><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
+        tail_update_kernel<true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
                                                                c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
     else
-        tail_update_kernel<false><<<tgrid, 256, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
+        tail_update_kernel<false><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
                                                                 c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
