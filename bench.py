@@ -112,9 +112,10 @@ def dense_to_padded(model, cfg, replica_layers):
     return out
 
 
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture
-# (profiles/ncu_full_inner_update_and_gemms_C3.md), valid only while the kernel source is unchanged.
-NCU_TRAFFIC = {}
+# DRAM bytes per launch (mean over the four launches of an inner step) of the dominant kernel from the committed
+# ncu capture (profiles/ncu_full_gemms_and_fused_update_C3.md), valid only while the kernel source is unchanged.
+NCU_TRAFFIC = {("C3", "wgrad_gemm_fused_update"): {"bytes": 2481.4e6 / 4, "source_sha256_16": "3cb53c5f13b19919",
+                                                   "source": "paper_1707_00424_b200/csrc/umma_wgrad_update.cuh"}}
 
 
 def ncu_traffic(workload: str, kernel: str):
@@ -139,13 +140,14 @@ def algorithmic_bytes_per_round(cfg, stride):
     out = {}
     # separate update: read g, y, x, z, write y, z (+2 B bf16 copy); first step of a round reads x for y and z
     out["inner_update"] = n * stride * ((24 + (2 if bf else 0)) * L - 8)
-    out["outer_mean"] = stride * ((12 + (2 if bf else 0)) * n + 8)
+    out["outer_mean"] = stride * (12 * n + 8)
     if bf:
         opnd = sum(2 * (act(l) + act(l + 1)) for l in range(nl))             # dH^T and H^T, bf16
         # fused: read y, x, z (12 B), write y, z, bf16 copy (10 B); first step reads only x
         out["wgrad_gemm_fused_update"] = n * (Pw * (22 * (L - 1) + 14) + opnd * L)
         out["wgrad_gemm"] = n * L * (4 * Pw + opnd)
         out["fwd_gemm"] = n * L * (2 * Pw + sum(2 * act(l) + 4 * act(l + 1) for l in range(nl)))
+        out["to_bf16"] = n * Pw * 6                                          # blocked bf16 weight copy from x, once per round
         out["dgrad_gemm"] = n * L * sum(2 * dims[l] * dims[l + 1] + 2 * act(l + 1) + 6 * act(l) for l in range(1, nl))
     return out
 
