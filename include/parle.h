@@ -172,6 +172,18 @@ int parle_set_fused_update(parle_ctx *ctx, int on);
 int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);
 int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
 
+/* Scoping (Eq. scoping, Section 3.1): gamma and rho of round number `round` = floor(k / L),
+ *   gamma = gamma0 (1 - 1/(2B))^round,  rho = rho0 (1 - 1/(2B))^round,   B = minibatches in the dataset,
+ * clipped from below at gamma_floor and rho_floor (the paper: gamma0 = 100, rho0 = 1, floors 1 and 0.1).
+ * Pure host arithmetic; feed the result to parle_set_coupling before the round.  gamma, rho: host pointers. */
+int parle_scoping(double gamma0, double rho0, long long minibatches_per_epoch, long long round,
+                  double gamma_floor, double rho_floor, double *gamma, double *rho);
+
+/* Weight-decay regulariser of f (Section 1.1: "along with a regularization term (say weight decay)"):
+ * parle_inner_step uses grad f(y) + lambda * y in Eq. (parle_y), for every parameter.  Default 0.
+ * loss_out stays the data term alone.  parle_inner_update applies its gradient argument as given. */
+int parle_set_weight_decay(parle_ctx *ctx, double lambda);
+
 /* Non-blocking read of the device status word (PARLE_FLAG_* bits) set by the
  * kernels launched so far; clears nothing.  parle_clear_status resets it. */
 int parle_status(parle_ctx *ctx, int *device_flags);

@@ -19,6 +19,7 @@ What each function follows:
 * ``outer_step``  -- Eq. (parle_xa).
 * ``replica_mean`` -- Eq. (parle_x) with eta'' = rho/n (Section 3.1), which
   turns the reference update into the plain replica mean.
+* ``scoping`` -- Eq. (scoping), the schedule of gamma and rho (Section 3.1).
 * ``parle_round`` -- the loop of Section 3: reset y^a (and z^a) to x^a, L
   inner steps, the outer step, the mean.
 
@@ -207,6 +208,17 @@ def replica_mean(xs):
     for a in range(xs.shape[0]):
         acc = acc + xs[a]
     return acc / xs.shape[0]
+
+
+def scoping(gamma0: float, rho0: float, batches: int, k: int, L: int,
+            gamma_floor: float = 1.0, rho_floor: float = 0.1):
+    """Eq. (scoping), Section 3.1: gamma_k = gamma_0 (1 - 1/(2B))^floor(k/L), rho_k likewise, B = number
+    of minibatches in the dataset; gamma clipped at gamma_floor (paper: 1), rho at rho_floor (paper: 0.1)."""
+    rounds_done = k // L
+    factor = 1.0
+    for _ in range(rounds_done):                  # the power written out as repeated multiplication
+        factor *= 1.0 - 1.0 / (2.0 * batches)
+    return max(gamma0 * factor, gamma_floor), max(rho0 * factor, rho_floor)
 
 
 GradFn = Callable[[int, int, np.ndarray], Tuple[float, np.ndarray]]

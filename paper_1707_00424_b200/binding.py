@@ -69,6 +69,8 @@ def lib() -> C.CDLL:
         "parle_set_coupling": (ci, [vp, cd, cd]),
         "parle_set_lr": (ci, [vp, cd, cd]),
         "parle_set_fused_update": (ci, [vp, ci]),
+        "parle_set_weight_decay": (ci, [vp, cd]),
+        "parle_scoping": (ci, [cd, cd, C.c_longlong, C.c_longlong, cd, cd, C.POINTER(cd), C.POINTER(cd)]),
         "parle_status": (ci, [vp, C.POINTER(ci)]),
         "parle_clear_status": (ci, [vp]),
         "parle_profile_enable": (ci, [vp, ci]),
@@ -111,6 +113,17 @@ def softmax_ce_static(logits, labels, n: int, B: int, C_: int, dlogits, loss, fl
                                            _ptr(flags), C.c_void_p(stream.cuda_stream))
     if rc != 0:
         raise ParleError(rc, "parle_softmax_ce_static")
+
+
+def scoping(gamma0: float, rho0: float, minibatches_per_epoch: int, round_index: int,
+            gamma_floor: float = 1.0, rho_floor: float = 0.1):
+    """(gamma, rho) of a round by Eq. (scoping) (parle_scoping)."""
+    g, r = C.c_double(), C.c_double()
+    rc = lib().parle_scoping(gamma0, rho0, minibatches_per_epoch, round_index, gamma_floor, rho_floor,
+                             C.byref(g), C.byref(r))
+    if rc != 0:
+        raise ParleError(rc, "parle_scoping")
+    return g.value, r.value
 
 
 class Parle:
@@ -216,6 +229,9 @@ class Parle:
 
     def set_lr(self, eta: float, eta_prime: float):
         self._check(self._L.parle_set_lr(self._h, eta, eta_prime), "parle_set_lr")
+
+    def set_weight_decay(self, lam: float):
+        self._check(self._L.parle_set_weight_decay(self._h, lam), "parle_set_weight_decay")
 
     def set_fused_update(self, on: bool):
         self._check(self._L.parle_set_fused_update(self._h, 1 if on else 0), "parle_set_fused_update")

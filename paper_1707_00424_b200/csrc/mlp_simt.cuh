@@ -191,7 +191,7 @@ struct TailPlan {
 template <bool FIRST>
 __global__ void __launch_bounds__(128)
 tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__ z, const float *__restrict__ x,
-                   long long stride, float eta_p, float inv_gamma, float alpha, int *status) {
+                   long long stride, float eta_p, float inv_gamma, float alpha, float wd, int *status) {
     const int l = blockIdx.y, g = blockIdx.z;
     const long long e = tp.begin[l] + (long long)blockIdx.x * 128 + threadIdx.x;     // one thread per element
     if (e >= tp.end[l]) return;
@@ -203,7 +203,7 @@ tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__
     const long long i = (long long)g * stride + e;
     const float xv = x[i];
     const float yo = FIRST ? xv : y[i], zo = FIRST ? xv : z[i];
-    const float yn = yo - eta_p * fmaf(inv_gamma, yo - xv, grad);
+    const float yn = yo - eta_p * fmaf(inv_gamma, yo - xv, fmaf(wd, yo, grad));
     const float zn = fmaf(alpha, zo, (1.0f - alpha) * yn);
     y[i] = yn;
     z[i] = zn;

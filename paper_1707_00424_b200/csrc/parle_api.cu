@@ -45,7 +45,7 @@ struct Workspace {
 struct parle_ctx {
     int n, n_layers, batch, gemm_dtype;
     int dims[PARLE_MAX_LAYERS + 1];
-    float inv_gamma, inv_rho, alpha, eta, eta_prime;
+    float inv_gamma, inv_rho, alpha, eta, eta_prime, weight_decay;
     size_t P, stride;
     size_t sh_stride;                // bf16 path: elements of one replica's blocked weight copy
     size_t sh_off[PARLE_MAX_LAYERS]; int sh_cb[PARLE_MAX_LAYERS], sh_rb[PARLE_MAX_LAYERS];   // per layer: offset, column / row blocks
@@ -302,7 +302,7 @@ int run_blocked_copy(parle_ctx *c, const float *src) {
     return PARLE_OK;
 }
 
-int run_inner_update(parle_ctx *c, const float *grad) {
+int run_inner_update(parle_ctx *c, const float *grad, float wd) {
     const size_t n4 = (size_t)c->n * c->stride / 4;
     constexpr int U = 2;
     const int grid = stream_grid(c, n4, U);
@@ -311,9 +311,9 @@ int run_inner_update(parle_ctx *c, const float *grad) {
     const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
     prof_begin(c, KC_INNER_UPDATE);
     if (c->fresh)
-        inner_update_kernel<true, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+        inner_update_kernel<true, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev);
     else
-        inner_update_kernel<false, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+        inner_update_kernel<false, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev);
     PARLE_LAUNCHED(c);
     c->fresh = false;
     c->shadow_is_x = false;
@@ -450,7 +450,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         p.y = c->buf.y + wo; p.z = c->buf.z + wo;
         p.shadow = shadow + c->sh_off[l]; p.shadow_gs = (long long)c->sh_stride; p.shadow_cb = c->sh_cb[l];
         p.gs = S; p.ld = din;
-        p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha;
+        p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha; p.wd = c->weight_decay;
         p.status = c->status_dev;
         const int tiles = p.groups * p.tiles_m * p.tiles_n;
         const int grid = tiles < c->sm_count ? tiles : c->sm_count;
@@ -478,10 +478,10 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     prof_begin(c, KC_TAIL_UPDATE);
     if (c->fresh)
         tail_update_kernel<true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
-                                                               c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+                                                               c->eta_prime, c->inv_gamma, c->alpha, c->weight_decay, c->status_dev);
     else
         tail_update_kernel<false><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
-                                                                c->eta_prime, c->inv_gamma, c->alpha, c->status_dev);
+                                                                c->eta_prime, c->inv_gamma, c->alpha, c->weight_decay, c->status_dev);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
@@ -637,7 +637,7 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
     } else {
         PARLE_TRY(forward_backward_fp32(c, inputs, labels, loss_out));
     }
-    return run_inner_update(c, c->buf.grad);
+    return run_inner_update(c, c->buf.grad, c->weight_decay);
 }
 
 int parle_inner_step_host(parle_ctx *c, const float *inputs_host, const int32_t *labels_host, float *loss_out_host) {
@@ -663,7 +663,7 @@ int parle_inner_update(parle_ctx *c, const float *grad) {
     if (!grad) return PARLE_EINVAL;
     if (reinterpret_cast<uintptr_t>(grad) % 16) return PARLE_EALIGN;
     if (!c->round_open) return PARLE_ESTATE;
-    return run_inner_update(c, grad);
+    return run_inner_update(c, grad, 0.f);
 }
 
 int parle_outer_step(parle_ctx *c) {
@@ -756,6 +756,24 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->fused_update = on != 0;
+    return PARLE_OK;
+}
+
+int parle_scoping(double gamma0, double rho0, long long minibatches_per_epoch, long long round,
+                  double gamma_floor, double rho_floor, double *gamma, double *rho) {
+    if (!gamma || !rho || !(gamma0 > 0.0) || !(rho0 > 0.0) || minibatches_per_epoch < 1 || round < 0 ||
+        !(gamma_floor > 0.0) || !(rho_floor > 0.0))
+        return PARLE_EINVAL;
+    const double f = pow(1.0 - 1.0 / (2.0 * (double)minibatches_per_epoch), (double)round);
+    const double g = gamma0 * f, r = rho0 * f;
+    *gamma = g < gamma_floor ? gamma_floor : g;
+    *rho = r < rho_floor ? rho_floor : r;
+    return PARLE_OK;
+}
+
+int parle_set_weight_decay(parle_ctx *c, double lambda) {
+    if (!c || !(lambda >= 0.0) || isinf(lambda)) return PARLE_EINVAL;
+    c->weight_decay = (float)lambda;
     return PARLE_OK;
 }
 

@@ -67,7 +67,7 @@ struct WgradUpdateParams {
     __nv_bfloat16 *shadow;       // blocked bf16 copy of W_l of replica 0 (128 x 64 blocks, row-block major)
     long long shadow_gs; int shadow_cb;   // replica pitch (elements) and column blocks per row block
     long long gs; int ld;
-    float eta_p, inv_gamma, alpha;
+    float eta_p, inv_gamma, alpha, wd;
     int *status;
 };
 
@@ -260,7 +260,7 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #pragma unroll
                     for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
                         const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
-                        const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j])), yo);
+                        const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j]))), yo);
                         const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
                         chk = fmaf(yn, 0.f, chk);
                         *yr = yn;
@@ -272,7 +272,7 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
                         if (j < rows) {
                             const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
-                            const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], __uint_as_float(r[j])), yo);
+                            const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j]))), yo);
                             const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
                             chk = fmaf(yn, 0.f, chk);
                             *yr = yn;

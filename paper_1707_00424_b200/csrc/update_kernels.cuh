@@ -17,13 +17,14 @@ __device__ __forceinline__ bool finite4(const float4 &v) {
 }
 
 // Eq. (parle_y): y <- y - eta' (g + (y - x)/gamma), Eq. (parle_z): z <- alpha z + (1-alpha) y_new.
+// wd: optional weight-decay regulariser of f (Section 1.1), g <- g + wd * y.
 // FIRST: first inner step of a round, where y = z = x (the reset is folded in:
 // x is read in place of y and z, which are only written).
 template <bool FIRST, int UNROLL>
 __global__ void __launch_bounds__(kUpdThreads)
 inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const float4 *__restrict__ x,
                     float4 *__restrict__ z, size_t n4,
-                    float eta_p, float inv_gamma, float alpha, int *status) {
+                    float eta_p, float inv_gamma, float alpha, float wd, int *status) {
     const size_t tid = (size_t)blockIdx.x * kUpdThreads + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
     const float one_m_alpha = 1.0f - alpha;
@@ -49,10 +50,10 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
                 float4 yo = FIRST ? xv[u] : yv[u];
                 float4 zo = FIRST ? xv[u] : zv[u];
                 float4 yn, zn;
-                yn.x = yo.x - eta_p * fmaf(inv_gamma, yo.x - xv[u].x, gv[u].x);
-                yn.y = yo.y - eta_p * fmaf(inv_gamma, yo.y - xv[u].y, gv[u].y);
-                yn.z = yo.z - eta_p * fmaf(inv_gamma, yo.z - xv[u].z, gv[u].z);
-                yn.w = yo.w - eta_p * fmaf(inv_gamma, yo.w - xv[u].w, gv[u].w);
+                yn.x = yo.x - eta_p * fmaf(inv_gamma, yo.x - xv[u].x, fmaf(wd, yo.x, gv[u].x));
+                yn.y = yo.y - eta_p * fmaf(inv_gamma, yo.y - xv[u].y, fmaf(wd, yo.y, gv[u].y));
+                yn.z = yo.z - eta_p * fmaf(inv_gamma, yo.z - xv[u].z, fmaf(wd, yo.z, gv[u].z));
+                yn.w = yo.w - eta_p * fmaf(inv_gamma, yo.w - xv[u].w, fmaf(wd, yo.w, gv[u].w));
                 zn.x = fmaf(alpha, zo.x, one_m_alpha * yn.x);
                 zn.y = fmaf(alpha, zo.y, one_m_alpha * yn.y);
                 zn.z = fmaf(alpha, zo.z, one_m_alpha * yn.z);

@@ -51,6 +51,8 @@ TAG_TEACHER = 3
 TAG_GRAD = 4
 TAG_STATE = 5
 TAG_QUAD = 6
+TAG_DATASET = 7
+TAG_INDEX = 8
 
 
 def stream_key(seed: int, *words: int) -> int:
@@ -249,3 +251,45 @@ def quadratic_spectrum(seed: int, d: int, lo: float = 0.05, hi: float = 2.0) -> 
     """Eigenvalues of a diagonal positive quadratic loss, uniform on [lo, hi]."""
     u = uniform01(stream_key(seed, TAG_QUAD), d)
     return lo + (hi - lo) * u
+
+
+# --------------------------------------------------------------------------
+# A finite synthetic dataset and its split between replicas (Section 5 of the paper:
+# the dataset xi is the union of shards xi^a and replica a samples minibatches from xi^a only)
+# --------------------------------------------------------------------------
+
+def dataset_sample(cfg: ParleConfig, index: int) -> np.ndarray:
+    """Sample `index` of the dataset: d_0 values drawn from the config's input distribution."""
+    key = stream_key(cfg.seed, TAG_DATASET, index)
+    d = cfg.dims[0]
+    return uniform_f32(key, (d,)) if cfg.input_dist == "uniform" else normal_f32(key, (d,))
+
+
+def shard_bounds(dataset_size: int, n: int, replica: int) -> Tuple[int, int]:
+    """Half-open index range of shard `replica` when the dataset is cut into n contiguous shards."""
+    return replica * dataset_size // n, (replica + 1) * dataset_size // n
+
+
+def dataset_minibatch_indices(cfg: ParleConfig, replica: int, rnd: int, step: int,
+                              dataset_size: int, split: bool) -> np.ndarray:
+    """Indices (with replacement) of the minibatch of `replica` at (rnd, step): from its own shard when
+    `split`, from the whole dataset otherwise."""
+    lo, hi = shard_bounds(dataset_size, cfg.n, replica) if split else (0, dataset_size)
+    u = uniform01(stream_key(cfg.seed, TAG_INDEX, replica, rnd, step), cfg.batch)
+    return lo + np.minimum((u * (hi - lo)).astype(np.int64), hi - lo - 1)
+
+
+def dataset_round_batches(cfg: ParleConfig, rnd: int, dataset_size: int, split: bool):
+    """X [L, n, batch, d_0], labels [L, n, batch] and the sample indices [L, n, batch] of one round."""
+    X = np.empty((cfg.L, cfg.n, cfg.batch, cfg.dims[0]), dtype=np.float32)
+    idx = np.empty((cfg.L, cfg.n, cfg.batch), dtype=np.int64)
+    cache = {}
+    for l in range(cfg.L):
+        for a in range(cfg.n):
+            idx[l, a] = dataset_minibatch_indices(cfg, a, rnd, l, dataset_size, split)
+            for i, k in enumerate(idx[l, a]):
+                if k not in cache:
+                    cache[k] = dataset_sample(cfg, int(k))
+                X[l, a, i] = cache[k]
+    c = teacher_labels(cfg, X.reshape(-1, cfg.dims[0])).reshape(cfg.L, cfg.n, cfg.batch)
+    return X, c, idx

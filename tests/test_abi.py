@@ -82,3 +82,18 @@ def test_calls_before_bind_fail_cleanly():
     assert L.parle_strerror(-5) == b"call out of order"
     assert L.parle_param_count(None) == 0
     assert L.parle_round_begin(None) == -1
+
+
+def test_scoping_schedule_host_function():
+    # Eq. (scoping) with the paper's constants; values worked out by hand
+    assert pb.scoping(100.0, 1.0, 50, 0) == (100.0, 1.0)
+    g, r = pb.scoping(100.0, 1.0, 50, 7)
+    assert abs(g - 100 * 0.99 ** 7) < 1e-10 and abs(r - 0.99 ** 7) < 1e-12
+    assert pb.scoping(100.0, 1.0, 50, 459) == (1.0, 0.1)
+    assert pb.scoping(100.0, 1.0, 50, 458)[0] > 1.0 and pb.scoping(100.0, 1.0, 50, 230)[1] == 0.1
+    with pytest.raises(pb.ParleError):
+        pb.scoping(100.0, 1.0, 0, 1)
+    m = pb.Parle(2, (8, 4), 4)
+    m.set_weight_decay(1e-3)
+    with pytest.raises(pb.ParleError):
+        m.set_weight_decay(-1.0)

@@ -407,3 +407,46 @@ def test_c5_full_shape_sampled_outputs_bf16():
         torch.cuda.empty_cache()
     for a, b in zip(*states):
         assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ scoping schedule and weight decay
+@pytest.mark.parametrize("gemm_dtype,dims", [(0, (64, 32, 10)), (1, (64, 128, 72, 10))])
+def test_scoped_rounds_with_weight_decay_match_oracle(gemm_dtype, dims):
+    """gamma and rho follow Eq. (scoping) from round to round (so gamma != rho != 1: the coefficient of
+    (x - z) in Eq. (parle_xa) is eta, not eta/gamma) and f carries a weight-decay term."""
+    cfg = si.C1.scaled(dims=dims, gemm_dtype=gemm_dtype, L=4)
+    wd, batches = 5e-3, 2
+    m, xo, xb, _ = make(cfg)
+    m.set_weight_decay(wd)
+    tol = TOL[gemm_dtype]
+    for r in range(3):
+        g_lib, r_lib = pb.scoping(100.0, 1.0, batches, r)
+        g_or, r_or = po.scoping(100.0, 1.0, batches, r * cfg.L, cfg.L)
+        assert abs(g_lib - g_or) < 1e-12 and abs(r_lib - r_or) < 1e-12 and g_lib != r_lib
+        m.set_coupling(g_lib, r_lib)
+        X, c = si.round_batches(cfg, r)
+        m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
+        hp = po.Hyper(cfg.eta, cfg.eta_prime, cfg.alpha, g_or, r_or)
+        out = po.parle_round(xo, xb, po.mlp_grad_fn(cfg.dims, X, c, weight_decay=wd), cfg.L, hp)
+        x_gpu = to_dense(m, m.x.cpu().numpy())
+        for a in range(cfg.n):
+            assert rel_l2(x_gpu[a], out["x"][a]) <= tol
+        assert rel_l2(x_gpu - xo, out["x"] - xo) <= (1e-4 if gemm_dtype == 0 else 5e-2)
+        assert rel_l2(to_dense(m, m.xbar.cpu().numpy()), out["xbar"]) <= tol
+        xo, xb = out["x"], out["xbar"]
+    assert m.status() == 0
+
+
+def test_split_data_round_matches_oracle():
+    """Section 5: every replica draws its minibatches from its own shard of a finite dataset.  Only the
+    inputs change; the round itself is the same computation."""
+    cfg = si.C1.scaled(L=4)
+    m, xo, xb, hp = make(cfg)
+    X, c, idx = si.dataset_round_batches(cfg, 0, 96, split=True)
+    for a in range(cfg.n):
+        lo, hi = si.shard_bounds(96, cfg.n, a)
+        assert idx[:, a].min() >= lo and idx[:, a].max() < hi
+    m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
+    out = po.parle_round(xo, xb, po.mlp_grad_fn(cfg.dims, X, c), cfg.L, hp)
+    x_gpu = to_dense(m, m.x.cpu().numpy())
+    assert rel_l2(x_gpu, out["x"]) <= 1e-4 and rel_l2(x_gpu - xo, out["x"] - xo) <= 1e-4

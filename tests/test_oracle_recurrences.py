@@ -218,3 +218,20 @@ def test_planted_mistakes_break_the_closed_form(monkeypatch, mutant):
         monkeypatch.setattr(po, "outer_step", lambda x, z, xb, h, u=False: x - h.eta * (x - z) - h.eta * h.inv_gamma * (x - xb))
     with pytest.raises(AssertionError):
         test_quadratic_closed_form_one_round(c)
+
+
+def test_scoping_schedule_closed_form_and_clipping():
+    # Section 3.1: gamma_0 = 100, rho_0 = 1, clipped at 1 and 0.1
+    B, L = 50, 25
+    g, r = po.scoping(100.0, 1.0, B, 0, L)
+    assert (g, r) == (100.0, 1.0)
+    assert po.scoping(100.0, 1.0, B, L - 1, L) == (100.0, 1.0)          # constant inside a round
+    g, r = po.scoping(100.0, 1.0, B, 7 * L + 3, L)
+    assert abs(g - 100 * 0.99 ** 7) < 1e-12 and abs(r - 0.99 ** 7) < 1e-14
+    # gamma hits its floor after ln(100)/-ln(0.99) = 458.2 rounds, rho after ln(10)/-ln(0.99) = 229.1
+    assert po.scoping(100.0, 1.0, B, 458 * L, L)[0] > 1.0 and po.scoping(100.0, 1.0, B, 459 * L, L)[0] == 1.0
+    assert po.scoping(100.0, 1.0, B, 229 * L, L)[1] > 0.1 and po.scoping(100.0, 1.0, B, 230 * L, L)[1] == 0.1
+    seq = [po.scoping(100.0, 1.0, B, k * L, L) for k in range(600)]
+    assert all(a[0] >= b[0] and a[1] >= b[1] for a, b in zip(seq, seq[1:]))
+    # exact rational check of one value
+    assert abs(po.scoping(3.0, 2.0, 2, 3, 1)[0] - float(Fr(3) * Fr(3, 4) ** 3)) < 1e-15

@@ -41,3 +41,21 @@ def test_mnist_shaped_teacher_uses_all_classes():
     X, c = si.round_batches(cfg, 0)
     assert X.min() >= 0 and X.max() <= 1
     assert len(np.unique(c)) >= 5
+
+
+def test_split_dataset_gives_each_replica_its_own_shard():
+    cfg = si.C1.scaled(n=3, L=4)
+    D = 90
+    X, c, idx = si.dataset_round_batches(cfg, 0, D, split=True)
+    for a in range(cfg.n):
+        lo, hi = si.shard_bounds(D, cfg.n, a)
+        assert (lo, hi) == (30 * a, 30 * a + 30)
+        assert idx[:, a].min() >= lo and idx[:, a].max() < hi
+    Xf, cf, idxf = si.dataset_round_batches(cfg, 0, D, split=False)
+    assert idxf[:, 0].max() >= 30 and idxf.min() >= 0 and idxf.max() < D      # full data: replica 0 leaves shard 0
+    # a sample is the same whoever draws it, and so is its label
+    k = int(idx[0, 1, 0])
+    assert np.array_equal(X[0, 1, 0], si.dataset_sample(cfg, k))
+    where = np.argwhere(idxf == k)
+    for l, a, i in where[:3]:
+        assert np.array_equal(Xf[l, a, i], X[0, 1, 0]) and cf[l, a, i] == c[0, 1, 0]
