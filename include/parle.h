@@ -172,6 +172,19 @@ int parle_set_fused_update(parle_ctx *ctx, int on);
 int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);
 int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
 
+/* Nesterov momentum on the y^a and x^a steps (Remark in Section 3.1; none on xbar).  The paper does not
+ * print the form; the one taken is that of SGD with Nesterov momentum: for a step with direction d and
+ * step size s,  v <- mu v + d,  p <- p - s (d + mu v), with
+ *   y^a: d = grad f(y) + (y - x^a)/gamma, s = eta', v = vy, which restarts from 0 in every round with y;
+ *   x^a: d = (x^a - z^a) + (x^a - xbar)/rho, s = eta, v = vx, which carries over between rounds.
+ * parle_bind_momentum attaches the two caller-owned buffers, dev [n, stride] fp32, 128-byte aligned;
+ * vx must be zero before the first round (vy needs no initialisation).  parle_set_momentum(mu), mu in
+ * [0, 1): 0 switches momentum off; ENOTBOUND if mu > 0 without buffers, ESTATE in the middle of a round.
+ * With momentum on, the bf16 path writes the gradient to `grad` and runs the separate update kernel
+ * (the fused weight-gradient epilogue has no momentum variant). */
+int parle_bind_momentum(parle_ctx *ctx, float *vy, float *vx);
+int parle_set_momentum(parle_ctx *ctx, double mu);
+
 /* Scoping (Eq. scoping, Section 3.1): gamma and rho of round number `round` = floor(k / L),
  *   gamma = gamma0 (1 - 1/(2B))^round,  rho = rho0 (1 - 1/(2B))^round,   B = minibatches in the dataset,
  * clipped from below at gamma_floor and rho_floor (the paper: gamma0 = 100, rho0 = 1, floors 1 and 0.1).

@@ -19,6 +19,8 @@ What each function follows:
 * ``outer_step``  -- Eq. (parle_xa).
 * ``replica_mean`` -- Eq. (parle_x) with eta'' = rho/n (Section 3.1), which
   turns the reference update into the plain replica mean.
+* ``inner_step_momentum`` / ``outer_step_momentum`` / ``parle_round_momentum`` -- the same
+  recurrences with Nesterov momentum (Remark, Section 3.1).
 * ``scoping`` -- Eq. (scoping), the schedule of gamma and rho (Section 3.1).
 * ``parle_round`` -- the loop of Section 3: reset y^a (and z^a) to x^a, L
   inner steps, the outer step, the mean.
@@ -208,6 +210,43 @@ def replica_mean(xs):
     for a in range(xs.shape[0]):
         acc = acc + xs[a]
     return acc / xs.shape[0]
+
+
+def inner_step_momentum(y, z, v, x, g, hp: Hyper, mu: float):
+    """Eq. (parle_y) with Nesterov momentum mu (Remark in Section 3.1; the paper does not print the form,
+    the reading taken is the usual one of SGD with Nesterov momentum): with the descent direction
+    d = g + (y - x)/gamma,   v <- mu v + d,   y <- y - eta' (d + mu v);   then Eq. (parle_z)."""
+    d = g + hp.inv_gamma * (y - x)
+    v_new = mu * v + d
+    y_new = y - hp.eta_prime * (d + mu * v_new)
+    z_new = hp.alpha * z + (1.0 - hp.alpha) * y_new
+    return y_new, z_new, v_new
+
+
+def outer_step_momentum(x, z, xbar, vx, hp: Hyper, mu: float):
+    """Eq. (parle_xa) with Nesterov momentum: d = (x - z) + (x - xbar)/rho, vx <- mu vx + d,
+    x <- x - eta (d + mu vx)."""
+    d = (x - z) + hp.inv_rho * (x - xbar)
+    vx_new = mu * vx + d
+    return x - hp.eta * (d + mu * vx_new), vx_new
+
+
+def parle_round_momentum(x, xbar, vx, grad_fn, L: int, hp: Hyper, mu: float):
+    """One round with Nesterov momentum on the y and x^a updates (none on xbar, as in the paper's Remark).
+    The y-momentum starts from zero in every round (it belongs to the trajectory that is reset); the
+    x^a-momentum vx [n, P] carries over between rounds."""
+    x = np.array(x, F64); xbar = np.array(xbar, F64); vx = np.array(vx, F64)
+    n = x.shape[0]
+    y, z, v = x.copy(), x.copy(), np.zeros_like(x)
+    losses = np.zeros((L, n), F64)
+    for l in range(L):
+        for a in range(n):
+            losses[l, a], g = grad_fn(a, l, y[a])
+            y[a], z[a], v[a] = inner_step_momentum(y[a], z[a], v[a], x[a], g, hp, mu)
+    x_new, vx_new = np.empty_like(x), np.empty_like(vx)
+    for a in range(n):
+        x_new[a], vx_new[a] = outer_step_momentum(x[a], z[a], xbar, vx[a], hp, mu)
+    return {"x": x_new, "xbar": replica_mean(x_new), "vx": vx_new, "y": y, "z": z, "loss": losses}
 
 
 def scoping(gamma0: float, rho0: float, batches: int, k: int, L: int,

@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
         "parle_set_lr": (ci, [vp, cd, cd]),
         "parle_set_fused_update": (ci, [vp, ci]),
         "parle_set_weight_decay": (ci, [vp, cd]),
+        "parle_bind_momentum": (ci, [vp, vp, vp]),
+        "parle_set_momentum": (ci, [vp, cd]),
         "parle_scoping": (ci, [cd, cd, C.c_longlong, C.c_longlong, cd, cd, C.POINTER(cd), C.POINTER(cd)]),
         "parle_status": (ci, [vp, C.POINTER(ci)]),
         "parle_clear_status": (ci, [vp]),
@@ -229,6 +231,15 @@ class Parle:
 
     def set_lr(self, eta: float, eta_prime: float):
         self._check(self._L.parle_set_lr(self._h, eta, eta_prime), "parle_set_lr")
+
+    def set_momentum(self, mu: float, vy=None, vx=None):
+        """Nesterov momentum on the y and x^a steps; allocates (zeroed) vy, vx with torch when not given."""
+        import torch
+        if mu > 0 and getattr(self, "vy", None) is None:
+            self.vy = vy if vy is not None else torch.zeros_like(self.x)
+            self.vx = vx if vx is not None else torch.zeros_like(self.x)
+            self._check(self._L.parle_bind_momentum(self._h, _ptr(self.vy), _ptr(self.vx)), "parle_bind_momentum")
+        self._check(self._L.parle_set_momentum(self._h, mu), "parle_set_momentum")
 
     def set_weight_decay(self, lam: float):
         self._check(self._L.parle_set_weight_decay(self._h, lam), "parle_set_weight_decay")

@@ -46,6 +46,8 @@ struct parle_ctx {
     int n, n_layers, batch, gemm_dtype;
     int dims[PARLE_MAX_LAYERS + 1];
     float inv_gamma, inv_rho, alpha, eta, eta_prime, weight_decay;
+    float momentum;                  // Nesterov momentum on the y and x^a steps (0 = off)
+    float *vy, *vx;                  // caller-owned momentum buffers [n, stride] (parle_bind_momentum)
     size_t P, stride;
     size_t sh_stride;                // bf16 path: elements of one replica's blocked weight copy
     size_t sh_off[PARLE_MAX_LAYERS]; int sh_cb[PARLE_MAX_LAYERS], sh_rb[PARLE_MAX_LAYERS];   // per layer: offset, column / row blocks
@@ -310,7 +312,13 @@ int run_inner_update(parle_ctx *c, const float *grad, float wd) {
     float4 *y = reinterpret_cast<float4 *>(c->buf.y), *z = reinterpret_cast<float4 *>(c->buf.z);
     const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
     prof_begin(c, KC_INNER_UPDATE);
-    if (c->fresh)
+    if (c->momentum > 0.f) {
+        float4 *v = reinterpret_cast<float4 *>(c->vy);
+        if (c->fresh)
+            inner_update_kernel<true, U, true><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev, v, c->momentum);
+        else
+            inner_update_kernel<false, U, true><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev, v, c->momentum);
+    } else if (c->fresh)
         inner_update_kernel<true, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev);
     else
         inner_update_kernel<false, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev);
@@ -422,7 +430,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
         return launch_umma<UEPI_DGRAD, UB_BLOCKED_MN>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d);
     };
-    if (!c->fused_update) {
+    if (!c->fused_update || c->momentum > 0.f) {
         for (int l = nl - 1; l >= 0; --l) {
             const int din = c->dims[l], dout = c->dims[l + 1];
             UmmaParams p = {};                                  // dW_l^T = H_{l-1}^T * dH_l
@@ -630,7 +638,7 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
     if (!c->round_open) return PARLE_ESTATE;
     if (c->gemm_dtype == PARLE_GEMM_BF16) {
         PARLE_TRY(forward_backward_bf16(c, inputs, labels, loss_out));
-        if (c->fused_update) {            // y, z and the operand copy were updated by the backward kernels
+        if (c->fused_update && !(c->momentum > 0.f)) {   // y, z and the operand copy were updated by the backward kernels
             c->fresh = false; c->shadow_is_x = false; c->steps_in_round++;
             return PARLE_OK;
         }
@@ -674,8 +682,13 @@ int parle_outer_step(parle_ctx *c) {
     float4 *x = reinterpret_cast<float4 *>(c->buf.x), *xbar = reinterpret_cast<float4 *>(c->buf.xbar);
     const float4 *z = reinterpret_cast<const float4 *>(c->buf.z);
     prof_begin(c, KC_OUTER_MEAN);
-    outer_mean_kernel<4><<<grid, kUpdThreads, 0, c->stream>>>(
-        x, z, xbar, s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
+    if (c->momentum > 0.f)
+        outer_mean_kernel<4, true><<<grid, kUpdThreads, 0, c->stream>>>(
+            x, z, xbar, s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev,
+            reinterpret_cast<float4 *>(c->vx), c->momentum, c->inv_rho);
+    else
+        outer_mean_kernel<4><<<grid, kUpdThreads, 0, c->stream>>>(
+            x, z, xbar, s4, c->n, c->eta, c->eta * c->inv_rho, (float)c->n, c->status_dev);
     PARLE_LAUNCHED(c);
     c->shadow_is_x = false;
     c->round_open = false; c->fresh = false; c->steps_in_round = 0;
@@ -756,6 +769,21 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->fused_update = on != 0;
+    return PARLE_OK;
+}
+
+int parle_bind_momentum(parle_ctx *c, float *vy, float *vx) {
+    if (!c || !vy || !vx) return PARLE_EINVAL;
+    if (reinterpret_cast<uintptr_t>(vy) % 128 || reinterpret_cast<uintptr_t>(vx) % 128) return PARLE_EALIGN;
+    c->vy = vy; c->vx = vx;
+    return PARLE_OK;
+}
+
+int parle_set_momentum(parle_ctx *c, double mu) {
+    if (!c || !(mu >= 0.0 && mu < 1.0)) return PARLE_EINVAL;
+    if (mu > 0.0 && (!c->vy || !c->vx)) return PARLE_ENOTBOUND;
+    if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
+    c->momentum = (float)mu;
     return PARLE_OK;
 }
 

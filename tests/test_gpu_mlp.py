@@ -450,3 +450,25 @@ def test_split_data_round_matches_oracle():
     out = po.parle_round(xo, xb, po.mlp_grad_fn(cfg.dims, X, c), cfg.L, hp)
     x_gpu = to_dense(m, m.x.cpu().numpy())
     assert rel_l2(x_gpu, out["x"]) <= 1e-4 and rel_l2(x_gpu - xo, out["x"] - xo) <= 1e-4
+
+
+@pytest.mark.parametrize("gemm_dtype,dims", [(0, (64, 32, 10)), (1, (64, 128, 72, 10))])
+def test_momentum_rounds_match_oracle(gemm_dtype, dims):
+    """Whole rounds of the MLP with Nesterov momentum 0.9 on the y and x^a steps (the paper's recipe)."""
+    cfg = si.C1.scaled(dims=dims, gemm_dtype=gemm_dtype, L=4, eta_prime=0.02)
+    mu = 0.9
+    m, xo, xb, hp = make(cfg)
+    m.set_momentum(mu)
+    vx = np.zeros_like(xo)
+    tol = TOL[gemm_dtype]
+    for r in range(3):
+        X, c = si.round_batches(cfg, r)
+        m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
+        out = po.parle_round_momentum(xo, xb, vx, po.mlp_grad_fn(cfg.dims, X, c), cfg.L, hp, mu)
+        x_gpu = to_dense(m, m.x.cpu().numpy())
+        for a in range(cfg.n):
+            assert rel_l2(x_gpu[a], out["x"][a]) <= tol
+        assert rel_l2(x_gpu - xo, out["x"] - xo) <= (1e-4 if gemm_dtype == 0 else 5e-2)
+        assert rel_l2(to_dense(m, m.xbar.cpu().numpy()), out["xbar"]) <= tol
+        xo, xb, vx = out["x"], out["xbar"], out["vx"]
+    assert m.status() == 0

@@ -165,3 +165,40 @@ def test_bind_rejects_misaligned_and_small_buffers():
     with pytest.raises(pb.ParleError) as e:
         m.bind(ok(), ok(), ok(), ok(), torch.zeros(S, device=DEV), ws[:16])
     assert e.value.code == -6
+
+
+def test_momentum_rounds_on_a_quadratic_match_oracle():
+    """Nesterov momentum on the y and x^a steps (Remark, Section 3.1) through parle_inner_update /
+    parle_outer_step on flat vectors, three rounds (vy restarts every round, vx carries over)."""
+    n, d, L, mu = 3, 4099, 5, 0.9
+    hp = dict(eta=0.2, eta_prime=0.05, alpha=0.75, gamma=2.0, rho=0.5)
+    lam = si.quadratic_spectrum(9, d)
+    x0, _, _, _ = si.sweep_state(6, n, d)
+    m = _flat(n, d, **hp)
+    xbar0 = x0.astype(np.float64).mean(axis=0).astype(np.float32)
+    _load(m, x0, xbar0)
+    with pytest.raises(pb.ParleError) as e:
+        m._check(pb.lib().parle_set_momentum(m._h, 0.5), "parle_set_momentum")       # no buffers bound yet
+    assert e.value.code == -2
+    m.set_momentum(mu)
+    m.vy.fill_(123.0)                                  # stale y-momentum must not survive the round start
+    lam_dev = torch.zeros(m.stride, device=DEV); lam_dev[:d] = torch.from_numpy(lam.astype(np.float32))
+    lam32 = lam.astype(np.float32).astype(np.float64)
+    xo, xb, vx = x0.astype(np.float64), xbar0.astype(np.float64), np.zeros((n, d))
+    for rnd in range(3):
+        m.round_begin()
+        for l in range(L):
+            m.inner_update((m.x if l == 0 else m.y) * lam_dev)
+        y_gpu = m.y.cpu().numpy()[:, :d]
+        m.outer_step(); torch.cuda.synchronize()
+        out = po.parle_round_momentum(xo, xb, vx, po.quadratic_grad_fn(lam32), L, po.Hyper(**hp), mu)
+        xo, xb, vx = out["x"], out["xbar"], out["vx"]
+        assert rel_l2(y_gpu, out["y"]) < TOL
+        assert rel_l2(m.x.cpu().numpy()[:, :d], xo) < TOL and rel_l2(m.xbar.cpu().numpy()[:d], xb) < TOL
+        assert rel_l2(m.vx.cpu().numpy()[:, :d], vx) < TOL
+    assert m.status() == 0
+    assert torch.all(m.x[:, d:] == 0) and torch.all(m.vx[:, d:] == 0)
+    m.set_momentum(0.0)                                # back to the plain steps
+    m.round_begin(); m.inner_update(m.x * lam_dev); m.outer_step(); torch.cuda.synchronize()
+    out = po.parle_round(xo, xb, po.quadratic_grad_fn(lam32), 1, po.Hyper(**hp))
+    assert rel_l2(m.x.cpu().numpy()[:, :d], out["x"]) < TOL

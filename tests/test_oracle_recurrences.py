@@ -235,3 +235,52 @@ def test_scoping_schedule_closed_form_and_clipping():
     assert all(a[0] >= b[0] and a[1] >= b[1] for a, b in zip(seq, seq[1:]))
     # exact rational check of one value
     assert abs(po.scoping(3.0, 2.0, 2, 3, 1)[0] - float(Fr(3) * Fr(3, 4) ** 3)) < 1e-15
+
+
+def test_momentum_round_matches_torch_nesterov_sgd():
+    """The momentum form is pinned to an independent implementation: torch.optim.SGD(nesterov=True)
+    stepping on the inner objective f(y) + |y - x|^2 / (2 gamma) (Section 2.3) and on the outer
+    objective |x - z|^2 / 2 + |x - xbar|^2 / (2 rho), whose gradients are the directions of Eq. (parle)."""
+    import torch
+    rng = np.random.default_rng(12)
+    d, n, L, mu = 7, 2, 6, 0.9
+    A = rng.normal(size=(d, d)); A = A @ A.T / d
+    hp = po.Hyper(eta=0.3, eta_prime=0.05, alpha=0.75, gamma=2.0, rho=0.5)
+    x = rng.normal(size=(n, d)); xbar = x.mean(axis=0) + 0.1; vx = np.zeros((n, d))
+    At = torch.tensor(A)
+    tx = [torch.tensor(x[a].copy(), requires_grad=True) for a in range(n)]
+    opt_x = [torch.optim.SGD([t], lr=hp.eta, momentum=mu, nesterov=True) for t in tx]
+    txbar = torch.tensor(xbar.copy())
+    for rnd in range(3):
+        out = po.parle_round_momentum(x, xbar, vx, lambda a, l, y: (0.0, A @ y), L, hp, mu)
+        for a in range(n):
+            xa = tx[a].detach().clone()
+            y = xa.clone().requires_grad_(True)
+            z = xa.clone()
+            opt_y = torch.optim.SGD([y], lr=hp.eta_prime, momentum=mu, nesterov=True)   # fresh buffer every round
+            for l in range(L):
+                opt_y.zero_grad()
+                (0.5 * y @ At @ y + ((y - xa) ** 2).sum() / (2 * hp.gamma)).backward()
+                opt_y.step()
+                z = hp.alpha * z + (1 - hp.alpha) * y.detach()
+            np.testing.assert_allclose(out["y"][a], y.detach().numpy(), rtol=1e-12, atol=1e-14)
+            np.testing.assert_allclose(out["z"][a], z.numpy(), rtol=1e-12, atol=1e-14)
+            opt_x[a].zero_grad()
+            (0.5 * ((tx[a] - z) ** 2).sum() + ((tx[a] - txbar) ** 2).sum() / (2 * hp.rho)).backward()
+            opt_x[a].step()                                                            # buffer persists across rounds
+            np.testing.assert_allclose(out["x"][a], tx[a].detach().numpy(), rtol=1e-12, atol=1e-14)
+        x, xbar, vx = out["x"], out["xbar"], out["vx"]
+        txbar = torch.stack([t.detach() for t in tx]).mean(dim=0)
+        np.testing.assert_allclose(xbar, txbar.numpy(), rtol=1e-13)
+
+
+def test_zero_momentum_is_the_plain_round():
+    cfg = si.C1
+    X, c = si.round_batches(cfg, 0)
+    x0 = np.stack([po.pack(si.init_replica(cfg, a)) for a in range(cfg.n)])
+    hp = po.Hyper(cfg.eta, cfg.eta_prime, cfg.alpha, 2.0, 0.5)
+    fn = po.mlp_grad_fn(cfg.dims, X, c)
+    a = po.parle_round(x0, x0.mean(axis=0), fn, cfg.L, hp)
+    b = po.parle_round_momentum(x0, x0.mean(axis=0), np.zeros_like(x0), fn, cfg.L, hp, 0.0)
+    for k in ("x", "xbar", "y", "z"):
+        np.testing.assert_allclose(b[k], a[k], rtol=1e-14, atol=1e-16)
