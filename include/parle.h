@@ -172,6 +172,12 @@ int parle_set_fused_update(parle_ctx *ctx, int on);
 int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);
 int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
 
+/* Tuning knob of the bf16 forward / data-gradient GEMMs: tiles of 128 x 256 instead of 128 x 128 are used
+ * when the batch has at least 256 rows and at least `tiles_per_sm` wide tiles fall on every SM (default 4;
+ * 0 = whenever the batch allows).  Results do not depend on it beyond fp32 summation order inside a tile
+ * (none: the k order is the same). */
+int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
+
 /* Nesterov momentum on the y^a and x^a steps (Remark in Section 3.1; none on xbar).  The paper does not
  * print the form; the one taken is that of SGD with Nesterov momentum: for a step with direction d and
  * step size s,  v <- mu v + d,  p <- p - s (d + mu v), with

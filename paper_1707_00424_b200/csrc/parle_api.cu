@@ -46,6 +46,7 @@ struct parle_ctx {
     int n, n_layers, batch, gemm_dtype;
     int dims[PARLE_MAX_LAYERS + 1];
     float inv_gamma, inv_rho, alpha, eta, eta_prime, weight_decay;
+    int wide_tiles_per_sm;           // 128 x 256 GEMM tiles are used when at least this many of them fall on every SM
     float momentum;                  // Nesterov momentum on the y and x^a steps (0 = off)
     float *vy, *vx;                  // caller-owned momentum buffers [n, stride] (parle_bind_momentum)
     size_t P, stride;
@@ -246,23 +247,37 @@ int build_tensor_maps(parle_ctx *c) {
     return PARLE_OK;
 }
 
-template <int EPI, int BKIND>
-int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
+template <int EPI, int BKIND, int BN>
+int launch_umma_bn(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
     p.groups = c->n;
     p.tiles_m = (p.M + UM_BM - 1) / UM_BM;
-    p.tiles_n = (p.N + UM_BN - 1) / UM_BN;
+    p.tiles_n = (p.N + BN - 1) / BN;
     p.status = c->status_dev;
     const int tiles = p.groups * p.tiles_m * p.tiles_n;
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     prof_begin(c, cls);
-    umma_gemm_kernel<EPI, BKIND><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
+    umma_gemm_kernel<EPI, BKIND, BN><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
     PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
 
+// 256-wide tiles where the product is compute-bound and still leaves every SM several tiles
+// (batch of at least 256 rows and four 128 x 256 tiles per SM); 128-wide tiles otherwise.
+template <int EPI, int BKIND>
+int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, const UmmaParams &p) {
+    if (BKIND != UB_ROWMAJOR_K && p.M >= 256) {
+        const long long wide_tiles = (long long)c->n * ((p.M + UM_BM - 1) / UM_BM) * ((p.N + 255) / 256);
+        if (wide_tiles >= (long long)c->wide_tiles_per_sm * c->sm_count) return launch_umma_bn<EPI, BKIND, 256>(c, cls, a, b, p);
+    }
+    return launch_umma_bn<EPI, BKIND, 128>(c, cls, a, b, p);
+}
+
 template <int EPI, int BKIND>
 cudaError_t allow_big_smem() {
-    return cudaFuncSetAttribute(umma_gemm_kernel<EPI, BKIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(umma_gemm_kernel<EPI, BKIND, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)UM_SMEM_BYTES);
+    if (e != cudaSuccess || BKIND == UB_ROWMAJOR_K) return e;
+    return cudaFuncSetAttribute(umma_gemm_kernel<EPI, BKIND, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)UM_SMEM_BYTES);
 }
 
@@ -553,6 +568,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         c->sh_stride += (size_t)c->sh_rb[l] * c->sh_cb[l] * 8192;
     }
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
+    c->wide_tiles_per_sm = 4;
     plan_workspace(c);
     *out = c;
     return PARLE_OK;
@@ -769,6 +785,12 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->fused_update = on != 0;
+    return PARLE_OK;
+}
+
+int parle_set_wide_tile_threshold(parle_ctx *c, int tiles_per_sm) {
+    if (!c || tiles_per_sm < 0) return PARLE_EINVAL;
+    c->wide_tiles_per_sm = tiles_per_sm;
     return PARLE_OK;
 }
 

@@ -28,7 +28,10 @@ constexpr int UM_STAGE_BYTES = UM_A_BYTES + UM_B_BYTES;    // one k-block of bot
 // replica's weights, which stream from HBM exactly once (about 3 us loaded latency), while the A operand
 // (activations) is shared by all n-tiles of a replica and comes from L2: B gets the deep ring.  With
 // 8 x 16 KiB of weights in flight on every SM the weight stream is not latency-bound.
-constexpr int UM_A_STAGES = 4, UM_B_STAGES = 8;
+constexpr int UM_A_STAGES = 4, UM_B_STAGES = 8;            // B stages of 128 rows; a 256-row tile uses them in pairs
+// Tile width BN (accumulator columns): 128, or 256 where the product is compute-bound and has tiles to spare --
+// per flop a 128 x 256 tile moves 25 % less through shared memory (the limit of a 128 x 128 tile whose both
+// operands stream from shared memory), at the price of all 512 tensor-memory columns for its two accumulators.
 // Warps: 0 = B producer, 1 = MMA issuer, 2..9 = epilogue (two per 32-lane quarter of tensor memory, each taking
 // two of the four 32-column chunks of a tile), 10 = A producer.
 __host__ __device__ constexpr int umma_epi_warps(int) { return 8; }
@@ -169,25 +172,29 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
     return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128.
-__host__ __device__ constexpr uint32_t make_idesc(bool a_mn_major, bool b_mn_major) {
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn_major, bool b_mn_major, int bn = UM_BN) {
     return (1u << 4)                       // D format fp32
          | (1u << 7) | (1u << 10)          // A, B format bf16
          | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16)
-         | ((uint32_t)(UM_BN >> 3) << 17) | ((uint32_t)(UM_BM >> 4) << 24);
+         | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(UM_BM >> 4) << 24);
 }
 
-__device__ __forceinline__ void tile_coords(const UmmaParams &p, int t, int &g, int &m0, int &n0) {
+__device__ __forceinline__ void tile_coords(const UmmaParams &p, int t, int bn, int &g, int &m0, int &n0) {
     const int per_g = p.tiles_m * p.tiles_n;
     g = t / per_g;
     const int r = t - g * per_g;
     m0 = (r % p.tiles_m) * UM_BM;
-    n0 = (r / p.tiles_m) * UM_BN;
+    n0 = (r / p.tiles_m) * bn;
 }
 
-template <int EPI, int BKIND>
+template <int EPI, int BKIND, int BN = UM_BN>
 __global__ void __launch_bounds__(umma_threads(EPI), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const UmmaParams p) {
+    static_assert(BN == 128 || BN == 256, "tile width");
+    constexpr int B_STAGES = UM_B_STAGES * UM_BN / BN;                 // stages of BN rows in the same ring bytes
+    constexpr int B_BYTES = BN * UM_BK * 2;
+    constexpr uint32_t TMEM_COLS = 2 * BN;                             // two accumulators
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // 1024-byte aligned (swizzle atom)
@@ -207,7 +214,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < UM_A_STAGES; ++s) { mbar_init(bar_afull + 8 * s, 1); mbar_init(bar_aempty + 8 * s, 1); }
-        for (int s = 0; s < UM_B_STAGES; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
+        for (int s = 0; s < B_STAGES; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, umma_epi_warps(EPI)); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -215,7 +222,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)UM_TMEM_COLS) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -228,29 +235,34 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                int g, m0, n0; tile_coords(p, t, g, m0, n0);
+                int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(bar_bempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t sb = b_base + stage * UM_B_BYTES;
+                    const uint32_t sb = b_base + stage * B_BYTES;
                     const uint32_t fb = bar_bfull + 8 * stage;
-                    mbar_expect_tx(fb, UM_B_BYTES);
+                    mbar_expect_tx(fb, B_BYTES);
                     if (BKIND == UB_ROWMAJOR_K) {
-                        tma_load_3d(sb, &tmB, fb, kb * UM_BK, n0, g);
+#pragma unroll
+                        for (int h = 0; h < BN / 128; ++h)
+                            tma_load_3d(sb + h * UM_B_BYTES, &tmB, fb, kb * UM_BK, n0 + h * 128, g);
                     } else if (BKIND == UB_BLOCKED_K) {
-                        // block (row block n0/128, column block kb) of the blocked weight copy
-                        tma_load_5d(sb, &tmB, fb, 0, 0, kb, n0 / UM_BN, g);
+                        // blocks (row block n0/128 [+1], column block kb) of the blocked weight copy
+#pragma unroll
+                        for (int h = 0; h < BN / 128; ++h)
+                            tma_load_5d(sb + h * UM_B_BYTES, &tmB, fb, 0, 0, kb, n0 / 128 + h, g);
                     } else {
-                        // k-rows kb*64 .. +63 = half of row block kb/2; n-columns n0 .. n0+127 = column blocks n0/64, n0/64+1
-                        tma_load_5d(sb, &tmB, fb, 0, (kb & 1) * 64, n0 / 64, kb >> 1, g);
-                        tma_load_5d(sb + UM_B_BYTES / 2, &tmB, fb, 0, (kb & 1) * 64, n0 / 64 + 1, kb >> 1, g);
+                        // k-rows kb*64 .. +63 = half of row block kb/2; n-columns n0 .. n0+BN-1 = column blocks n0/64 ...
+#pragma unroll
+                        for (int h = 0; h < BN / 64; ++h)
+                            tma_load_5d(sb + h * (UM_B_BYTES / 2), &tmB, fb, 0, (kb & 1) * 64, n0 / 64 + h, kb >> 1, g);
                     }
-                    if (++stage == UM_B_STAGES) { stage = 0; phase ^= 1u; }
+                    if (++stage == B_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
             if (!ok) {
                 // gave up: let the copies already issued land before the CTA exits
                 // (slots below `stage` were armed in this pass of the ring, the others in the previous one)
-                for (int s = 0; s < UM_B_STAGES; ++s) {
+                for (int s = 0; s < B_STAGES; ++s) {
                     const uint32_t armed_parity = (s < stage) ? phase : (phase ^ 1u);
                     const unsigned long long t0 = global_ns();
                     while (!mbar_try_wait(bar_bfull + 8 * s, armed_parity) && global_ns() - t0 < 20000000ull) {}
@@ -262,7 +274,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                int g, m0, n0; tile_coords(p, t, g, m0, n0);
+                int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(bar_aempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = bar_afull + 8 * stage;
@@ -283,17 +295,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr bool B_MN = (BKIND == UB_BLOCKED_MN);
-            constexpr uint32_t idesc = make_idesc(false, B_MN);
+            constexpr uint32_t idesc = make_idesc(false, B_MN, BN);
             int sa_i = 0, sb_i = 0; uint32_t pa = 0, pb = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * UM_BN;
+                const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(bar_afull + 8 * sa_i, pa, abort_flag)) { ok = false; break; }
                     if (!mbar_wait(bar_bfull + 8 * sb_i, pb, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = a_base + sa_i * UM_A_BYTES, sb = b_base + sb_i * UM_B_BYTES;
+                    const uint32_t sa = a_base + sa_i * UM_A_BYTES, sb = b_base + sb_i * B_BYTES;
                     const uint64_t adesc = make_smem_desc(sa, 16, 1024);
                     const uint64_t bdesc = B_MN ? make_smem_desc(sb, UM_B_BYTES / 2, 1024)
                                                 : make_smem_desc(sb, 16, 1024);
@@ -307,7 +319,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     tc_commit(bar_aempty + 8 * sa_i);        // both slots are free once these MMAs retire
                     tc_commit(bar_bempty + 8 * sb_i);
                     if (++sa_i == UM_A_STAGES) { sa_i = 0; pa ^= 1u; }
-                    if (++sb_i == UM_B_STAGES) { sb_i = 0; pb ^= 1u; }
+                    if (++sb_i == B_STAGES) { sb_i = 0; pb ^= 1u; }
                 }
                 if (!ok) break;
                 tc_commit(bar_tfull + 8 * acc);              // accumulator complete
@@ -320,24 +332,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int half = (warp - 2) >> 2;                    // chunks 2*half, 2*half + 1 of every tile
         int acc = 0; uint32_t acc_phase = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-            int g, m0, n0; tile_coords(p, t, g, m0, n0);
+            int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);
             const int m = m0 + q * 32 + lane;                // output row of this thread
             const bool m_ok = m < p.M;
             // what the epilogue needs besides the accumulator is fetched before the accumulator is awaited
-            float bias_lane[2] = {0.f, 0.f};                 // bias[nb + lane] of this warp's two chunks
-            uint4 mk[2][4];                                  // ReLU mask source: 32 bf16 of row m per chunk
+            constexpr int CPW = BN / 64;                     // 32-column chunks per epilogue warp
+            constexpr bool MASK_AHEAD = (BN == 128);         // wide tiles: the mask is read chunk by chunk (registers)
+            float bias_lane[CPW];                            // bias[nb + lane] of this warp's chunks
+            uint4 mk[MASK_AHEAD ? CPW : 1][4];               // ReLU mask source: 32 bf16 of row m per chunk
             if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_FWD_LAST) {
                 const float *bias = p.bias + (long long)g * p.bias_gs;
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int col = n0 + (2 * half + cc) * 32 + lane;
-                    if (col < p.N) bias_lane[cc] = __ldg(bias + col);
+                for (int cc = 0; cc < CPW; ++cc) {
+                    const int col = n0 + (CPW * half + cc) * 32 + lane;
+                    bias_lane[cc] = (col < p.N) ? __ldg(bias + col) : 0.f;
                 }
             }
-            if (EPI == UEPI_DGRAD) {
+            if (EPI == UEPI_DGRAD && MASK_AHEAD) {
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int nb = n0 + (2 * half + cc) * 32;
+                for (int cc = 0; cc < CPW; ++cc) {
+                    const int nb = n0 + (CPW * half + cc) * 32;
                     const __nv_bfloat16 *mkp = p.mask + (long long)g * p.mask_gs + (long long)m * p.mask_ld + nb;
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8) {
@@ -351,12 +365,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tc_fence_after();
             {
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                const int c = 2 * half + cc;
+            for (int cc = 0; cc < CPW; ++cc) {
+                const int c = CPW * half + cc;
                 const int nb = n0 + c * 32;
                 if (nb >= p.N) break;                        // warp-uniform
+                if (EPI == UEPI_DGRAD && !MASK_AHEAD) {
+                    const __nv_bfloat16 *mkp = p.mask + (long long)g * p.mask_gs + (long long)m * p.mask_ld + nb;
+#pragma unroll
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        mk[0][j8] = make_uint4(0u, 0u, 0u, 0u);
+                        if (m_ok && nb + j8 * 8 < p.N) mk[0][j8] = *reinterpret_cast<const uint4 *>(mkp + j8 * 8);
+                    }
+                }
                 uint32_t r[32];
-                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * UM_BN + c * 32), r);
+                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
                 tc_wait_ld();
                 float v[32];
 #pragma unroll
@@ -371,7 +393,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (EPI == UEPI_DGRAD) {
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8) {
-                        const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&mk[cc][j8]);
+                        const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&mk[MASK_AHEAD ? cc : 0][j8]);
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
                             if (!(__bfloat162float(h[j]) > 0.f)) v[j8 * 8 + j] = 0.f;
@@ -433,7 +455,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (threadIdx.x == 0 && *abort_flag) p.status[SLOT_WAIT_LIMIT] = 1;
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                     ::"r"(tmem_base), "r"((uint32_t)UM_TMEM_COLS) : "memory");
+                     ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 

@@ -472,3 +472,24 @@ def test_momentum_rounds_match_oracle(gemm_dtype, dims):
         assert rel_l2(to_dense(m, m.xbar.cpu().numpy()), out["xbar"]) <= tol
         xo, xb, vx = out["x"], out["xbar"], out["vx"]
     assert m.status() == 0
+
+
+def test_wide_gemm_tiles_give_the_same_step_bf16():
+    """128 x 256 tiles (forced) against 128 x 128 tiles: same k order, so activations, gradients and the
+    updated state agree bit for bit; batch 256 (two M-tiles), widths with a ragged last 256-tile."""
+    cfg = si.C1.scaled(name="wide", n=2, dims=(320, 1152, 648, 101), batch=256, gemm_dtype=1, L=2)
+    X, c = si.round_batches(cfg, 0)
+    res = []
+    for thr in (1 << 20, 0):
+        m, *_ = make(cfg, fused=False)
+        m.set_wide_tile_threshold(thr)
+        m.round_begin()
+        for l in range(cfg.L):
+            m.inner_step(torch.from_numpy(X[l]).to(DEV), torch.from_numpy(c[l]).to(DEV))
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        res.append([m.y.clone(), m.grad.clone(), m.debug_buffer(m.DBG_LOGITS).clone()] +
+                   [m.debug_buffer(m.DBG_ACT, l).clone() for l in range(2)] +
+                   [m.debug_buffer(m.DBG_DACT_T, l).clone() for l in range(3)])
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
