@@ -209,7 +209,7 @@ int parle_status(parle_ctx *ctx, int *device_flags);
 int parle_clear_status(parle_ctx *ctx);
 
 /* Per-kernel-class device timing.  While enabled, every kernel launch is
- * bracketed by a pair of CUDA events on the bound stream (at most 16384
+ * bracketed by a pair of CUDA events on the bound stream (at most 65536
  * launches between two reads; later ones are counted in *dropped).
  * parle_profile_read is the one call that synchronises the stream: it then
  * sums the elapsed times per class into ms[k] / launches[k] for

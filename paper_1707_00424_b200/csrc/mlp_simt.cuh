@@ -87,15 +87,31 @@ __global__ void __launch_bounds__(SG_THREADS) simt_gemm_kernel(SimtGemmArgs p) {
 //   row_loss = logsumexp - logits[label].
 // Writes fp32 dlogits [rows, C] (d32 != NULL) and/or bf16 copies in both
 // layouts: dbf [B, ld_b] per replica and dbfT [C, B] per replica.
+// With parts > 1 the logits arrive as split-K partial sums: logits = bias + sum_s part_s (s in fixed order),
+// formed here first and written back over part 0 (= the logits buffer).
 __global__ void __launch_bounds__(256)
-softmax_ce_backward_kernel(const float *__restrict__ logits, const int32_t *__restrict__ labels,
+softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict__ labels,
                            float *__restrict__ d32, __nv_bfloat16 *__restrict__ dbf,
                            __nv_bfloat16 *__restrict__ dbfT, float *__restrict__ row_loss,
-                           int rows, int B, int C, int ld_b, int *status) {
+                           int rows, int B, int C, int ld_b, int *status,
+                           int parts = 1, long long part_stride = 0, const float *__restrict__ bias = nullptr,
+                           long long bias_gs = 0) {
     const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const int lane = threadIdx.x % 32;
     if (row >= rows) return;
-    const float *lg = logits + (size_t)row * C;
+    float *lg = logits + (size_t)row * C;
+    if (parts > 1) {
+        const float *bg = bias + (long long)(row / B) * bias_gs;
+        for (int j = lane; j < C; j += 32) {
+            float pv[8];                             // parts <= 8: all loads in flight before the fixed-order sum
+#pragma unroll
+            for (int q = 0; q < 8; ++q) pv[q] = (q < parts) ? lg[(long long)q * part_stride + j] : 0.f;
+            float s = pv[0];
+#pragma unroll
+            for (int q = 1; q < 8; ++q) s += pv[q];
+            lg[j] = s + bg[j];                       // read back below by the same lane
+        }
+    }
     float mx = -INFINITY;
     for (int j = lane; j < C; j += 32) mx = fmaxf(mx, lg[j]);
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));

@@ -15,7 +15,7 @@ using namespace parle;
 namespace {
 
 constexpr size_t kWsAlign = 1024;
-constexpr int kProfCapacity = 16384;       // launches recorded between two parle_profile_read calls
+constexpr int kProfCapacity = 65536;       // launches recorded between two parle_profile_read calls
 
 enum KernelClass {
     KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_LOSS_MEAN, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
@@ -29,7 +29,7 @@ struct Workspace {
     // byte offsets into parle_buffers.workspace; index = layer (0-based)
     size_t act[PARLE_MAX_LAYERS];      // fp32 mode: output of layer l  [n,B,d_{l+1}] fp32 (last = logits)
     size_t dact[PARLE_MAX_LAYERS];     // fp32 mode: gradient w.r.t. layer l's output [n,B,d_{l+1}] fp32
-    size_t logits;                     // bf16 mode: fp32 logits [n,B,C]
+    size_t logits;                     // bf16 mode: fp32 logits [n,B,C] (x last_ksplit partial sums when split-K is used)
     size_t shadow;                     // bf16 mode: blocked bf16 copy of the weights [n, sh_stride]
     size_t xb, xbT;                    // bf16 mode: inputs [n,B,d_0] and transposed [n,d_0,B]
     size_t hb[PARLE_MAX_LAYERS], hbT[PARLE_MAX_LAYERS];      // hidden activations, both layouts
@@ -46,6 +46,7 @@ struct parle_ctx {
     int n, n_layers, batch, gemm_dtype;
     int dims[PARLE_MAX_LAYERS + 1];
     float inv_gamma, inv_rho, alpha, eta, eta_prime, weight_decay;
+    int last_ksplit;                 // split-K factor of the last forward layer (1 = off)
     int wide_tiles_per_sm;           // 128 x 256 GEMM tiles are used when at least this many of them fall on every SM
     float momentum;                  // Nesterov momentum on the y and x^a steps (0 = off)
     float *vy, *vx;                  // caller-owned momentum buffers [n, stride] (parle_bind_momentum)
@@ -126,7 +127,7 @@ void plan_workspace(parle_ctx *c) {
             w.hb[l] = take(n * B * c->dims[l + 1] * 2);
             w.hbT[l] = take(n * B * c->dims[l + 1] * 2);
         }
-        w.logits = take(n * B * C * sizeof(float));
+        w.logits = take(n * B * C * sizeof(float) * (size_t)c->last_ksplit);
         for (int l = 0; l < nl; ++l) {
             w.dh_ld[l] = (int)round_up(c->dims[l + 1], 8);
             w.dhb[l] = take(n * B * w.dh_ld[l] * 2);
@@ -253,7 +254,7 @@ int launch_umma_bn(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMa
     p.tiles_m = (p.M + UM_BM - 1) / UM_BM;
     p.tiles_n = (p.N + BN - 1) / BN;
     p.status = c->status_dev;
-    const int tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int tiles = p.groups * p.tiles_m * p.tiles_n * ((EPI == UEPI_FWD_LAST && p.ksplit > 1) ? p.ksplit : 1);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     prof_begin(c, cls);
     umma_gemm_kernel<EPI, BKIND, BN><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
@@ -421,6 +422,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
             PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         } else {
             p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
+            p.ksplit = c->last_ksplit; p.part_ss = (long long)n * B * dout;
             PARLE_TRY((launch_umma<UEPI_FWD_LAST, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         }
     }
@@ -429,7 +431,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
         ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
-        c->status_dev);
+        c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S);
     PARLE_LAUNCHED(c);
     if (loss_out) {
         prof_begin(c, KC_LOSS_MEAN);
@@ -569,6 +571,18 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
     }
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
     c->wide_tiles_per_sm = 4;
+    c->last_ksplit = 1;
+    if (c->fused_update) {
+        // the last forward layer often has one tile per replica: when its tiles would leave most SMs idle, its k-blocks are
+        // split over several CTAs (partial sums, added up with the bias by the softmax kernel in fixed order)
+        const int nl = c->n_layers;
+        const int tiles = c->n * ((c->batch + 127) / 128) * ((c->dims[nl] + 127) / 128);
+        const int num_kb = (c->dims[nl - 1] + 63) / 64;
+        int s = 148 / (tiles > 0 ? tiles : 1);
+        if (s > 8) s = 8;
+        if (s > num_kb / 2) s = num_kb / 2;
+        if (s >= 2) c->last_ksplit = s;
+    }
     plan_workspace(c);
     *out = c;
     return PARLE_OK;

@@ -63,6 +63,9 @@ struct UmmaParams {
     __nv_bfloat16 *outT; long long outT_gs; int outT_ld;
     float *outf; long long outf_gs; int outf_ld;
     const __nv_bfloat16 *mask; long long mask_gs; int mask_ld;
+    // split-K (UEPI_FWD_LAST only): each tile's k-blocks are divided among ksplit work items, each of which
+    // stores its raw partial sums (no bias) at outf + split * part_ss; a later kernel adds them up in fixed order
+    int ksplit; long long part_ss;
     int *status;
 };
 
@@ -211,6 +214,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.groups * p.tiles_m * p.tiles_n;
     const int num_kb = (p.K + UM_BK - 1) / UM_BK;
+    const int ksplit = (EPI == UEPI_FWD_LAST && p.ksplit > 1) ? p.ksplit : 1;
+    const int total_items = total_tiles * ksplit;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < UM_A_STAGES; ++s) { mbar_init(bar_afull + 8 * s, 1); mbar_init(bar_aempty + 8 * s, 1); }
@@ -234,9 +239,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------ TMA producer of the B operand (deep ring)
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+                const int t = it / ksplit, split = it - t * ksplit;
+                const int kb_lo = split * num_kb / ksplit, kb_hi = (split + 1) * num_kb / ksplit;
                 int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(bar_bempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sb = b_base + stage * B_BYTES;
                     const uint32_t fb = bar_bfull + 8 * stage;
@@ -273,9 +280,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------ TMA producer of the A operand
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+                const int t = it / ksplit, split = it - t * ksplit;
+                const int kb_lo = split * num_kb / ksplit, kb_hi = (split + 1) * num_kb / ksplit;
                 int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(bar_aempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = bar_afull + 8 * stage;
                     mbar_expect_tx(fb, UM_A_BYTES);
@@ -297,11 +306,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             constexpr bool B_MN = (BKIND == UB_BLOCKED_MN);
             constexpr uint32_t idesc = make_idesc(false, B_MN, BN);
             int sa_i = 0, sb_i = 0; uint32_t pa = 0, pb = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+                const int t = it / ksplit, split = it - t * ksplit;
+                const int kb_lo = split * num_kb / ksplit, kb_hi = (split + 1) * num_kb / ksplit;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(bar_afull + 8 * sa_i, pa, abort_flag)) { ok = false; break; }
                     if (!mbar_wait(bar_bfull + 8 * sb_i, pb, abort_flag)) { ok = false; break; }
                     tc_fence_after();
@@ -314,7 +325,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         // K-major: 16 bf16 = 32 B further along the row; MN-major: two 8-row groups = 2048 B
                         const uint64_t a_k = adesc + (uint64_t)(k * 2);
                         const uint64_t b_k = bdesc + (uint64_t)(B_MN ? k * 128 : k * 2);
-                        tc_mma_bf16(d_tmem, a_k, b_k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc_mma_bf16(d_tmem, a_k, b_k, idesc, (kb != kb_lo || k != 0) ? 1u : 0u);
                     }
                     tc_commit(bar_aempty + 8 * sa_i);        // both slots are free once these MMAs retire
                     tc_commit(bar_bempty + 8 * sb_i);
@@ -331,7 +342,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;                              // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;                    // chunks 2*half, 2*half + 1 of every tile
         int acc = 0; uint32_t acc_phase = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        for (int it = blockIdx.x; it < total_items; it += gridDim.x) {
+            const int t = it / ksplit, split = it - t * ksplit;
             int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);
             const int m = m0 + q * 32 + lane;                // output row of this thread
             const bool m_ok = m < p.M;
@@ -345,7 +357,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                 for (int cc = 0; cc < CPW; ++cc) {
                     const int col = n0 + (CPW * half + cc) * 32 + lane;
-                    bias_lane[cc] = (col < p.N) ? __ldg(bias + col) : 0.f;
+                    bias_lane[cc] = (col < p.N && ksplit == 1) ? __ldg(bias + col) : 0.f;
                 }
             }
             if (EPI == UEPI_DGRAD && MASK_AHEAD) {
@@ -425,7 +437,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 if (EPI == UEPI_FWD_LAST) {
                     if (m_ok) {
-                        float *o = p.outf + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
+                        float *o = p.outf + (long long)split * p.part_ss + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             if (nb + j < p.N) o[j] = v[j];
