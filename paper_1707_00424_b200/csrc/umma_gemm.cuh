@@ -37,8 +37,12 @@ constexpr int UM_A_STAGES = 4, UM_B_STAGES = 8;            // B stages of 128 ro
 __host__ __device__ constexpr int umma_epi_warps(int) { return 8; }
 __host__ __device__ constexpr int umma_threads(int epi) { return 96 + 32 * umma_epi_warps(epi); }
 constexpr int UM_TMEM_COLS = 256;                          // two 128-column accumulators
+// Per epilogue warp: a 32 x 32 bf16 scratch tile (rows padded to 80 bytes) through which the transposed copy of an
+// output chunk is turned into 16-byte stores.
+constexpr int UM_EPI_PITCH = 40;                           // bf16 elements per scratch row (32 + 8 padding)
+constexpr int UM_EPI_SCRATCH = 32 * UM_EPI_PITCH * 2;      // bytes per warp
 constexpr size_t UM_SMEM_BYTES = (size_t)UM_A_STAGES * UM_A_BYTES + (size_t)UM_B_STAGES * UM_B_BYTES +
-                                 1024 /*alignment slack*/ + 256 /*barriers*/;
+                                 8 * UM_EPI_SCRATCH + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long UM_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
 
 // How the B operand is fetched.
@@ -202,7 +206,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // 1024-byte aligned (swizzle atom)
     const uint32_t a_base = tiles_base, b_base = tiles_base + UM_A_STAGES * UM_A_BYTES;
-    uint8_t *ctl = smem_raw + (tiles_base - raw) + (size_t)UM_A_STAGES * UM_A_BYTES + (size_t)UM_B_STAGES * UM_B_BYTES;
+    uint8_t *epi_scratch = smem_raw + (tiles_base - raw) + (size_t)UM_A_STAGES * UM_A_BYTES + (size_t)UM_B_STAGES * UM_B_BYTES;
+    uint8_t *ctl = epi_scratch + 8 * UM_EPI_SCRATCH;
     uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);   // a_full[SA], a_empty[SA], b_full[SB], b_empty[SB], tfull[2], tempty[2]
     constexpr int NBARS = 2 * UM_A_STAGES + 2 * UM_B_STAGES + 4;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * NBARS);
@@ -428,11 +433,27 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                 *reinterpret_cast<uint4 *>(o + j8) = pk;
                             }
                         }
-                        // transposed bf16 [N, ldT]: the 32 lanes write 32 consecutive batch rows
-                        __nv_bfloat16 *oT = p.outT + (long long)g * p.outT_gs + m;
+                    }
+                    // transposed bf16 [N, ldT]: through this warp's scratch tile, so that a lane stores 8 consecutive
+                    // batch rows of one feature (16 bytes) instead of 32 two-byte pieces
+                    {
+                        __nv_bfloat16 *sT = reinterpret_cast<__nv_bfloat16 *>(epi_scratch + (warp - 2) * UM_EPI_SCRATCH);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < p.N) oT[(long long)(nb + j) * p.outT_ld] = __float2bfloat16_rn(v[j]);
+                        for (int j = 0; j < 32; ++j) sT[j * UM_EPI_PITCH + lane] = __float2bfloat16_rn(v[j]);
+                        __syncwarp();
+                        const int seg = lane & 3;                          // 8 batch rows each
+                        const int mrow = m0 + q * 32 + seg * 8;
+                        if (mrow < p.M) {                                  // M % 8 == 0: the whole group is inside
+                            __nv_bfloat16 *oT = p.outT + (long long)g * p.outT_gs + mrow;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int f = (lane >> 2) + 8 * i;
+                                if (nb + f < p.N)
+                                    *reinterpret_cast<uint4 *>(oT + (long long)(nb + f) * p.outT_ld) =
+                                        *reinterpret_cast<const uint4 *>(sT + f * UM_EPI_PITCH + seg * 8);
+                            }
+                        }
+                        __syncwarp();
                     }
                 }
                 if (EPI == UEPI_FWD_LAST) {
