@@ -493,3 +493,19 @@ def test_wide_gemm_tiles_give_the_same_step_bf16():
                    [m.debug_buffer(m.DBG_DACT_T, l).clone() for l in range(3)])
     for a, b in zip(*res):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("n,dims,batch", [(1, (8, 8, 3), 8), (5, (16, 8, 24, 2), 8), (16, (72, 264, 10), 40),
+                                          (2, (136, 128, 256, 129), 264)])
+def test_edge_shapes_round_bf16(n, dims, batch):
+    """Smallest legal sizes, one replica, a batch that is not a multiple of the 128-row tile (264 = 2 tiles + 8),
+    widths straddling the 64-column blocks of the weight copy: whole-round parity, fused and unfused agree bit for bit."""
+    cfg = si.C1.scaled(name="edge", n=n, dims=dims, batch=batch, gemm_dtype=1, L=3)
+    run_rounds(cfg, 2, disp_tol=6e-2)
+    X, c = si.round_batches(cfg, 0)
+    res = []
+    for fused in (True, False):
+        m, *_ = make(cfg, fused=fused)
+        m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
+        res.append((m.x.clone(), m.xbar.clone()))
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
