@@ -186,8 +186,8 @@ int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
  * parle_bind_momentum attaches the two caller-owned buffers, dev [n, stride] fp32, 128-byte aligned;
  * vx must be zero before the first round (vy needs no initialisation).  parle_set_momentum(mu), mu in
  * [0, 1): 0 switches momentum off; ENOTBOUND if mu > 0 without buffers, ESTATE in the middle of a round.
- * With momentum on, the bf16 path writes the gradient to `grad` and runs the separate update kernel
- * (the fused weight-gradient epilogue has no momentum variant). */
+ * Call parle_bind_momentum after parle_bind (and again after every later parle_bind).  On the bf16 path the
+ * fused weight-gradient kernel has a momentum variant (vy is staged with x, y, z: 30 bytes per weight and step). */
 int parle_bind_momentum(parle_ctx *ctx, float *vy, float *vx);
 int parle_set_momentum(parle_ctx *ctx, double mu);
 

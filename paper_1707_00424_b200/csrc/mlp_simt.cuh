@@ -204,10 +204,11 @@ struct TailPlan {
     const __nv_bfloat16 *dHT[PARLE_MAX_LAYERS];      // [n, d_out, B]
 };
 
-template <bool FIRST>
+template <bool FIRST, bool MOM = false>
 __global__ void __launch_bounds__(128)
 tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__ z, const float *__restrict__ x,
-                   long long stride, float eta_p, float inv_gamma, float alpha, float wd, int *status) {
+                   long long stride, float eta_p, float inv_gamma, float alpha, float wd, int *status,
+                   float *__restrict__ v = nullptr, float mu = 0.f) {
     const int l = blockIdx.y, g = blockIdx.z;
     const long long e = tp.begin[l] + (long long)blockIdx.x * 128 + threadIdx.x;     // one thread per element
     if (e >= tp.end[l]) return;
@@ -219,7 +220,13 @@ tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__
     const long long i = (long long)g * stride + e;
     const float xv = x[i];
     const float yo = FIRST ? xv : y[i], zo = FIRST ? xv : z[i];
-    const float yn = yo - eta_p * fmaf(inv_gamma, yo - xv, fmaf(wd, yo, grad));
+    float d = fmaf(inv_gamma, yo - xv, fmaf(wd, yo, grad));
+    if (MOM) {                                    // Nesterov momentum, v = 0 at the start of a round
+        const float vn = FIRST ? d : fmaf(mu, v[i], d);
+        v[i] = vn;
+        d = fmaf(mu, vn, d);
+    }
+    const float yn = yo - eta_p * d;
     const float zn = fmaf(alpha, zo, (1.0f - alpha) * yn);
     y[i] = yn;
     z[i] = zn;

@@ -69,6 +69,8 @@ struct parle_ctx {
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_sx[PARLE_MAX_LAYERS], tm_sy[PARLE_MAX_LAYERS], tm_sz[PARLE_MAX_LAYERS];   // fp32 W_l segments of x, y, z
+    CUtensorMap tm_mx[PARLE_MAX_LAYERS], tm_my[PARLE_MAX_LAYERS], tm_mz[PARLE_MAX_LAYERS], tm_mv[PARLE_MAX_LAYERS];   // same + vy, 16-row boxes (momentum variant)
+    bool mom_maps;
     // host-buffer rounds: a second stream uploads the next minibatch while the current step runs
     cudaStream_t copy_stream;
     cudaEvent_t ev_copied[2], ev_consumed[2];
@@ -447,7 +449,8 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
         return launch_umma<UEPI_DGRAD, UB_BLOCKED_MN>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d);
     };
-    if (!c->fused_update || c->momentum > 0.f) {
+    const bool mom = c->momentum > 0.f;
+    if (!c->fused_update) {
         for (int l = nl - 1; l >= 0; --l) {
             const int din = c->dims[l], dout = c->dims[l + 1];
             UmmaParams p = {};                                  // dW_l^T = H_{l-1}^T * dH_l
@@ -480,12 +483,20 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         const int tiles = p.groups * p.tiles_m * p.tiles_n;
         const int grid = tiles < c->sm_count ? tiles : c->sm_count;
         prof_begin(c, KC_WGRAD_UPDATE);
-        if (c->fresh)
+        if (mom) {
+            p.v = c->vy + wo; p.mu = c->momentum;
+            if (c->fresh)
+                umma_wgrad_update_kernel<true, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(
+                    c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p);
+            else
+                umma_wgrad_update_kernel<false, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(
+                    c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p);
+        } else if (c->fresh)
             umma_wgrad_update_kernel<true, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
-                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], p);
+                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p);
         else
             umma_wgrad_update_kernel<false, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
-                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], p);
+                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p);
         PARLE_LAUNCHED(c);
     }
     TailPlan tp = {};
@@ -501,7 +512,13 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     }
     const dim3 tgrid((unsigned)((longest + 127) / 128), nl, n);
     prof_begin(c, KC_TAIL_UPDATE);
-    if (c->fresh)
+    if (mom && c->fresh)
+        tail_update_kernel<true, true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S, c->eta_prime, c->inv_gamma,
+                                                                     c->alpha, c->weight_decay, c->status_dev, c->vy, c->momentum);
+    else if (mom)
+        tail_update_kernel<false, true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S, c->eta_prime, c->inv_gamma,
+                                                                      c->alpha, c->weight_decay, c->status_dev, c->vy, c->momentum);
+    else if (c->fresh)
         tail_update_kernel<true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
                                                                c->eta_prime, c->inv_gamma, c->alpha, c->weight_decay, c->status_dev);
     else
@@ -642,6 +659,9 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, UB_ROWMAJOR_K>()));
         PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
         PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true, WuMomentum, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuMomentum::SMEM_BYTES));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false, WuMomentum, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuMomentum::SMEM_BYTES));
+        c->mom_maps = false;
         PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, UB_BLOCKED_MN>()));
         PARLE_TRY(build_tensor_maps(c));
         // rows / columns of the blocked weight copy beyond the matrices are never written: they must read as zero
@@ -668,7 +688,7 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
     if (!c->round_open) return PARLE_ESTATE;
     if (c->gemm_dtype == PARLE_GEMM_BF16) {
         PARLE_TRY(forward_backward_bf16(c, inputs, labels, loss_out));
-        if (c->fused_update && !(c->momentum > 0.f)) {   // y, z and the operand copy were updated by the backward kernels
+        if (c->fused_update) {            // y, z and the operand copy were updated by the backward kernels
             c->fresh = false; c->shadow_is_x = false; c->steps_in_round++;
             return PARLE_OK;
         }
@@ -812,12 +832,26 @@ int parle_bind_momentum(parle_ctx *c, float *vy, float *vx) {
     if (!c || !vy || !vx) return PARLE_EINVAL;
     if (reinterpret_cast<uintptr_t>(vy) % 128 || reinterpret_cast<uintptr_t>(vx) % 128) return PARLE_EALIGN;
     c->vy = vy; c->vx = vx;
+    c->mom_maps = false;
+    if (c->bound && c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16) {
+        // tensor maps of the fused weight-gradient kernel's momentum variant (16-row boxes of x, y, z, vy)
+        for (int l = 0; l < c->n_layers; ++l) {
+            const size_t din = c->dims[l], dout = c->dims[l + 1], wo = c->layers[l].w_off;
+            float *base[4] = {c->buf.x + wo, c->buf.y + wo, c->buf.z + wo, vy + wo};
+            CUtensorMap *tm[4] = {&c->tm_mx[l], &c->tm_my[l], &c->tm_mz[l], &c->tm_mv[l]};
+            for (int k = 0; k < 4; ++k)
+                PARLE_TRY(encode_f32_map(c, tm[k], base[k], din, dout, c->n, din, c->stride, UM_BM, WU_CHUNK_ROWS_MOM));
+        }
+        c->mom_maps = true;
+    }
     return PARLE_OK;
 }
 
 int parle_set_momentum(parle_ctx *c, double mu) {
     if (!c || !(mu >= 0.0 && mu < 1.0)) return PARLE_EINVAL;
     if (mu > 0.0 && (!c->vy || !c->vx)) return PARLE_ENOTBOUND;
+    if (mu > 0.0 && c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16 && !c->mom_maps)
+        return PARLE_ENOTBOUND;      // momentum buffers were attached before parle_bind (or parle_bind was called again)
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->momentum = (float)mu;
     return PARLE_OK;

@@ -35,12 +35,12 @@ constexpr int WU_STATE_RING_BYTES = 144 * 1024;                // shared memory 
 
 // Shape of the epilogue: G groups of 4 warps share chunks of CR W-rows (accumulator columns);
 // every thread owns CR / G rows of one column.
-template <int G, int CR>
+template <int G, int CR, int NA = 3>
 struct WuShape {
     static constexpr int GROUPS = G, CHUNK_ROWS = CR, RPG = CR / G;
     static constexpr int CHUNKS = UM_BN / CR;
-    static constexpr int ARRAY_BYTES = CR * UM_BM * 4;          // one fp32 box of x, y or z
-    static constexpr int STATE_BYTES = 3 * ARRAY_BYTES;         // x | y | z
+    static constexpr int ARRAY_BYTES = CR * UM_BM * 4;          // one fp32 box of x, y, z (or the momentum v)
+    static constexpr int STATE_BYTES = NA * ARRAY_BYTES;        // x | y | z [| v]
     static constexpr int STAGES = WU_STATE_RING_BYTES / STATE_BYTES;
     static constexpr int THREADS = 96 + 128 * G;
     static constexpr size_t SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)STAGES * STATE_BYTES +
@@ -49,7 +49,9 @@ struct WuShape {
     static_assert(STAGES >= 2 && 2 * WU_OP_STAGES + 4 + 2 * STAGES <= 30, "stage count");
 };
 using WuDefault = WuShape<4, 32>;
+using WuMomentum = WuShape<4, 16, 4>;                          // with the momentum buffer staged too: 16-row chunks
 constexpr int WU_CHUNK_ROWS = WuDefault::CHUNK_ROWS;           // TMA box height of the x/y/z tensor maps
+constexpr int WU_CHUNK_ROWS_MOM = WuMomentum::CHUNK_ROWS;      // ... of the maps used by the momentum variant
 
 template <int N> __device__ __forceinline__ void tc_ld_cols(uint32_t taddr, uint32_t (&r)[N]);
 template <> __device__ __forceinline__ void tc_ld_cols<4>(uint32_t taddr, uint32_t (&r)[4]) { tc_ld_32x4(taddr, r); }
@@ -68,14 +70,18 @@ struct WgradUpdateParams {
     long long shadow_gs; int shadow_cb;   // replica pitch (elements) and column blocks per row block
     long long gs; int ld;
     float eta_p, inv_gamma, alpha, wd;
+    float *v; float mu;          // Nesterov momentum buffer of y (same addressing as y), used by the MOM variant
     int *status;
 };
 
-template <bool FIRST, class SH>
+// MOM: Nesterov momentum on the y step (see inner_update_kernel): v <- mu v + d, y <- y - eta' (d + mu v),
+// v = 0 at the start of a round (FIRST: v is only written).
+template <bool FIRST, class SH, bool MOM = false>
 __global__ void __launch_bounds__(SH::THREADS, 1)
 umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
-                         const __grid_constant__ CUtensorMap tmZ, const WgradUpdateParams p) {
+                         const __grid_constant__ CUtensorMap tmZ, const __grid_constant__ CUtensorMap tmV,
+                         const WgradUpdateParams p) {
     constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
     constexpr int WU_STATE_BYTES = SH::STATE_BYTES, WU_STATE_STAGES = SH::STAGES, RPG = SH::RPG;
     constexpr int WU_CHUNK_ROWS = SH::CHUNK_ROWS;
@@ -185,11 +191,12 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     if (!mbar_wait(bar_sempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t dst = st_base + stage * WU_STATE_BYTES;
                     const uint32_t fb = bar_sfull + 8 * stage;
-                    mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES);
+                    mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES);   // STATE_BYTES counts v when MOM
                     tma_load_3d(dst, &tmX, fb, m0, nb, g);
                     if (!FIRST) {
                         tma_load_3d(dst + WU_ARRAY_BYTES, &tmY, fb, m0, nb, g);
                         tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &tmZ, fb, m0, nb, g);
+                        if (MOM) tma_load_3d(dst + 3 * WU_ARRAY_BYTES, &tmV, fb, m0, nb, g);
                     }
                     if (++stage == WU_STATE_STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -223,12 +230,14 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             const long long tile_e0 = (long long)g * p.gs + (long long)(n0 + grp * RPG) * p.ld + m;
             const long long chunk_step = (long long)WU_CHUNK_ROWS * p.ld;
             float *yp = p.y + tile_e0, *zp = p.z + tile_e0;
+            float *vp = MOM ? p.v + tile_e0 : nullptr;
             // blocked copy: W row r, column m live in block (r/128, m/64) at (r%128)*64 + m%64; n0 % 128 == 0
             __nv_bfloat16 *sp = p.shadow + (long long)g * p.shadow_gs +
                                 ((long long)(n0 / UM_BN) * p.shadow_cb + (m >> 6)) * (UM_BN * 64) +
                                 (grp * RPG) * 64 + (m & 63);
 #pragma unroll 1
             for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
+                if (MOM && c > 0) vp += chunk_step;
                 const int nb0 = n0 + c * WU_CHUNK_ROWS;
                 if (nb0 >= p.N) break;                       // same rule as the loader
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
@@ -236,13 +245,14 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 const int nb = nb0 + grp * RPG;
                 const float *sx = reinterpret_cast<const float *>(st_ptr + (size_t)stage * WU_STATE_BYTES) +
                                   grp * RPG * UM_BM + col;
-                float xv[RPG], yv[RPG], zv[RPG];
+                float xv[RPG], yv[RPG], zv[RPG], vv[RPG];
 #pragma unroll
                 for (int j = 0; j < RPG; ++j) {
                     xv[j] = sx[j * UM_BM];
                     if (!FIRST) {
                         yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
                         zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
+                        if (MOM) vv[j] = sx[3 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                     }
                 }
                 uint32_t r[RPG];
@@ -254,31 +264,34 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
                 if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
                 const int rows = m_ok ? (p.N - nb) : 0;      // rows of this thread that exist
-                float *yr = yp, *zr = zp;
+                float *yr = yp, *zr = zp, *vr = vp;
                 __nv_bfloat16 *sr = sp;
+                auto update_row = [&](int j) {
+                    const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
+                    float d = fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j])));
+                    if (MOM) {
+                        const float vn = FIRST ? d : fmaf(p.mu, vv[j], d);      // v = 0 before the first step of a round
+                        *vr = vn;
+                        d = fmaf(p.mu, vn, d);
+                    }
+                    const float yn = fmaf(neg_eta_p, d, yo);
+                    const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
+                    chk = fmaf(yn, 0.f, chk);
+                    *yr = yn;
+                    *zr = zn;
+                    *sr = __float2bfloat16_rn(yn);
+                };
                 if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
                     for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
-                        const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
-                        const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j]))), yo);
-                        const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
-                        chk = fmaf(yn, 0.f, chk);
-                        *yr = yn;
-                        *zr = zn;
-                        *sr = __float2bfloat16_rn(yn);
+                        update_row(j);
+                        if (MOM) vr += p.ld;
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
-                        if (j < rows) {
-                            const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
-                            const float yn = fmaf(neg_eta_p, fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j]))), yo);
-                            const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
-                            chk = fmaf(yn, 0.f, chk);
-                            *yr = yn;
-                            *zr = zn;
-                            *sr = __float2bfloat16_rn(yn);
-                        }
+                        if (j < rows) update_row(j);
+                        if (MOM) vr += p.ld;
                     }
                 }
             }

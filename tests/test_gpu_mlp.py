@@ -509,3 +509,25 @@ def test_edge_shapes_round_bf16(n, dims, batch):
         m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)); torch.cuda.synchronize()
         res.append((m.x.clone(), m.xbar.clone()))
     assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+
+
+@pytest.mark.parametrize("dims,batch,n", [((64, 128, 72, 10), 16, 3), ((200, 328, 136, 101), 136, 2),
+                                          ((3072, 2048, 2048, 100), 128, 2)])
+def test_fused_momentum_update_equals_separate_update_bf16(dims, batch, n):
+    """Momentum variant of the fused weight-gradient kernel == gradient written out + update kernel with
+    momentum: y, z, the momentum buffer and the bf16 copy agree bit for bit over two rounds."""
+    cfg = si.C1.scaled(name="fusedmom", n=n, dims=dims, batch=batch, gemm_dtype=1, L=3, eta_prime=0.02)
+    res = []
+    for fused in (True, False):
+        m, *_ = make(cfg, fused=fused)
+        m.set_momentum(0.9)
+        m.vy.fill_(5.0)                                  # stale y-momentum must not survive the round start
+        for r in range(2):
+            X, c = si.round_batches(cfg, r)
+            m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV))
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        res.append((m.x.clone(), m.y.clone(), m.z.clone(), m.vy.clone(), m.vx.clone(),
+                    m.debug_buffer(m.DBG_OPERAND_COPY).clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
