@@ -191,6 +191,7 @@ def run_ours(args):
     else:
         model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
     model.mean()
+    model.set_round_graphs(bool(args.graphs))
     sets = 2
     Xh, ch = make_round_inputs(cfg, sets)
     Xd, cd = torch.from_numpy(Xh).to(dev), torch.from_numpy(ch).to(dev)
@@ -291,6 +292,7 @@ def run_ours(args):
                                f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else 'fp32'}",
                    "step": "one Parle round (L inner steps + outer step + replica mean)",
                    "l2": "state + gradients per round >> 126 MB L2 (no flush needed)" if cfg.n * model.stride * 16 > 4e8 else "working set may be L2 resident",
+                   "launch": "rounds replayed from CUDA graphs (same kernels, same order)" if args.graphs else "one launch per kernel",
                    "parallelism": f"{world} x {cfg.n} replicas, one all-reduce of xbar per round" if world > 1 else "single GPU"},
         "gpu_launches": launches, "device_flags": flags, "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -376,6 +378,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))
+    ap.add_argument("--graphs", type=int, default=1, help="replay rounds from CUDA graphs (parle_set_round_graphs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

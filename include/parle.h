@@ -150,6 +150,17 @@ int parle_mean(parle_ctx *ctx);
 int parle_round(parle_ctx *ctx, int L, const float *inputs, const int32_t *labels,
                 float *loss_out);
 
+/* on: parle_round replays the round from a CUDA graph.  The first call with a given (L, inputs, labels, loss_out)
+ * and unchanged settings records the round's launches on a stream of the library's own (created at that
+ * moment) and instantiates them; later calls with the same arguments launch the graph on the bound stream: same kernels, same order, same results, without the per-launch cost.  Up to eight graphs are cached
+ * (least recently used is dropped); changing a setting, the buffers or the stream makes a new graph.  Off by
+ * default.  parle_round_host then replays each inner step from a graph of its own (its staging buffers have
+ * fixed addresses).  Ignored while per-kernel timing is enabled.  If the stream cannot be captured the library falls
+ * back to plain launches by itself. */
+int parle_set_round_graphs(parle_ctx *ctx, int on);
+/* Number of round graphs currently cached; -1 when graph replay is off (never switched on, or given up). */
+int parle_round_graph_count(const parle_ctx *ctx);
+
 /* A whole round from host buffers: inputs host [L, n, B, d_0], labels host
  * [L, n, B], loss_out host [L, n] or NULL.  The minibatch of step l+1 is uploaded
  * on a second stream into a second staging buffer while step l computes, so with

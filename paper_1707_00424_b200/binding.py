@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
         "parle_mean": (ci, [vp]),
         "parle_round": (ci, [vp, ci, vp, vp, vp]),
         "parle_round_host": (ci, [vp, ci, vp, vp, vp]),
+        "parle_set_round_graphs": (ci, [vp, ci]),
+        "parle_round_graph_count": (ci, [vp]),
         "parle_set_coupling": (ci, [vp, cd, cd]),
         "parle_set_lr": (ci, [vp, cd, cd]),
         "parle_set_fused_update": (ci, [vp, ci]),
@@ -226,6 +228,13 @@ class Parle:
     def round_host(self, L: int, inputs_host, labels_host, loss_out_host=None):
         self._check(self._L.parle_round_host(self._h, L, _ptr(inputs_host), _ptr(labels_host), _ptr(loss_out_host)),
                     "parle_round_host")
+
+    def set_round_graphs(self, on: bool):
+        self._check(self._L.parle_set_round_graphs(self._h, 1 if on else 0), "parle_set_round_graphs")
+
+    @property
+    def round_graph_count(self) -> int:
+        return self._L.parle_round_graph_count(self._h)
 
     def set_coupling(self, gamma: float, rho: float):
         self._check(self._L.parle_set_coupling(self._h, gamma, rho), "parle_set_coupling")

@@ -42,6 +42,24 @@ struct Workspace {
 
 }  // namespace
 
+namespace {
+// Everything a captured round depends on: if any of it changes, the graph is rebuilt.
+struct RoundKey {
+    int L;
+    const void *inputs, *labels, *loss;
+    float scal[7];                   // 1/gamma, 1/rho, alpha, eta, eta', weight decay, momentum
+    int fused, wide_thr, shadow_is_x, fresh;   // L == 0: a single inner step (fresh = first of its round)
+    const void *ptrs[9];             // x, y, z, grad, xbar, workspace, vy, vx, stream
+};
+struct RoundGraph {
+    RoundKey key;
+    cudaGraphExec_t exec;
+    long long launches;              // kernels inside the graph
+    unsigned long long last_use;
+};
+constexpr int kRoundGraphs = 8;
+}  // namespace
+
 struct parle_ctx {
     int n, n_layers, batch, gemm_dtype;
     int dims[PARLE_MAX_LAYERS + 1];
@@ -71,6 +89,12 @@ struct parle_ctx {
     CUtensorMap tm_sx[PARLE_MAX_LAYERS], tm_sy[PARLE_MAX_LAYERS], tm_sz[PARLE_MAX_LAYERS];   // fp32 W_l segments of x, y, z
     CUtensorMap tm_mx[PARLE_MAX_LAYERS], tm_my[PARLE_MAX_LAYERS], tm_mz[PARLE_MAX_LAYERS], tm_mv[PARLE_MAX_LAYERS];   // same + vy, 16-row boxes (momentum variant)
     bool mom_maps;
+    // parle_round as a CUDA graph (optional): a small cache of instantiated rounds
+    bool graphs_on;
+    cudaStream_t capture_stream;     // rounds are captured here (the bound stream may be the default stream, which cannot be)
+    RoundGraph graphs[kRoundGraphs];
+    int n_graphs;
+    unsigned long long graph_clock;
     // host-buffer rounds: a second stream uploads the next minibatch while the current step runs
     cudaStream_t copy_stream;
     cudaEvent_t ev_copied[2], ev_consumed[2];
@@ -81,6 +105,8 @@ struct parle_ctx {
     cudaEvent_t *prof_ev;            // 2 * kProfCapacity events
     unsigned char *prof_cls;
 };
+
+extern "C" { static void drop_round_graphs(parle_ctx *c); }
 
 namespace {
 
@@ -608,6 +634,8 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
 void parle_destroy(parle_ctx *c) {
     if (!c) return;
     if (c->status_host) cudaFreeHost(c->status_host);
+    drop_round_graphs(c);
+    if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
     if (c->copy_ready) {
         cudaStreamDestroy(c->copy_stream);
         for (int b = 0; b < 2; ++b) { cudaEventDestroy(c->ev_copied[b]); cudaEventDestroy(c->ev_consumed[b]); }
@@ -639,6 +667,7 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         if (reinterpret_cast<uintptr_t>(p) % 128) return PARLE_EALIGN;
     if (b->workspace_bytes < c->ws.total) return PARLE_EWORKSPACE;
     c->bound = false;
+    drop_round_graphs(c);
     int dev = 0;
     PARLE_CUDA(c, cudaGetDevice(&dev));
     PARLE_CUDA(c, cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
@@ -755,9 +784,121 @@ int parle_mean(parle_ctx *c) {
     return PARLE_OK;
 }
 
+static int round_direct(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out);
+
+static RoundKey make_round_key(const parle_ctx *c, int L, const void *in, const void *lab, const void *loss) {
+    RoundKey k;
+    memset(&k, 0, sizeof(k));
+    k.L = L; k.inputs = in; k.labels = lab; k.loss = loss;
+    const float sc[7] = {c->inv_gamma, c->inv_rho, c->alpha, c->eta, c->eta_prime, c->weight_decay, c->momentum};
+    memcpy(k.scal, sc, sizeof(sc));
+    k.fused = c->fused_update; k.wide_thr = c->wide_tiles_per_sm; k.shadow_is_x = c->shadow_is_x; k.fresh = c->fresh;
+    const void *pt[9] = {c->buf.x, c->buf.y, c->buf.z, c->buf.grad, c->buf.xbar, c->buf.workspace, c->vy, c->vx, c->stream};
+    memcpy(k.ptrs, pt, sizeof(pt));
+    return k;
+}
+
+static void restore_before(parle_ctx *c, const RoundKey &key, int L, int steps_before) {
+    c->shadow_is_x = key.shadow_is_x != 0;
+    c->fresh = key.fresh != 0;
+    c->steps_in_round = steps_before;
+    c->round_open = (L == 0);        // a round call starts with no round open, a step call inside an open round
+}
+
+static void drop_round_graphs(parle_ctx *c) {
+    for (int i = 0; i < c->n_graphs; ++i) cudaGraphExecDestroy(c->graphs[i].exec);
+    c->n_graphs = 0;
+}
+
+// The whole round replayed from an instantiated CUDA graph: the kernels are the same and run in the same
+// order, only the per-launch host and scheduling cost goes away (one graph launch instead of ~14 L launches).
+static int round_graphed(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
+    const RoundKey key = make_round_key(c, L, inputs, labels, loss_out);
+    RoundGraph *g = nullptr;
+    for (int i = 0; i < c->n_graphs; ++i)
+        if (memcmp(&c->graphs[i].key, &key, sizeof(key)) == 0) g = &c->graphs[i];
+    if (!g) {
+        cudaGraph_t graph = nullptr;
+        const long long before = c->launches;
+        if (!c->capture_stream && cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError();
+            c->capture_stream = nullptr; c->graphs_on = false;
+            return L > 0 ? round_direct(c, L, inputs, labels, loss_out) : parle_inner_step(c, inputs, labels, loss_out);
+        }
+        if (cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+            cudaGetLastError();
+            c->graphs_on = false;                       // capture is not possible here: plain launches from now on
+            return L > 0 ? round_direct(c, L, inputs, labels, loss_out) : parle_inner_step(c, inputs, labels, loss_out);
+        }
+        cudaStream_t bound = c->stream;
+        c->stream = c->capture_stream;                  // the launches of this one round are recorded, not run
+        const int steps_before = c->steps_in_round;
+        const int rc = L > 0 ? round_direct(c, L, inputs, labels, loss_out)
+                             : parle_inner_step(c, inputs, labels, loss_out);
+        c->stream = bound;
+        const cudaError_t e = cudaStreamEndCapture(c->capture_stream, &graph);
+        const long long inside = c->launches - before;
+        c->launches = before;
+        if (rc != PARLE_OK || e != cudaSuccess || !graph) {
+            if (graph) cudaGraphDestroy(graph);
+            cudaGetLastError();
+            c->graphs_on = false;
+            // nothing ran during the failed capture: restore the host state of before and run it plainly
+            restore_before(c, key, L, steps_before);
+            if (rc != PARLE_OK) return rc;
+            return L > 0 ? round_direct(c, L, inputs, labels, loss_out) : parle_inner_step(c, inputs, labels, loss_out);
+        }
+        cudaGraphExec_t exec = nullptr;
+        const cudaError_t ei = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (ei != cudaSuccess) {
+            cudaGetLastError();
+            c->graphs_on = false;
+            restore_before(c, key, L, steps_before);
+            return L > 0 ? round_direct(c, L, inputs, labels, loss_out) : parle_inner_step(c, inputs, labels, loss_out);
+        }
+        // the captured call advanced the host state as if it had run; rewind, the launch below replays it
+        restore_before(c, key, L, steps_before);
+        int slot = c->n_graphs;
+        if (slot == kRoundGraphs) {                     // evict the least recently used
+            slot = 0;
+            for (int i = 1; i < kRoundGraphs; ++i)
+                if (c->graphs[i].last_use < c->graphs[slot].last_use) slot = i;
+            cudaGraphExecDestroy(c->graphs[slot].exec);
+        } else {
+            c->n_graphs++;
+        }
+        g = &c->graphs[slot];
+        g->key = key; g->exec = exec; g->launches = inside;
+    }
+    g->last_use = ++c->graph_clock;
+    PARLE_CUDA(c, cudaGraphLaunch(g->exec, c->stream));
+    c->launches += g->launches;
+    if (L > 0) {      // host-side state after a round (what round_direct leaves behind)
+        c->round_open = false; c->fresh = false; c->steps_in_round = 0; c->shadow_is_x = false;
+    } else {          // ... after one inner step
+        c->fresh = false; c->shadow_is_x = false; c->steps_in_round++;
+    }
+    return PARLE_OK;
+}
+
 int parle_round(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
     PARLE_TRY(check_bound(c));
     if (L < 1 || c->n_layers == 0 || !inputs || !labels) return PARLE_EINVAL;
+    if (c->graphs_on && !c->prof_on) return round_graphed(c, L, inputs, labels, loss_out);
+    return round_direct(c, L, inputs, labels, loss_out);
+}
+
+int parle_round_graph_count(const parle_ctx *c) { return c ? (c->graphs_on ? c->n_graphs : -1) : 0; }
+
+int parle_set_round_graphs(parle_ctx *c, int on) {
+    if (!c) return PARLE_EINVAL;
+    c->graphs_on = on != 0;
+    if (!on) drop_round_graphs(c);
+    return PARLE_OK;
+}
+
+static int round_direct(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
     PARLE_TRY(parle_round_begin(c));
     const size_t nb = (size_t)c->n * c->batch;
     for (int l = 0; l < L; ++l)
@@ -798,8 +939,12 @@ int parle_round_host(parle_ctx *c, int L, const float *inputs_host, const int32_
         if (l + 1 < L) PARLE_TRY(upload(l + 1));
         PARLE_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
         float *dloss = ws_ptr<float>(c, c->ws.stage_loss[b]);
-        PARLE_TRY(parle_inner_step(c, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
-                                   loss_out_host ? dloss : nullptr));
+        if (c->graphs_on && !c->prof_on)       // the step's kernels as one cached graph (staging buffers have fixed addresses)
+            PARLE_TRY(round_graphed(c, 0, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
+                                    loss_out_host ? dloss : nullptr));
+        else
+            PARLE_TRY(parle_inner_step(c, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
+                                       loss_out_host ? dloss : nullptr));
         if (loss_out_host)
             PARLE_CUDA(c, cudaMemcpyAsync(loss_out_host + (size_t)l * c->n, dloss, c->n * sizeof(float),
                                           cudaMemcpyDeviceToHost, c->stream));

@@ -531,3 +531,49 @@ def test_fused_momentum_update_equals_separate_update_bf16(dims, batch, n):
                     m.debug_buffer(m.DBG_OPERAND_COPY).clone()))
     for a, b in zip(*res):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("gemm_dtype,dims", [(0, (64, 32, 10)), (1, (64, 128, 72, 10))])
+def test_graph_rounds_equal_plain_rounds(gemm_dtype, dims):
+    """parle_round replayed from a CUDA graph gives bit-identical state, also when the inputs alternate
+    between two sets (two cached graphs), when a setting changes (new graph) and with more input sets than
+    the cache holds."""
+    cfg = si.C1.scaled(dims=dims, gemm_dtype=gemm_dtype, L=4)
+    sets = [si.round_batches(cfg, r) for r in range(10)]
+    dev = [(torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)) for X, c in sets]
+    res = []
+    for graphs in (False, True):
+        m, *_ = make(cfg)
+        m.set_round_graphs(graphs)
+        loss = torch.zeros(cfg.L, cfg.n, device=DEV)
+        before = m.launch_count
+        for r in (0, 1, 0, 1):
+            m.round(cfg.L, dev[r][0], dev[r][1], loss)
+        per_round = (m.launch_count - before) // 4
+        assert m.round_graph_count == (2 if graphs else -1)
+        m.set_coupling(3.0, 0.5)                          # a changed setting must not replay the old graph
+        m.round(cfg.L, dev[0][0], dev[0][1], loss)
+        for r in range(10):                               # more input sets than cached graphs (8)
+            m.round(cfg.L, dev[r][0], dev[r][1], loss)
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        assert m.round_graph_count == (8 if graphs else -1)
+        res.append((m.x.clone(), m.xbar.clone(), m.y.clone(), m.z.clone(), loss.clone(), per_round))
+    for a, b in zip(res[0][:5], res[1][:5]):
+        assert torch.equal(a, b)
+    assert res[0][5] == res[1][5] > 0                     # the launch count reports the kernels inside the graph
+    # host-buffer rounds: every inner step replayed from a step graph (two staging buffers, first / later step)
+    X, c = sets[0]
+    Xh, ch = torch.from_numpy(X).pin_memory(), torch.from_numpy(c).pin_memory()
+    outs = []
+    for graphs in (False, True):
+        m, *_ = make(cfg)
+        m.set_round_graphs(graphs)
+        lh = torch.zeros(cfg.L, cfg.n).pin_memory()
+        for r in range(3):
+            m.round_host(cfg.L, Xh, ch, lh)
+        torch.cuda.synchronize()
+        assert m.round_graph_count == (3 if graphs else -1)
+        outs.append((m.x.clone(), m.xbar.clone(), lh.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
