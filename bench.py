@@ -114,18 +114,26 @@ def dense_to_padded(model, cfg, replica_layers):
 
 # DRAM bytes per launch (mean over the four launches of an inner step) of the dominant kernel from the committed
 # ncu capture (profiles/ncu_full_gemms_and_fused_update_C3.md), valid only while the kernel source is unchanged.
-NCU_TRAFFIC = {("C3", "wgrad_gemm_fused_update"): {"bytes": 2481.4e6 / 4, "source_sha256_16": "3cb53c5f13b19919",
-                                                   "source": "paper_1707_00424_b200/csrc/umma_wgrad_update.cuh"}}
+NCU_TRAFFIC = {("C3", "wgrad_gemm_fused_update"): {
+    # dram__bytes_read.sum + dram__bytes_write.sum, mean over the four layers' launches of one inner step
+    "bytes": 2479.96e6 / 4,
+    "sources": ("paper_1707_00424_b200/csrc/umma_wgrad_update.cuh", "paper_1707_00424_b200/csrc/umma_gemm.cuh"),
+    "sources_sha256_16": "9d3a29e7efb49222"}}
+
+
+def sources_digest(sources):
+    import hashlib
+    h = hashlib.sha256()
+    for rel in sources:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
 
 
 def ncu_traffic(workload: str, kernel: str):
-    import hashlib
     rec = NCU_TRAFFIC.get((workload, kernel))
-    if not rec:
-        return None
-    with open(os.path.join(ROOT, rec["source"]), "rb") as f:
-        if hashlib.sha256(f.read()).hexdigest()[:16] != rec["source_sha256_16"]:
-            return None         # kernel changed since the counters were taken
+    if not rec or sources_digest(rec["sources"]) != rec["sources_sha256_16"]:
+        return None             # no capture, or the kernel changed since the counters were taken
     return rec["bytes"]
 
 
