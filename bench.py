@@ -200,7 +200,6 @@ def run_ours(args):
         model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
     model.mean()
     model.set_round_graphs(bool(args.graphs))
-    model.set_launch_overlap(bool(args.overlap))
     sets = 2
     Xh, ch = make_round_inputs(cfg, sets)
     Xd, cd = torch.from_numpy(Xh).to(dev), torch.from_numpy(ch).to(dev)
@@ -388,8 +387,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))
     ap.add_argument("--graphs", type=int, default=1, help="replay rounds from CUDA graphs (parle_set_round_graphs)")
-    ap.add_argument("--overlap", type=int, default=1,
-                    help="with --graphs 0: let each kernel of a step start while its predecessor drains (parle_set_launch_overlap)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

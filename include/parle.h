@@ -183,18 +183,6 @@ int parle_set_fused_update(parle_ctx *ctx, int on);
 int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);
 int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
 
-/* Scheduling knob of the bf16 path (default on; it has no effect on rounds replayed from CUDA graphs,
- * whose kernel nodes already run back to back): inside an inner step, and from step to step inside
- * parle_round, every kernel after the first is launched so that it may be scheduled while the kernel
- * before it is still draining (programmatic dependent launch): its set-up, and loads of data that the
- * kernel before it does not write (weights for the forward and data-gradient products of Section 2.1's
- * gradient, x/y/z tiles for the fused update of Eq. parle_y / parle_z), overlap that kernel's tail; it
- * waits for the predecessor's completion before it touches anything else.  The first kernel of every call
- * is an ordinary launch, so work queued on the stream by others is always complete first.  The arithmetic
- * and its order are unchanged: results are bit-identical with the knob on or off.  The paper has no
- * counterpart (it is a property of this implementation's launches). */
-int parle_set_launch_overlap(parle_ctx *ctx, int on);
-
 /* Tuning knob of the bf16 forward / data-gradient GEMMs: tiles of 128 x 256 instead of 128 x 128 are used
  * when the batch has at least 256 rows and at least `tiles_per_sm` wide tiles fall on every SM (default 4;
  * 0 = whenever the batch allows).  Results do not depend on it beyond fp32 summation order inside a tile

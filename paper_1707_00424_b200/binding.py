@@ -73,7 +73,6 @@ def lib() -> C.CDLL:
         "parle_set_fused_update": (ci, [vp, ci]),
         "parle_set_weight_decay": (ci, [vp, cd]),
         "parle_set_wide_tile_threshold": (ci, [vp, ci]),
-        "parle_set_launch_overlap": (ci, [vp, ci]),
         "parle_bind_momentum": (ci, [vp, vp, vp]),
         "parle_set_momentum": (ci, [vp, cd]),
         "parle_scoping": (ci, [cd, cd, C.c_longlong, C.c_longlong, cd, cd, C.POINTER(cd), C.POINTER(cd)]),
@@ -251,9 +250,6 @@ class Parle:
             self.vx = vx if vx is not None else torch.zeros_like(self.x)
             self._check(self._L.parle_bind_momentum(self._h, _ptr(self.vy), _ptr(self.vx)), "parle_bind_momentum")
         self._check(self._L.parle_set_momentum(self._h, mu), "parle_set_momentum")
-
-    def set_launch_overlap(self, on: bool):
-        self._check(self._L.parle_set_launch_overlap(self._h, int(bool(on))), "parle_set_launch_overlap")
 
     def set_wide_tile_threshold(self, tiles_per_sm: int):
         self._check(self._L.parle_set_wide_tile_threshold(self._h, tiles_per_sm), "parle_set_wide_tile_threshold")

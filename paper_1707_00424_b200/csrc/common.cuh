@@ -17,15 +17,6 @@ enum StatusSlot { SLOT_NONFINITE = 0, SLOT_WAIT_LIMIT = 1, SLOT_BAD_LABEL = 2, S
 
 __host__ __device__ inline size_t round_up(size_t v, size_t m) { return (v + m - 1) / m * m; }
 
-// Programmatic dependent launch.  A kernel launched with the stream-serialization attribute may start
-// while the kernel before it in the stream is still running; dep_wait() returns once that kernel has
-// completed and its writes are visible, dep_release() lets the kernel after this one start.  Every
-// kernel here calls dep_release() only after dep_wait(), so when a kernel starts, everything older than
-// its immediate predecessor has completed: what a kernel touches before dep_wait() must be data that
-// the immediate predecessor does not write.  Both are no-ops in a kernel launched the ordinary way.
-__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
 struct LayerPlan {
     int d_in, d_out;
     size_t w_off, b_off;          // element offsets inside one replica's vector

@@ -96,8 +96,6 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
                            int rows, int B, int C, int ld_b, int *status,
                            int parts = 1, long long part_stride = 0, const float *__restrict__ bias = nullptr,
                            long long bias_gs = 0) {
-    dep_wait();
-    dep_release();
     const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const int lane = threadIdx.x % 32;
     if (row >= rows) return;
@@ -145,8 +143,6 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
 __global__ void __launch_bounds__(256)
 loss_mean_kernel(const float *__restrict__ row_loss, float *__restrict__ loss, int B) {
     __shared__ float sh[256];
-    dep_wait();
-    dep_release();
     const int g = blockIdx.x;
     float s = 0.f;
     for (int i = threadIdx.x; i < B; i += 256) s += row_loss[(size_t)g * B + i];
@@ -213,8 +209,6 @@ __global__ void __launch_bounds__(128)
 tail_update_kernel(const TailPlan tp, float *__restrict__ y, float *__restrict__ z, const float *__restrict__ x,
                    long long stride, float eta_p, float inv_gamma, float alpha, float wd, int *status,
                    float *__restrict__ v = nullptr, float mu = 0.f) {
-    dep_wait();
-    dep_release();
     const int l = blockIdx.y, g = blockIdx.z;
     const long long e = tp.begin[l] + (long long)blockIdx.x * 128 + threadIdx.x;     // one thread per element
     if (e >= tp.end[l]) return;
@@ -280,8 +274,6 @@ __global__ void __launch_bounds__(256)
 input_to_bf16_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ Xb,
                      __nv_bfloat16 *__restrict__ XbT, int B, int d) {
     __shared__ __nv_bfloat16 tile[64][64 + 8];
-    dep_wait();
-    dep_release();
     const int g = blockIdx.z;
     const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
     const int c4 = (threadIdx.x % 16) * 4, r0 = threadIdx.x / 16;          // 16 threads x 4 features per batch row

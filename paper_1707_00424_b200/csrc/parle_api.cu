@@ -3,7 +3,6 @@
 #include <math.h>
 #include <new>
 #include <string.h>
-#include <utility>
 
 #include "common.cuh"
 #include "mlp_simt.cuh"
@@ -17,9 +16,6 @@ namespace {
 
 constexpr size_t kWsAlign = 1024;
 constexpr int kProfCapacity = 65536;       // launches recorded between two parle_profile_read calls
-
-// Kernels of an inner step's launch chain (see launch_chained).
-enum PrevKind { PK_NONE = 0, PK_INPUT_CVT, PK_FWD, PK_SOFTMAX, PK_LOSS_MEAN, PK_DGRAD, PK_WGRAD_UPDATE, PK_TAIL };
 
 enum KernelClass {
     KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_LOSS_MEAN, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
@@ -83,10 +79,6 @@ struct parle_ctx {
     int *status_host, *status_dev;
     bool round_open, fresh, shadow_is_x;
     bool fused_update;               // bf16 path: apply Eq. (parle_y)/(parle_z) inside the weight-gradient GEMM
-    // programmatic dependent launch inside an inner step of the bf16 path: what the previous launch of the
-    // current chain was (PK_NONE: the next launch is an ordinary, fully serialised one)
-    bool overlap_on, chain_steps;
-    int prev_kind, prev_layer;
     int steps_in_round;
     long long launches;
     int last_cuda;
@@ -123,7 +115,7 @@ inline int cuda_fail(parle_ctx *c, cudaError_t e) {
     return PARLE_ECUDA;
 }
 #define PARLE_CUDA(c, expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
-#define PARLE_LAUNCHED(c) do { (c)->launches++; (c)->prev_kind = PK_NONE; prof_end(c); cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
+#define PARLE_LAUNCHED(c) do { (c)->launches++; prof_end(c); cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return cuda_fail((c), e_); } while (0)
 
 inline void prof_begin(parle_ctx *c, int cls) {
     if (!c->prof_on) return;
@@ -139,29 +131,6 @@ inline void prof_end(parle_ctx *c) {
     c->prof_open = false;
 }
 #define PARLE_TRY(expr) do { int rc_ = (expr); if (rc_ != PARLE_OK) return rc_; } while (0)
-
-// A launch that belongs to the chain of an inner step.  After the first kernel of a chain every kernel is
-// launched with the programmatic stream-serialization attribute: it may be scheduled while its predecessor
-// is still running and waits for it inside the kernel (dep_wait) before it touches anything the predecessor
-// writes.  `kind` / `layer` are remembered so that the next launch can tell what its predecessor writes.
-template <class... P, class... A>
-int launch_chained(parle_ctx *c, int cls, int kind, int layer, void (*kern)(P...), dim3 grid, dim3 block, size_t smem,
-                   A &&...args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = (c->overlap_on && c->prev_kind != PK_NONE) ? 1 : 0;
-    prof_begin(c, cls);
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...);
-    PARLE_LAUNCHED(c);
-    if (e != cudaSuccess) return cuda_fail(c, e);
-    c->prev_kind = kind; c->prev_layer = layer;
-    return PARLE_OK;
-}
-inline bool chained(const parle_ctx *c) { return c->overlap_on && c->prev_kind != PK_NONE; }
 
 inline bool coupling_ok(double v) { return v > 0.0 && !isnan(v); }
 inline float inverse_or_zero(double v) { return isinf(v) ? 0.0f : (float)(1.0 / v); }
@@ -307,47 +276,29 @@ int build_tensor_maps(parle_ctx *c) {
     return PARLE_OK;
 }
 
-// What the B operand's producer may do before the dependency wait: the forward product reads the bf16
-// weight copy, which neither the input conversion nor another forward product writes; the data-gradient
-// product of layer l reads the copy of W_l, which the loss kernels and the fused update of another layer
-// leave alone.  Anything else (or an ordinary launch): wait first.
-inline int early_b_allowed(const parle_ctx *c, int kind, int layer) {
-    if (!chained(c)) return 0;
-    if (kind == PK_FWD) return c->prev_kind == PK_INPUT_CVT || c->prev_kind == PK_FWD;
-    if (kind == PK_DGRAD)
-        return c->prev_kind == PK_SOFTMAX || c->prev_kind == PK_LOSS_MEAN ||
-               (c->prev_kind == PK_WGRAD_UPDATE && c->prev_layer != layer);
-    return 0;
-}
-
 template <int EPI, int BKIND, int BN>
-int launch_umma_bn(parle_ctx *c, int cls, int kind, int layer, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
+int launch_umma_bn(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, UmmaParams p) {
     p.groups = c->n;
     p.tiles_m = (p.M + UM_BM - 1) / UM_BM;
     p.tiles_n = (p.N + BN - 1) / BN;
     p.status = c->status_dev;
     const int tiles = p.groups * p.tiles_m * p.tiles_n * ((EPI == UEPI_FWD_LAST && p.ksplit > 1) ? p.ksplit : 1);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    if (kind == PK_NONE) {
-        prof_begin(c, cls);
-        umma_gemm_kernel<EPI, BKIND, BN><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
-        PARLE_LAUNCHED(c);
-        return PARLE_OK;
-    }
-    p.early_b = early_b_allowed(c, kind, layer);
-    return launch_chained(c, cls, kind, layer, umma_gemm_kernel<EPI, BKIND, BN>, dim3(grid), dim3(umma_threads(EPI)),
-                          UM_SMEM_BYTES, a, b, p);
+    prof_begin(c, cls);
+    umma_gemm_kernel<EPI, BKIND, BN><<<grid, umma_threads(EPI), UM_SMEM_BYTES, c->stream>>>(a, b, p);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
 }
 
 // 256-wide tiles where the product is compute-bound and still leaves every SM several tiles
 // (batch of at least 256 rows and four 128 x 256 tiles per SM); 128-wide tiles otherwise.
 template <int EPI, int BKIND>
-int launch_umma(parle_ctx *c, int cls, int kind, int layer, const CUtensorMap &a, const CUtensorMap &b, const UmmaParams &p) {
+int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, const UmmaParams &p) {
     if (BKIND != UB_ROWMAJOR_K && p.M >= 256) {
         const long long wide_tiles = (long long)c->n * ((p.M + UM_BM - 1) / UM_BM) * ((p.N + 255) / 256);
-        if (wide_tiles >= (long long)c->wide_tiles_per_sm * c->sm_count) return launch_umma_bn<EPI, BKIND, 256>(c, cls, kind, layer, a, b, p);
+        if (wide_tiles >= (long long)c->wide_tiles_per_sm * c->sm_count) return launch_umma_bn<EPI, BKIND, 256>(c, cls, a, b, p);
     }
-    return launch_umma_bn<EPI, BKIND, 128>(c, cls, kind, layer, a, b, p);
+    return launch_umma_bn<EPI, BKIND, 128>(c, cls, a, b, p);
 }
 
 template <int EPI, int BKIND>
@@ -483,9 +434,10 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     const float *params = c->fresh ? c->buf.x : c->buf.y;      // fp32 biases come from the master copy
     {
         const int d0 = c->dims[0];
-        PARLE_TRY(launch_chained(c, KC_INPUT_CVT, PK_INPUT_CVT, 0, input_to_bf16_kernel,
-                                 dim3((d0 + 63) / 64, (B + 63) / 64, n), dim3(256), 0,
-                                 inputs, ws_ptr<__nv_bfloat16>(c, w.xb), ws_ptr<__nv_bfloat16>(c, w.xbT), B, d0));
+        prof_begin(c, KC_INPUT_CVT);
+        input_to_bf16_kernel<<<dim3((d0 + 63) / 64, (B + 63) / 64, n), 256, 0, c->stream>>>(
+            inputs, ws_ptr<__nv_bfloat16>(c, w.xb), ws_ptr<__nv_bfloat16>(c, w.xbT), B, d0);
+        PARLE_LAUNCHED(c);
     }
     for (int l = 0; l < nl; ++l) {
         const int din = c->dims[l], dout = c->dims[l + 1];
@@ -495,22 +447,25 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         if (l + 1 < nl) {
             p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
             p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
-            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, PK_FWD, l, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         } else {
             p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
             p.ksplit = c->last_ksplit; p.part_ss = (long long)n * B * dout;
-            PARLE_TRY((launch_umma<UEPI_FWD_LAST, UB_BLOCKED_K>(c, KC_FWD_GEMM, PK_FWD, l, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_FWD_LAST, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         }
     }
     const int C = c->dims[nl], rows = n * B;
-    PARLE_TRY(launch_chained(c, KC_SOFTMAX_CE, PK_SOFTMAX, 0, softmax_ce_backward_kernel, dim3((rows + 7) / 8), dim3(256), 0,
-                             ws_ptr<float>(c, w.logits), labels, (float *)nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
-                             ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C,
-                             w.dh_ld[nl - 1], c->status_dev, c->last_ksplit, (long long)n * B * C,
-                             params + c->layers[nl - 1].b_off, S));
-    if (loss_out)
-        PARLE_TRY(launch_chained(c, KC_LOSS_MEAN, PK_LOSS_MEAN, 0, loss_mean_kernel, dim3(n), dim3(256), 0,
-                                 ws_ptr<float>(c, w.row_loss), loss_out, B));
+    prof_begin(c, KC_SOFTMAX_CE);
+    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+        ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
+        ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
+        c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S);
+    PARLE_LAUNCHED(c);
+    if (loss_out) {
+        prof_begin(c, KC_LOSS_MEAN);
+        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
+        PARLE_LAUNCHED(c);
+    }
     auto dgrad = [&](int l) -> int {                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
         const int din = c->dims[l], dout = c->dims[l + 1];
         UmmaParams d = {};
@@ -518,7 +473,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
         d.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); d.outT_gs = (long long)B * din; d.outT_ld = B;
         d.mask = ws_ptr<__nv_bfloat16>(c, w.hb[l - 1]); d.mask_gs = (long long)B * din; d.mask_ld = din;
-        return launch_umma<UEPI_DGRAD, UB_BLOCKED_MN>(c, KC_DGRAD_GEMM, PK_DGRAD, l, c->tm_dg_a[l], c->tm_dg_b[l], d);
+        return launch_umma<UEPI_DGRAD, UB_BLOCKED_MN>(c, KC_DGRAD_GEMM, c->tm_dg_a[l], c->tm_dg_b[l], d);
     };
     const bool mom = c->momentum > 0.f;
     if (!c->fused_update) {
@@ -527,7 +482,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
             UmmaParams p = {};                                  // dW_l^T = H_{l-1}^T * dH_l
             p.M = din; p.N = dout; p.K = B;
             p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
-            PARLE_TRY((launch_umma<UEPI_WGRAD, UB_ROWMAJOR_K>(c, KC_WGRAD_GEMM, PK_NONE, l, c->tm_wg_a[l], c->tm_wg_b[l], p)));
+            PARLE_TRY((launch_umma<UEPI_WGRAD, UB_ROWMAJOR_K>(c, KC_WGRAD_GEMM, c->tm_wg_a[l], c->tm_wg_b[l], p)));
             prof_begin(c, KC_BIAS_GRAD);
             bias_grad_bf16_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(
                 ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), c->buf.grad + c->layers[l].b_off, S, B, dout);
@@ -552,32 +507,23 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha; p.wd = c->weight_decay;
         p.status = c->status_dev;
         const int tiles = p.groups * p.tiles_m * p.tiles_n;
-        const dim3 grid(tiles < c->sm_count ? tiles : c->sm_count);
-        // x, y, z (and v) of layer l are written by this layer's kernel only: the state loader need not wait for
-        // a data-gradient product or for the fused update of another layer
-        p.early_state = chained(c) && (c->prev_kind == PK_DGRAD || (c->prev_kind == PK_WGRAD_UPDATE && c->prev_layer != l));
+        const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+        prof_begin(c, KC_WGRAD_UPDATE);
         if (mom) {
             p.v = c->vy + wo; p.mu = c->momentum;
-            const dim3 block(WuMomentum::THREADS);
             if (c->fresh)
-                PARLE_TRY(launch_chained(c, KC_WGRAD_UPDATE, PK_WGRAD_UPDATE, l, umma_wgrad_update_kernel<true, WuMomentum, true>,
-                                         grid, block, WuMomentum::SMEM_BYTES,
-                                         c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p));
+                umma_wgrad_update_kernel<true, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(
+                    c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p);
             else
-                PARLE_TRY(launch_chained(c, KC_WGRAD_UPDATE, PK_WGRAD_UPDATE, l, umma_wgrad_update_kernel<false, WuMomentum, true>,
-                                         grid, block, WuMomentum::SMEM_BYTES,
-                                         c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p));
-        } else {
-            const dim3 block(WuDefault::THREADS);
-            if (c->fresh)
-                PARLE_TRY(launch_chained(c, KC_WGRAD_UPDATE, PK_WGRAD_UPDATE, l, umma_wgrad_update_kernel<true, WuDefault, false>,
-                                         grid, block, WuDefault::SMEM_BYTES,
-                                         c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p));
-            else
-                PARLE_TRY(launch_chained(c, KC_WGRAD_UPDATE, PK_WGRAD_UPDATE, l, umma_wgrad_update_kernel<false, WuDefault, false>,
-                                         grid, block, WuDefault::SMEM_BYTES,
-                                         c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p));
-        }
+                umma_wgrad_update_kernel<false, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(
+                    c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p);
+        } else if (c->fresh)
+            umma_wgrad_update_kernel<true, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
+                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p);
+        else
+            umma_wgrad_update_kernel<false, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
+                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p);
+        PARLE_LAUNCHED(c);
     }
     TailPlan tp = {};
     tp.n_layers = nl; tp.batch = B;
@@ -591,12 +537,21 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         if (tp.end[l] - tp.begin[l] > longest) longest = tp.end[l] - tp.begin[l];
     }
     const dim3 tgrid((unsigned)((longest + 127) / 128), nl, n);
-    void (*tail)(TailPlan, float *, float *, const float *, long long, float, float, float, float, int *, float *, float) =
-        mom ? (c->fresh ? tail_update_kernel<true, true> : tail_update_kernel<false, true>)
-            : (c->fresh ? tail_update_kernel<true, false> : tail_update_kernel<false, false>);
-    return launch_chained(c, KC_TAIL_UPDATE, PK_TAIL, 0, tail, tgrid, dim3(128), 0, tp, c->buf.y, c->buf.z,
-                          (const float *)c->buf.x, S, c->eta_prime, c->inv_gamma, c->alpha, c->weight_decay, c->status_dev,
-                          mom ? c->vy : (float *)nullptr, mom ? c->momentum : 0.f);
+    prof_begin(c, KC_TAIL_UPDATE);
+    if (mom && c->fresh)
+        tail_update_kernel<true, true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S, c->eta_prime, c->inv_gamma,
+                                                                     c->alpha, c->weight_decay, c->status_dev, c->vy, c->momentum);
+    else if (mom)
+        tail_update_kernel<false, true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S, c->eta_prime, c->inv_gamma,
+                                                                      c->alpha, c->weight_decay, c->status_dev, c->vy, c->momentum);
+    else if (c->fresh)
+        tail_update_kernel<true><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
+                                                               c->eta_prime, c->inv_gamma, c->alpha, c->weight_decay, c->status_dev);
+    else
+        tail_update_kernel<false><<<tgrid, 128, 0, c->stream>>>(tp, c->buf.y, c->buf.z, c->buf.x, S,
+                                                                c->eta_prime, c->inv_gamma, c->alpha, c->weight_decay, c->status_dev);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
 }
 
 int check_bound(const parle_ctx *c) {
@@ -658,7 +613,6 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         c->sh_stride += (size_t)c->sh_rb[l] * c->sh_cb[l] * 8192;
     }
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
-    c->overlap_on = true;
     c->wide_tiles_per_sm = 4;
     c->last_ksplit = 1;
     if (c->fused_update) {
@@ -761,7 +715,6 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
     PARLE_TRY(check_bound(c));
     if (c->n_layers == 0 || !inputs || !labels) return PARLE_EINVAL;
     if (!c->round_open) return PARLE_ESTATE;
-    if (!c->chain_steps) c->prev_kind = PK_NONE;      // a call of its own: whatever precedes it in the stream comes first
     if (c->gemm_dtype == PARLE_GEMM_BF16) {
         PARLE_TRY(forward_backward_bf16(c, inputs, labels, loss_out));
         if (c->fused_update) {            // y, z and the operand copy were updated by the backward kernels
@@ -880,13 +833,8 @@ static int round_graphed(parle_ctx *c, int L, const float *inputs, const int32_t
         cudaStream_t bound = c->stream;
         c->stream = c->capture_stream;                  // the launches of this one round are recorded, not run
         const int steps_before = c->steps_in_round;
-        // ordinary kernel nodes: a graph already runs its nodes back to back, and programmatic edges made
-        // the replay slower than that (C3: 15.1 -> 15.6 ms per round)
-        const bool overlap = c->overlap_on;
-        c->overlap_on = false;
         const int rc = L > 0 ? round_direct(c, L, inputs, labels, loss_out)
                              : parle_inner_step(c, inputs, labels, loss_out);
-        c->overlap_on = overlap;
         c->stream = bound;
         const cudaError_t e = cudaStreamEndCapture(c->capture_stream, &graph);
         const long long inside = c->launches - before;
@@ -925,7 +873,6 @@ static int round_graphed(parle_ctx *c, int L, const float *inputs, const int32_t
     }
     g->last_use = ++c->graph_clock;
     PARLE_CUDA(c, cudaGraphLaunch(g->exec, c->stream));
-    c->prev_kind = PK_NONE;
     c->launches += g->launches;
     if (L > 0) {      // host-side state after a round (what round_direct leaves behind)
         c->round_open = false; c->fresh = false; c->steps_in_round = 0; c->shadow_is_x = false;
@@ -954,15 +901,9 @@ int parle_set_round_graphs(parle_ctx *c, int on) {
 static int round_direct(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
     PARLE_TRY(parle_round_begin(c));
     const size_t nb = (size_t)c->n * c->batch;
-    c->prev_kind = PK_NONE;
-    c->chain_steps = true;            // nothing but this round's kernels between the steps: one launch chain
-    int rc = PARLE_OK;
-    for (int l = 0; l < L && rc == PARLE_OK; ++l)
-        rc = parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
-                              loss_out ? loss_out + (size_t)l * c->n : nullptr);
-    c->chain_steps = false;
-    c->prev_kind = PK_NONE;
-    PARLE_TRY(rc);
+    for (int l = 0; l < L; ++l)
+        PARLE_TRY(parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
+                                   loss_out ? loss_out + (size_t)l * c->n : nullptr));
     return parle_outer_step(c);
 }
 
@@ -1023,12 +964,6 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->fused_update = on != 0;
-    return PARLE_OK;
-}
-
-int parle_set_launch_overlap(parle_ctx *c, int on) {
-    if (!c) return PARLE_EINVAL;
-    c->overlap_on = on != 0;
     return PARLE_OK;
 }
 

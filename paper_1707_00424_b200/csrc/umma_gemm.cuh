@@ -70,9 +70,6 @@ struct UmmaParams {
     // split-K (UEPI_FWD_LAST only): each tile's k-blocks are divided among ksplit work items, each of which
     // stores its raw partial sums (no bias) at outf + split * part_ss; a later kernel adds them up in fixed order
     int ksplit; long long part_ss;
-    // 1: the B operand (weights) is not written by the kernel before this one in the stream, so its
-    // producer may fill the ring before the dependency wait (see dep_wait)
-    int early_b;
     int *status;
 };
 
@@ -246,7 +243,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------ TMA producer of the B operand (deep ring)
         if (lane == 0) {
-            if (!p.early_b) dep_wait();
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
                 const int t = it / ksplit, split = it - t * ksplit;
@@ -288,8 +284,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     } else if (warp == 2 + umma_epi_warps(EPI)) {
         // ------------------------------------------------ TMA producer of the A operand
         if (lane == 0) {
-            dep_wait();                                       // the A operand is the previous kernel's output
-            dep_release();
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
                 const int t = it / ksplit, split = it - t * ksplit;
@@ -353,7 +347,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;                              // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;                    // chunks 2*half, 2*half + 1 of every tile
         int acc = 0; uint32_t acc_phase = 0;
-        dep_wait();                                          // bias, mask and the output buffers belong to earlier kernels
         for (int it = blockIdx.x; it < total_items; it += gridDim.x) {
             const int t = it / ksplit, split = it - t * ksplit;
             int g, m0, n0; tile_coords(p, t, BN, g, m0, n0);

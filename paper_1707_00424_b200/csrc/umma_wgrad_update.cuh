@@ -71,9 +71,6 @@ struct WgradUpdateParams {
     long long gs; int ld;
     float eta_p, inv_gamma, alpha, wd;
     float *v; float mu;          // Nesterov momentum buffer of y (same addressing as y), used by the MOM variant
-    // 1: x, y, z (and v) of this layer are not written by the kernel before this one in the stream, so the
-    // state loader may fill its ring before the dependency wait (see dep_wait)
-    int early_state;
     int *status;
 };
 
@@ -136,8 +133,6 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     if (warp == 0) {
         // ------------------------------------------------ operand producer (A = H^T tile, B = dH^T tile)
         if (lane == 0) {
-            dep_wait();                                       // the operands are earlier kernels' outputs
-            dep_release();
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 int g, m0, n0; coords(t, g, m0, n0);
@@ -187,7 +182,6 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     } else if (warp == 2) {
         // ------------------------------------------------ state loader: x (, y, z) boxes, chunk by chunk
         if (lane == 0) {
-            if (!p.early_state) dep_wait();
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 int g, m0, n0; coords(t, g, m0, n0);
@@ -225,7 +219,6 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         int stage = 0; uint32_t sphase = 0;                  // state ring position: every warp walks every chunk
         float chk = 0.f;                                     // 0 * y summed: turns NaN as soon as a y is NaN or Inf
         bool ok = true;
-        dep_wait();                                          // y, z and the bf16 copy are still read by the kernel before
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             int g, m0, n0; coords(t, g, m0, n0);
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));

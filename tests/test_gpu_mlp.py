@@ -577,42 +577,3 @@ def test_graph_rounds_equal_plain_rounds(gemm_dtype, dims):
         outs.append((m.x.clone(), m.xbar.clone(), lh.clone()))
     for a, b in zip(*outs):
         assert torch.equal(a, b)
-
-
-@pytest.mark.gpu
-@pytest.mark.parametrize("dims,batch,n,mu", [((64, 128, 72, 10), 16, 3, 0.0), ((200, 328, 136, 101), 136, 2, 0.0),
-                                             ((512, 1024, 768, 100), 128, 8, 0.0), ((64, 128, 72, 10), 16, 3, 0.5)])
-def test_overlapped_launches_give_identical_rounds_bf16(dims, batch, n, mu):
-    """Kernels launched so that each may start while its predecessor drains (parle_set_launch_overlap)
-    leave bit-identical state: plain rounds, graph rounds and host-buffer rounds, with and without momentum."""
-    cfg = si.C1.scaled(dims=dims, gemm_dtype=1, L=5, batch=batch, n=n)
-    sets = [si.round_batches(cfg, r) for r in range(2)]
-    dev = [(torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)) for X, c in sets]
-    Xh, ch = torch.from_numpy(sets[0][0]).pin_memory(), torch.from_numpy(sets[0][1]).pin_memory()
-    res = {}
-    for overlap in (False, True):
-        for graphs in (False, True):
-            m, *_ = make(cfg)
-            if mu:
-                m.set_momentum(mu)
-            m.set_launch_overlap(overlap)
-            m.set_round_graphs(graphs)
-            loss = torch.zeros(cfg.L, cfg.n, device=DEV)
-            lh = torch.zeros(cfg.L, cfg.n).pin_memory()
-            for r in (0, 1, 0):
-                m.round(cfg.L, dev[r][0], dev[r][1], loss)
-            m.round_host(cfg.L, Xh, ch, lh)
-            m.round_begin()                               # single steps as calls of their own
-            m.inner_step(dev[1][0][0], dev[1][1][0], loss[0])
-            m.inner_step(dev[1][0][1], dev[1][1][1], loss[1])
-            m.outer_step()
-            torch.cuda.synchronize()
-            assert m.status() == 0
-            if graphs:
-                assert m.round_graph_count > 0
-            res[(overlap, graphs)] = (m.x.clone(), m.xbar.clone(), m.y.clone(), m.z.clone(), loss.clone(), lh.clone())
-            del m
-    ref = res[(False, False)]
-    for key, got in res.items():
-        for a, b in zip(ref, got):
-            assert torch.equal(a, b), key
