@@ -82,6 +82,150 @@ __global__ void __launch_bounds__(SG_THREADS) simt_gemm_kernel(SimtGemmArgs p) {
     }
 }
 
+// ---------------------------------------------------------------- register-tiled SGEMM (larger problems)
+// Same product, same epilogues and the same summation order (every output sums its K products in
+// ascending k with one fused multiply-add each, so results are bit-identical to simt_gemm_kernel),
+// but 8 x 8 outputs per thread, 16-byte shared-memory reads that a half-warp makes from one
+// contiguous run, 16-byte global loads where the operand's layout allows, and the next k-block
+// fetched into registers while the current one is multiplied (two shared-memory buffers, one
+// barrier per k-block).  The FMA pipes are the bound: 64 FMAs per 4 shared-memory reads.
+constexpr int ST_BK = 16;
+
+// One operand tile X(r, k) = X[r * rs + k * ks], rows r0 .. r0 + ROWS - 1, k-block k0 .. k0 + 15,
+// as ROWS * 16 / 4 four-element units dealt round-robin to the threads.  A unit runs along k when
+// ks == 1 ("k-fast": activations, W in the forward product) and along r otherwise.
+template <int ROWS, int THREADS>
+struct OperandTile {
+    static constexpr int UNITS = ROWS * ST_BK / 4, PER_THREAD = UNITS / THREADS;
+    static_assert(UNITS % THREADS == 0, "units per thread");
+    const float *X; long long rs, ks; int R, K, r0; bool kfast, vec;
+
+    __device__ __forceinline__ void init(const float *X_, long long rs_, long long ks_, int R_, int K_, int r0_) {
+        X = X_; rs = rs_; ks = ks_; R = R_; K = K_; r0 = r0_;
+        kfast = (ks == 1);
+        // 16-byte loads need the unit's first element 16-byte aligned for every (r, k) it can start at
+        const long long slow = kfast ? rs : ks;
+        vec = (kfast || rs == 1) && (slow % 4 == 0) && (reinterpret_cast<uintptr_t>(X) % 16 == 0);
+    }
+    __device__ __forceinline__ void fetch(int k0, float4 (&reg)[PER_THREAD]) const {
+#pragma unroll
+        for (int i = 0; i < PER_THREAD; ++i) {
+            const int u = threadIdx.x + i * THREADS;
+            int rr, kk;                                   // first element of the unit inside the tile
+            if (kfast) { rr = u / (ST_BK / 4); kk = (u % (ST_BK / 4)) * 4; }
+            else       { kk = u / (ROWS / 4);  rr = (u % (ROWS / 4)) * 4; }
+            const int r = r0 + rr, k = k0 + kk;
+            const int last_r = kfast ? r : r + 3, last_k = kfast ? k + 3 : k;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (vec && last_r < R && last_k < K) {
+                v = *reinterpret_cast<const float4 *>(X + (long long)r * rs + (long long)k * ks);
+            } else {
+                float e[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int rj = kfast ? r : r + j, kj = kfast ? k + j : k;
+                    e[j] = (rj < R && kj < K) ? X[(long long)rj * rs + (long long)kj * ks] : 0.f;
+                }
+                v = make_float4(e[0], e[1], e[2], e[3]);
+            }
+            reg[i] = v;
+        }
+    }
+    // shared-memory tile: Xs[k][r], row pitch ROWS + 4 floats
+    __device__ __forceinline__ void stash(float (*Xs)[ROWS + 4], const float4 (&reg)[PER_THREAD]) const {
+#pragma unroll
+        for (int i = 0; i < PER_THREAD; ++i) {
+            const int u = threadIdx.x + i * THREADS;
+            if (kfast) {
+                const int rr = u / (ST_BK / 4), kk = (u % (ST_BK / 4)) * 4;
+                Xs[kk + 0][rr] = reg[i].x; Xs[kk + 1][rr] = reg[i].y; Xs[kk + 2][rr] = reg[i].z; Xs[kk + 3][rr] = reg[i].w;
+            } else {
+                const int kk = u / (ROWS / 4), rr = (u % (ROWS / 4)) * 4;
+                *reinterpret_cast<float4 *>(&Xs[kk][rr]) = reg[i];
+            }
+        }
+    }
+};
+
+// C[g] = A[g] * B[g], tile BM x BN per CTA, (BM/8) x (BN/8) threads.  A thread owns rows
+// ty*4 .. +3 and BM/2 + ty*4 .. +3, columns tx*4 .. +3 and BN/2 + tx*4 .. +3 of the tile.
+template <int EPI, int BM, int BN>
+__global__ void __launch_bounds__((BM / 8) * (BN / 8)) simt_gemm_tiled_kernel(SimtGemmArgs p) {
+    constexpr int TX = BN / 8, THREADS = (BM / 8) * (BN / 8);
+    __shared__ __align__(16) float As[2][ST_BK][BM + 4];
+    __shared__ __align__(16) float Bs[2][ST_BK][BN + 4];
+    const int g = blockIdx.z;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int tx = threadIdx.x % TX, ty = threadIdx.x / TX;
+    OperandTile<BM, THREADS> ta;
+    OperandTile<BN, THREADS> tb;
+    ta.init(p.A + (long long)g * p.a_gs, p.a_ms, p.a_ks, p.M, p.K, m0);
+    tb.init(p.B + (long long)g * p.b_gs, p.b_ns, p.b_ks, p.N, p.K, n0);
+    float4 ra[OperandTile<BM, THREADS>::PER_THREAD], rb[OperandTile<BN, THREADS>::PER_THREAD];
+    float acc[8][8] = {};
+
+    ta.fetch(0, ra); tb.fetch(0, rb);
+    ta.stash(As[0], ra); tb.stash(Bs[0], rb);
+    __syncthreads();
+    int cur = 0;
+    for (int k0 = 0; k0 < p.K; k0 += ST_BK) {
+        const bool more = k0 + ST_BK < p.K;
+        if (more) { ta.fetch(k0 + ST_BK, ra); tb.fetch(k0 + ST_BK, rb); }
+#pragma unroll
+        for (int kk = 0; kk < ST_BK; ++kk) {
+            const float4 a0 = *reinterpret_cast<const float4 *>(&As[cur][kk][ty * 4]);
+            const float4 a1 = *reinterpret_cast<const float4 *>(&As[cur][kk][BM / 2 + ty * 4]);
+            const float4 b0 = *reinterpret_cast<const float4 *>(&Bs[cur][kk][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4 *>(&Bs[cur][kk][BN / 2 + tx * 4]);
+            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        if (more) {
+            // the other buffer was last read in the previous iteration, which ended with a barrier
+            ta.stash(As[cur ^ 1], ra); tb.stash(Bs[cur ^ 1], rb);
+            __syncthreads();
+            cur ^= 1;
+        }
+    }
+
+    float *C = p.C + (long long)g * p.c_gs;
+    const float *bias = (EPI == EPI_BIAS || EPI == EPI_BIAS_RELU) ? p.bias + (long long)g * p.bias_gs : nullptr;
+    const float *mask = (EPI == EPI_MASK) ? p.mask + (long long)g * p.mask_gs : nullptr;
+    const bool c_vec = (p.ldc % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int m = m0 + (i < 4 ? ty * 4 + i : BM / 2 + ty * 4 + i - 4);
+        if (m >= p.M) continue;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int n = n0 + (h ? BN / 2 : 0) + tx * 4;
+            if (n >= p.N) continue;
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                v[j] = acc[i][h * 4 + j];
+                if (n + j < p.N) {
+                    if (EPI == EPI_BIAS || EPI == EPI_BIAS_RELU) v[j] += bias[n + j];
+                    if (EPI == EPI_BIAS_RELU) v[j] = fmaxf(v[j], 0.f);
+                    if (EPI == EPI_MASK) v[j] = (mask[(long long)m * p.ldmask + n + j] > 0.f) ? v[j] : 0.f;
+                }
+            }
+            float *o = C + (long long)m * p.ldc + n;
+            if (c_vec && n + 3 < p.N) {
+                *reinterpret_cast<float4 *>(o) = make_float4(v[0], v[1], v[2], v[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (n + j < p.N) o[j] = v[j];
+            }
+        }
+    }
+}
+
 // Softmax cross-entropy backward, one warp per batch row:
 //   p = softmax(logits) (row max subtracted), dlogits = (p - onehot)/B,
 //   row_loss = logsumexp - logits[label].

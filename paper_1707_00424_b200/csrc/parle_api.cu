@@ -310,11 +310,23 @@ cudaError_t allow_big_smem() {
                                 (int)UM_SMEM_BYTES);
 }
 
+// fp32 product: the largest register tile (8 x 8 outputs per thread) that still gives (nearly) every SM a
+// CTA; small problems get 64 x 64 tiles with 4 x 4 outputs per thread (more warps per output).
 template <int EPI>
 int launch_simt(parle_ctx *c, int cls, const SimtGemmArgs &a) {
-    dim3 grid((a.N + SG_BN - 1) / SG_BN, (a.M + SG_BM - 1) / SG_BM, c->n);
+    auto ctas = [&](int bm, int bn) { return (long long)((a.M + bm - 1) / bm) * ((a.N + bn - 1) / bn) * c->n; };
+    const long long want = (long long)c->sm_count * 85 / 100;
     prof_begin(c, cls);
-    simt_gemm_kernel<EPI><<<grid, SG_THREADS, 0, c->stream>>>(a);
+    if (ctas(128, 128) >= want) {
+        dim3 grid((a.N + 127) / 128, (a.M + 127) / 128, c->n);
+        simt_gemm_tiled_kernel<EPI, 128, 128><<<grid, 256, 0, c->stream>>>(a);
+    } else if (ctas(128, 64) >= want) {
+        dim3 grid((a.N + 63) / 64, (a.M + 127) / 128, c->n);
+        simt_gemm_tiled_kernel<EPI, 128, 64><<<grid, 128, 0, c->stream>>>(a);
+    } else {
+        dim3 grid((a.N + SG_BN - 1) / SG_BN, (a.M + SG_BM - 1) / SG_BM, c->n);
+        simt_gemm_kernel<EPI><<<grid, SG_THREADS, 0, c->stream>>>(a);
+    }
     PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
