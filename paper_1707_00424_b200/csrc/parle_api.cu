@@ -36,6 +36,7 @@ struct Workspace {
     size_t dhb[PARLE_MAX_LAYERS], dhbT[PARLE_MAX_LAYERS];    // their gradients, both layouts
     int dh_ld[PARLE_MAX_LAYERS];       // row pitch of dhb[l] (d_{l+1} rounded up to 8)
     size_t row_loss;                   // [n,B] fp32
+    size_t sched;                      // bf16 mode: two ints, the tile counters of the fused weight-gradient kernel (zero between launches)
     size_t stage_in[2], stage_lab[2], stage_loss[2];   // double-buffered staging for the host-buffer entry points
     size_t total;
 };
@@ -161,6 +162,7 @@ void plan_workspace(parle_ctx *c) {
             w.dhb[l] = take(n * B * w.dh_ld[l] * 2);
             w.dhbT[l] = take(n * B * c->dims[l + 1] * 2);
         }
+        w.sched = take(2 * sizeof(int));
     }
     w.row_loss = take(n * B * sizeof(float));
     for (int b = 0; b < 2; ++b) {
@@ -518,6 +520,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         p.gs = S; p.ld = din;
         p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha; p.wd = c->weight_decay;
         p.status = c->status_dev;
+        p.sched = ws_ptr<int>(c, w.sched);
         const int tiles = p.groups * p.tiles_m * p.tiles_n;
         const int grid = tiles < c->sm_count ? tiles : c->sm_count;
         prof_begin(c, KC_WGRAD_UPDATE);
@@ -707,6 +710,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_TRY(build_tensor_maps(c));
         // rows / columns of the blocked weight copy beyond the matrices are never written: they must read as zero
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.shadow), 0, (size_t)c->n * c->sh_stride * 2, c->stream));
+        // tile counters of the fused weight-gradient kernel: every launch leaves them at zero again
+        PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.sched), 0, 2 * sizeof(int), c->stream));
     }
     c->bound = true;
     c->round_open = false; c->fresh = false; c->shadow_is_x = false; c->steps_in_round = 0;

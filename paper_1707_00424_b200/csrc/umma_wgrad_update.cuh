@@ -23,6 +23,16 @@
 // memory).  Every epilogue warp consumes every chunk, in order -- group g takes
 // its own slice of the chunk's rows -- so each stage barrier sees all its
 // consumers in every phase and no waiter can fall a phase behind.
+//
+// Tiles are handed out dynamically.  SMs do not get equal shares of a saturated
+// memory system (with a fixed tile list per CTA the first CTA of a 2048 x 2048
+// layer finished after 85 us and the last after 120 us), so after its first tile
+// (blockIdx.x) a CTA claims the next one from a global counter.  The operand
+// producer is the scheduler: it publishes every claimed tile index (or -1: no
+// tiles left) through a small shared-memory ring with full/empty barriers, and
+// the other roles read it from there.  The last CTA to leave resets the counter
+// pair, so consecutive launches on one stream can share it.  Which CTA runs a
+// tile does not change what is computed for it: results stay bit-identical.
 // All waits are bounded.
 #pragma once
 
@@ -32,6 +42,8 @@ namespace parle {
 
 constexpr int WU_OP_STAGES = 2;                                // operand ring (K = batch is short)
 constexpr int WU_STATE_RING_BYTES = 144 * 1024;                // shared memory given to the x/y/z stages
+constexpr int WU_TILE_SLOTS = 4;                               // depth of the tile-index ring
+constexpr int WU_CTL_BYTES = 512;                              // barriers, tile ring, tensor-memory slot, abort flag
 
 // Shape of the epilogue: G groups of 4 warps share chunks of CR W-rows (accumulator columns);
 // every thread owns CR / G rows of one column.
@@ -44,9 +56,10 @@ struct WuShape {
     static constexpr int STAGES = WU_STATE_RING_BYTES / STATE_BYTES;
     static constexpr int THREADS = 96 + 128 * G;
     static constexpr size_t SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)STAGES * STATE_BYTES +
-                                         1024 /*alignment slack*/ + 256 /*barriers*/;
+                                         1024 /*alignment slack*/ + WU_CTL_BYTES;
     static_assert(RPG == 4 || RPG == 8 || RPG == 16, "rows per thread must match a tcgen05.ld shape");
-    static_assert(STAGES >= 2 && 2 * WU_OP_STAGES + 4 + 2 * STAGES <= 30, "stage count");
+    static_assert(STAGES >= 2 && 8 * (2 * WU_OP_STAGES + 4 + 2 * STAGES + 2 * WU_TILE_SLOTS) + 8 + 4 * WU_TILE_SLOTS <= WU_CTL_BYTES,
+                  "stage count");
 };
 using WuDefault = WuShape<4, 32>;
 using WuMomentum = WuShape<4, 16, 4>;                          // with the momentum buffer staged too: 16-row chunks
@@ -71,6 +84,7 @@ struct WgradUpdateParams {
     long long gs; int ld;
     float eta_p, inv_gamma, alpha, wd;
     float *v; float mu;          // Nesterov momentum buffer of y (same addressing as y), used by the MOM variant
+    int *sched;                  // sched[0]: tiles claimed beyond the first of every CTA, sched[1]: CTAs that have left; both 0 between launches
     int *status;
 };
 
@@ -91,14 +105,16 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     const uint32_t st_base = op_base + WU_OP_STAGES * UM_STAGE_BYTES;
     uint8_t *st_ptr = smem_raw + (st_base - raw);
     uint8_t *ctl = st_ptr + (size_t)WU_STATE_STAGES * WU_STATE_BYTES;
-    // barriers: op_full[2], op_empty[2], tfull[2], tempty[2], st_full[S], st_empty[S]
+    // barriers: op_full[2], op_empty[2], tfull[2], tempty[2], st_full[S], st_empty[S], tile_full[T], tile_empty[T]
     uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);
-    constexpr int NBARS = 2 * WU_OP_STAGES + 4 + 2 * WU_STATE_STAGES;
+    constexpr int NBARS = 2 * WU_OP_STAGES + 4 + 2 * WU_STATE_STAGES + 2 * WU_TILE_SLOTS;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * NBARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    volatile int *tile_ids = reinterpret_cast<volatile int *>(tmem_slot + 2);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * WU_OP_STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * WU_OP_STAGES, bar_tempty = bar_tfull + 16;
     const uint32_t bar_sfull = bar_tempty + 16, bar_sempty = bar_sfull + 8 * WU_STATE_STAGES;
+    const uint32_t bar_qfull = bar_sempty + 8 * WU_STATE_STAGES, bar_qempty = bar_qfull + 8 * WU_TILE_SLOTS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.groups * p.tiles_m * p.tiles_n;
@@ -109,6 +125,8 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         for (int s = 0; s < WU_OP_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, 4 * WU_GROUPS); }
         for (int s = 0; s < WU_STATE_STAGES; ++s) { mbar_init(bar_sfull + 8 * s, 1); mbar_init(bar_sempty + 8 * s, 4 * WU_GROUPS); }
+        // a tile index is read by the MMA issuer, the state loader and every epilogue warp
+        for (int s = 0; s < WU_TILE_SLOTS; ++s) { mbar_init(bar_qfull + 8 * s, 1); mbar_init(bar_qempty + 8 * s, 2 + 4 * WU_GROUPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -129,12 +147,29 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         m0 = (r % p.tiles_m) * UM_BM;
         n0 = (r / p.tiles_m) * UM_BN;
     };
+    // Consumer side of the tile ring (one lane per role calls it): the next tile of this CTA, -1 when there is
+    // none, -2 when a wait gave up.
+    auto take_tile = [&](int &slot, uint32_t &ph) -> int {
+        if (!mbar_wait(bar_qfull + 8 * slot, ph, abort_flag)) return -2;
+        const int t = tile_ids[slot];
+        mbar_arrive(bar_qempty + 8 * slot);
+        if (++slot == WU_TILE_SLOTS) { slot = 0; ph ^= 1u; }
+        return t;
+    };
 
     if (warp == 0) {
-        // ------------------------------------------------ operand producer (A = H^T tile, B = dH^T tile)
+        // ------------------------------------------------ tile scheduler + operand producer (A = H^T tile, B = dH^T tile)
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            int qslot = 0; uint32_t qphase = 0;
+            int t = blockIdx.x;                                               // the first tile needs no claim
+            int t_next = (int)gridDim.x + atomicAdd(p.sched, 1);              // claimed one tile ahead: its latency is hidden
+            while (ok) {
+                if (!mbar_wait(bar_qempty + 8 * qslot, qphase ^ 1u, abort_flag)) { ok = false; break; }
+                tile_ids[qslot] = t < total_tiles ? t : -1;
+                mbar_arrive(bar_qfull + 8 * qslot);                           // release: the index is visible to the waiters
+                if (++qslot == WU_TILE_SLOTS) { qslot = 0; qphase ^= 1u; }
+                if (t >= total_tiles) break;
                 int g, m0, n0; coords(t, g, m0, n0);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -145,6 +180,8 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     tma_load_3d(sb, &tmB, fb, kb * UM_BK, n0, g);
                     if (++stage == WU_OP_STAGES) { stage = 0; phase ^= 1u; }
                 }
+                t = t_next;
+                if (t < total_tiles) t_next = (int)gridDim.x + atomicAdd(p.sched, 1);
             }
             if (!ok) {
                 for (int s = 0; s < WU_OP_STAGES; ++s) {
@@ -159,7 +196,8 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(false, false);
             int stage = 0; uint32_t phase = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            int qslot = 0; uint32_t qphase = 0;
+            while (ok && take_tile(qslot, qphase) >= 0) {
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * UM_BN;
@@ -183,7 +221,8 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // ------------------------------------------------ state loader: x (, y, z) boxes, chunk by chunk
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            int qslot = 0; uint32_t qphase = 0;
+            for (int t; ok && (t = take_tile(qslot, qphase)) >= 0;) {
                 int g, m0, n0; coords(t, g, m0, n0);
                 for (int c = 0; c < WU_CHUNKS; ++c) {
                     const int nb = n0 + c * WU_CHUNK_ROWS;
@@ -219,7 +258,15 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         int stage = 0; uint32_t sphase = 0;                  // state ring position: every warp walks every chunk
         float chk = 0.f;                                     // 0 * y summed: turns NaN as soon as a y is NaN or Inf
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int qslot = 0; uint32_t qphase = 0;
+        while (ok) {
+            // every lane waits for the tile index and reads it; lane 0 hands the slot back for the warp
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_qfull + 8 * qslot, qphase, abort_flag))) break;
+            const int t = tile_ids[qslot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_qempty + 8 * qslot);
+            if (++qslot == WU_TILE_SLOTS) { qslot = 0; qphase ^= 1u; }
+            if (t < 0) break;
             int g, m0, n0; coords(t, g, m0, n0);
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
@@ -307,6 +354,15 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && *abort_flag) p.status[SLOT_WAIT_LIMIT] = 1;
+    if (threadIdx.x == 0) {
+        // all claims of this CTA are done; the last CTA to leave puts both counters back to zero for the next launch
+        __threadfence();
+        if (atomicAdd(p.sched + 1, 1) == (int)gridDim.x - 1) {
+            __threadfence();
+            p.sched[0] = 0;
+            p.sched[1] = 0;
+        }
+    }
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem_base), "r"((uint32_t)UM_TMEM_COLS) : "memory");
