@@ -87,8 +87,8 @@ struct parle_ctx {
     CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
-    CUtensorMap tm_sx[PARLE_MAX_LAYERS], tm_sy[PARLE_MAX_LAYERS], tm_sz[PARLE_MAX_LAYERS];   // fp32 W_l segments of x, y, z
-    CUtensorMap tm_mx[PARLE_MAX_LAYERS], tm_my[PARLE_MAX_LAYERS], tm_mz[PARLE_MAX_LAYERS], tm_mv[PARLE_MAX_LAYERS];   // same + vy, 16-row boxes (momentum variant)
+    WuMaps wu_maps;                  // fused weight-gradient kernel: operands + fp32 W_l segments of x, y, z (32-row boxes)
+    WuMaps wu_maps_mom;              // its momentum variant: same + vy, 16-row boxes
     bool mom_maps;
     // parle_round as a CUDA graph (optional): a small cache of instantiated rounds
     bool graphs_on;
@@ -264,9 +264,11 @@ int build_tensor_maps(parle_ctx *c) {
         PARLE_TRY(encode_bf16_map(c, &c->tm_wg_b[l], ws_ptr<__nv_bfloat16>(c, w.dhbT[l]), B, dout, n, B, dout * B, UM_BK, UM_BN));
         // fused update: the W_l segments of x, y, z as [n][dout][din] fp32, fetched in 16-row x 128-column boxes
         const size_t wo = c->layers[l].w_off;
-        PARLE_TRY(encode_f32_map(c, &c->tm_sx[l], c->buf.x + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
-        PARLE_TRY(encode_f32_map(c, &c->tm_sy[l], c->buf.y + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
-        PARLE_TRY(encode_f32_map(c, &c->tm_sz[l], c->buf.z + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
+        PARLE_TRY(encode_f32_map(c, &c->wu_maps.x[l], c->buf.x + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
+        PARLE_TRY(encode_f32_map(c, &c->wu_maps.y[l], c->buf.y + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
+        PARLE_TRY(encode_f32_map(c, &c->wu_maps.z[l], c->buf.z + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
+        c->wu_maps.v[l] = c->wu_maps.z[l];                                   // not read without momentum
+        c->wu_maps.a[l] = c->tm_wg_a[l]; c->wu_maps.b[l] = c->tm_wg_b[l];
         if (l > 0) {
             // data gradient: A = dH [B, dout] K-major (K = dout); B = W [dout (K), din (N)] MN-major,
             // fetched as 64 k-rows x 64 n-columns boxes
@@ -505,41 +507,42 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         }
         return PARLE_OK;
     }
-    // Fused: the weight gradient never reaches memory.  dgrad(l) must read W_l before the fused
-    // kernel of layer l overwrites its bf16 copy, so it goes first.
-    __nv_bfloat16 *shadow = ws_ptr<__nv_bfloat16>(c, w.shadow);
-    for (int l = nl - 1; l >= 0; --l) {
-        const int din = c->dims[l], dout = c->dims[l + 1];
-        if (l > 0) PARLE_TRY(dgrad(l));
-        WgradUpdateParams p = {};
-        p.M = din; p.N = dout; p.K = B;
-        p.groups = n; p.tiles_m = (din + UM_BM - 1) / UM_BM; p.tiles_n = (dout + UM_BN - 1) / UM_BN;
-        const size_t wo = c->layers[l].w_off;
-        p.y = c->buf.y + wo; p.z = c->buf.z + wo;
-        p.shadow = shadow + c->sh_off[l]; p.shadow_gs = (long long)c->sh_stride; p.shadow_cb = c->sh_cb[l];
-        p.gs = S; p.ld = din;
-        p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha; p.wd = c->weight_decay;
-        p.status = c->status_dev;
-        p.sched = ws_ptr<int>(c, w.sched);
-        const int tiles = p.groups * p.tiles_m * p.tiles_n;
-        const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-        prof_begin(c, KC_WGRAD_UPDATE);
-        if (mom) {
-            p.v = c->vy + wo; p.mu = c->momentum;
-            if (c->fresh)
-                umma_wgrad_update_kernel<true, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(
-                    c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p);
-            else
-                umma_wgrad_update_kernel<false, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(
-                    c->tm_wg_a[l], c->tm_wg_b[l], c->tm_mx[l], c->tm_my[l], c->tm_mz[l], c->tm_mv[l], p);
-        } else if (c->fresh)
-            umma_wgrad_update_kernel<true, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
-                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p);
-        else
-            umma_wgrad_update_kernel<false, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(
-                c->tm_wg_a[l], c->tm_wg_b[l], c->tm_sx[l], c->tm_sy[l], c->tm_sz[l], c->tm_sz[l], p);
-        PARLE_LAUNCHED(c);
+    // Fused: the weight gradient never reaches memory.  All data-gradient products go first (they read the bf16
+    // weight copies that the fused kernel overwrites); then ONE launch of the fused kernel walks the W tiles of
+    // every layer, so the stream of x, y, z through the SMs starts up and drains once per step, not once per layer.
+    for (int l = nl - 1; l > 0; --l) PARLE_TRY(dgrad(l));
+    WgradUpdateParams p = {};
+    p.K = B; p.groups = n; p.n_layers = nl;
+    int tiles = 0;
+    for (int l = 0; l < nl; ++l) {
+        WuLayer &ly = p.layer[l];
+        ly.M = c->dims[l]; ly.N = c->dims[l + 1];
+        ly.tiles_m = (ly.M + UM_BM - 1) / UM_BM; ly.tiles_n = (ly.N + UM_BN - 1) / UM_BN;
+        ly.tile_begin = tiles;
+        tiles += n * ly.tiles_m * ly.tiles_n;
+        ly.ld = ly.M; ly.shadow_cb = c->sh_cb[l];
+        ly.w_off = (long long)c->layers[l].w_off; ly.shadow_off = (long long)c->sh_off[l];
     }
+    p.total_tiles = tiles;
+    p.y = c->buf.y; p.z = c->buf.z;
+    p.shadow = ws_ptr<__nv_bfloat16>(c, w.shadow); p.shadow_gs = (long long)c->sh_stride;
+    p.gs = S;
+    p.eta_p = c->eta_prime; p.inv_gamma = c->inv_gamma; p.alpha = c->alpha; p.wd = c->weight_decay;
+    p.status = c->status_dev;
+    p.sched = ws_ptr<int>(c, w.sched);
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    prof_begin(c, KC_WGRAD_UPDATE);
+    if (mom) {
+        p.v = c->vy; p.mu = c->momentum;
+        if (c->fresh)
+            umma_wgrad_update_kernel<true, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(c->wu_maps_mom, p);
+        else
+            umma_wgrad_update_kernel<false, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(c->wu_maps_mom, p);
+    } else if (c->fresh)
+        umma_wgrad_update_kernel<true, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(c->wu_maps, p);
+    else
+        umma_wgrad_update_kernel<false, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(c->wu_maps, p);
+    PARLE_LAUNCHED(c);
     TailPlan tp = {};
     tp.n_layers = nl; tp.batch = B;
     long long longest = 0;
@@ -1000,9 +1003,10 @@ int parle_bind_momentum(parle_ctx *c, float *vy, float *vx) {
         for (int l = 0; l < c->n_layers; ++l) {
             const size_t din = c->dims[l], dout = c->dims[l + 1], wo = c->layers[l].w_off;
             float *base[4] = {c->buf.x + wo, c->buf.y + wo, c->buf.z + wo, vy + wo};
-            CUtensorMap *tm[4] = {&c->tm_mx[l], &c->tm_my[l], &c->tm_mz[l], &c->tm_mv[l]};
+            CUtensorMap *tm[4] = {&c->wu_maps_mom.x[l], &c->wu_maps_mom.y[l], &c->wu_maps_mom.z[l], &c->wu_maps_mom.v[l]};
             for (int k = 0; k < 4; ++k)
                 PARLE_TRY(encode_f32_map(c, tm[k], base[k], din, dout, c->n, din, c->stride, UM_BM, WU_CHUNK_ROWS_MOM));
+            c->wu_maps_mom.a[l] = c->tm_wg_a[l]; c->wu_maps_mom.b[l] = c->tm_wg_b[l];
         }
         c->mom_maps = true;
     }

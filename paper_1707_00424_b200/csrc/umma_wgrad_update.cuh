@@ -75,27 +75,42 @@ template <> __device__ __forceinline__ void tc_ld_cols<8>(uint32_t taddr, uint32
 }
 template <> __device__ __forceinline__ void tc_ld_cols<16>(uint32_t taddr, uint32_t (&r)[16]) { tc_ld_32x16(taddr, r); }
 
+// One launch covers the W segments of all layers: its tile list is layer 0's tiles (replica-major, then
+// n-tile, then m-tile), then layer 1's, ...
+struct WuLayer {
+    int M, N;                    // M = d_in (tile rows), N = d_out (tile columns)
+    int tiles_m, tiles_n;
+    int tile_begin;              // index of the layer's first tile in the launch's list
+    int ld;                      // row pitch of W_l (= d_in)
+    int shadow_cb;               // column blocks per row block of the blocked bf16 copy
+    long long w_off;             // W_l inside a replica's parameter vector (elements)
+    long long shadow_off;        // blocked copy of W_l inside a replica's copy (elements)
+};
 struct WgradUpdateParams {
-    int M, N, K;                 // M = d_in (tile rows), N = d_out (tile columns), K = batch
-    int groups, tiles_m, tiles_n;
-    float *y, *z;                // W_l segment of replica 0; element (replica g, W row r, W col c) at g*gs + r*ld + c
-    __nv_bfloat16 *shadow;       // blocked bf16 copy of W_l of replica 0 (128 x 64 blocks, row-block major)
-    long long shadow_gs; int shadow_cb;   // replica pitch (elements) and column blocks per row block
-    long long gs; int ld;
+    int K;                       // batch
+    int groups, n_layers, total_tiles;
+    WuLayer layer[PARLE_MAX_LAYERS];
+    float *y, *z;                // replica 0; element (replica g, layer l, W row r, W col c) at g*gs + w_off + r*ld + c
+    __nv_bfloat16 *shadow;       // blocked bf16 copy of replica 0 (128 x 64 blocks, row-block major)
+    long long shadow_gs;         // replica pitch of the copy (elements)
+    long long gs;
     float eta_p, inv_gamma, alpha, wd;
     float *v; float mu;          // Nesterov momentum buffer of y (same addressing as y), used by the MOM variant
     int *sched;                  // sched[0]: tiles claimed beyond the first of every CTA, sched[1]: CTAs that have left; both 0 between launches
     int *status;
+};
+// Tensor maps of every layer: A = H_{l-1}^T, B = dH_l^T (bf16 operands), and the W_l segments of x, y, z (and the
+// momentum buffer) as fp32 boxes.
+struct WuMaps {
+    CUtensorMap a[PARLE_MAX_LAYERS], b[PARLE_MAX_LAYERS];
+    CUtensorMap x[PARLE_MAX_LAYERS], y[PARLE_MAX_LAYERS], z[PARLE_MAX_LAYERS], v[PARLE_MAX_LAYERS];
 };
 
 // MOM: Nesterov momentum on the y step (see inner_update_kernel): v <- mu v + d, y <- y - eta' (d + mu v),
 // v = 0 at the start of a round (FIRST: v is only written).
 template <bool FIRST, class SH, bool MOM = false>
 __global__ void __launch_bounds__(SH::THREADS, 1)
-umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                         const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
-                         const __grid_constant__ CUtensorMap tmZ, const __grid_constant__ CUtensorMap tmV,
-                         const WgradUpdateParams p) {
+umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_constant__ WgradUpdateParams p) {
     constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
     constexpr int WU_STATE_BYTES = SH::STATE_BYTES, WU_STATE_STAGES = SH::STAGES, RPG = SH::RPG;
     constexpr int WU_CHUNK_ROWS = SH::CHUNK_ROWS;
@@ -117,9 +132,8 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     const uint32_t bar_qfull = bar_sempty + 8 * WU_STATE_STAGES, bar_qempty = bar_qfull + 8 * WU_TILE_SLOTS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int total_tiles = p.total_tiles;
     const int num_kb = (p.K + UM_BK - 1) / UM_BK;
-    const int per_g = p.tiles_m * p.tiles_n;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < WU_OP_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -141,11 +155,16 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    auto coords = [&](int t, int &g, int &m0, int &n0) {
+    auto coords = [&](int t, int &l, int &g, int &m0, int &n0) {
+        l = 0;
+        while (l + 1 < p.n_layers && t >= p.layer[l + 1].tile_begin) ++l;
+        const WuLayer &ly = p.layer[l];
+        const int per_g = ly.tiles_m * ly.tiles_n;
+        t -= ly.tile_begin;
         g = t / per_g;
         const int r = t - g * per_g;
-        m0 = (r % p.tiles_m) * UM_BM;
-        n0 = (r / p.tiles_m) * UM_BN;
+        m0 = (r % ly.tiles_m) * UM_BM;
+        n0 = (r / ly.tiles_m) * UM_BN;
     };
     // Consumer side of the tile ring (one lane per role calls it): the next tile of this CTA, -1 when there is
     // none, -2 when a wait gave up.
@@ -170,14 +189,14 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 mbar_arrive(bar_qfull + 8 * qslot);                           // release: the index is visible to the waiters
                 if (++qslot == WU_TILE_SLOTS) { qslot = 0; qphase ^= 1u; }
                 if (t >= total_tiles) break;
-                int g, m0, n0; coords(t, g, m0, n0);
+                int l, g, m0, n0; coords(t, l, g, m0, n0);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sa = op_base + stage * UM_STAGE_BYTES, sb = sa + UM_A_BYTES;
                     const uint32_t fb = bar_full + 8 * stage;
                     mbar_expect_tx(fb, UM_STAGE_BYTES);
-                    tma_load_3d(sa, &tmA, fb, kb * UM_BK, m0, g);
-                    tma_load_3d(sb, &tmB, fb, kb * UM_BK, n0, g);
+                    tma_load_3d(sa, &maps.a[l], fb, kb * UM_BK, m0, g);
+                    tma_load_3d(sb, &maps.b[l], fb, kb * UM_BK, n0, g);
                     if (++stage == WU_OP_STAGES) { stage = 0; phase ^= 1u; }
                 }
                 t = t_next;
@@ -223,19 +242,20 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             int stage = 0; uint32_t phase = 0; bool ok = true;
             int qslot = 0; uint32_t qphase = 0;
             for (int t; ok && (t = take_tile(qslot, qphase)) >= 0;) {
-                int g, m0, n0; coords(t, g, m0, n0);
+                int l, g, m0, n0; coords(t, l, g, m0, n0);
+                const int N = p.layer[l].N;
                 for (int c = 0; c < WU_CHUNKS; ++c) {
                     const int nb = n0 + c * WU_CHUNK_ROWS;
-                    if (nb >= p.N) break;
+                    if (nb >= N) break;
                     if (!mbar_wait(bar_sempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t dst = st_base + stage * WU_STATE_BYTES;
                     const uint32_t fb = bar_sfull + 8 * stage;
                     mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES);   // STATE_BYTES counts v when MOM
-                    tma_load_3d(dst, &tmX, fb, m0, nb, g);
+                    tma_load_3d(dst, &maps.x[l], fb, m0, nb, g);
                     if (!FIRST) {
-                        tma_load_3d(dst + WU_ARRAY_BYTES, &tmY, fb, m0, nb, g);
-                        tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &tmZ, fb, m0, nb, g);
-                        if (MOM) tma_load_3d(dst + 3 * WU_ARRAY_BYTES, &tmV, fb, m0, nb, g);
+                        tma_load_3d(dst + WU_ARRAY_BYTES, &maps.y[l], fb, m0, nb, g);
+                        tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &maps.z[l], fb, m0, nb, g);
+                        if (MOM) tma_load_3d(dst + 3 * WU_ARRAY_BYTES, &maps.v[l], fb, m0, nb, g);
                     }
                     if (++stage == WU_STATE_STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -267,26 +287,27 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             if (lane == 0) mbar_arrive(bar_qempty + 8 * qslot);
             if (++qslot == WU_TILE_SLOTS) { qslot = 0; qphase ^= 1u; }
             if (t < 0) break;
-            int g, m0, n0; coords(t, g, m0, n0);
+            int l, g, m0, n0; coords(t, l, g, m0, n0);
+            const int N = p.layer[l].N, ld = p.layer[l].ld;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
             tc_fence_after();
             const int col = q * 32 + lane;                   // tile column along d_in
             const int m = m0 + col;
-            const bool m_ok = m < p.M;
-            const long long tile_e0 = (long long)g * p.gs + (long long)(n0 + grp * RPG) * p.ld + m;
-            const long long chunk_step = (long long)WU_CHUNK_ROWS * p.ld;
+            const bool m_ok = m < p.layer[l].M;
+            const long long tile_e0 = (long long)g * p.gs + p.layer[l].w_off + (long long)(n0 + grp * RPG) * ld + m;
+            const long long chunk_step = (long long)WU_CHUNK_ROWS * ld;
             float *yp = p.y + tile_e0, *zp = p.z + tile_e0;
             float *vp = MOM ? p.v + tile_e0 : nullptr;
             // blocked copy: W row r, column m live in block (r/128, m/64) at (r%128)*64 + m%64; n0 % 128 == 0
-            __nv_bfloat16 *sp = p.shadow + (long long)g * p.shadow_gs +
-                                ((long long)(n0 / UM_BN) * p.shadow_cb + (m >> 6)) * (UM_BN * 64) +
+            __nv_bfloat16 *sp = p.shadow + (long long)g * p.shadow_gs + p.layer[l].shadow_off +
+                                ((long long)(n0 / UM_BN) * p.layer[l].shadow_cb + (m >> 6)) * (UM_BN * 64) +
                                 (grp * RPG) * 64 + (m & 63);
 #pragma unroll 1
             for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
                 if (MOM && c > 0) vp += chunk_step;
                 const int nb0 = n0 + c * WU_CHUNK_ROWS;
-                if (nb0 >= p.N) break;                       // same rule as the loader
+                if (nb0 >= N) break;                         // same rule as the loader
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
                 if (!ok) break;
                 const int nb = nb0 + grp * RPG;
@@ -310,7 +331,7 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
                 if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
-                const int rows = m_ok ? (p.N - nb) : 0;      // rows of this thread that exist
+                const int rows = m_ok ? (N - nb) : 0;        // rows of this thread that exist
                 float *yr = yp, *zr = zp, *vr = vp;
                 __nv_bfloat16 *sr = sp;
                 auto update_row = [&](int j) {
@@ -330,15 +351,15 @@ umma_wgrad_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 };
                 if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
+                    for (int j = 0; j < RPG; ++j, yr += ld, zr += ld, sr += 64) {
                         update_row(j);
-                        if (MOM) vr += p.ld;
+                        if (MOM) vr += ld;
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j, yr += p.ld, zr += p.ld, sr += 64) {
+                    for (int j = 0; j < RPG; ++j, yr += ld, zr += ld, sr += 64) {
                         if (j < rows) update_row(j);
-                        if (MOM) vr += p.ld;
+                        if (MOM) vr += ld;
                     }
                 }
             }
