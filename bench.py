@@ -137,9 +137,10 @@ def ncu_traffic(workload: str, kernel: str):
     return rec["bytes"]
 
 
-def algorithmic_bytes_per_round(cfg, stride):
+def algorithmic_bytes_per_round(cfg, stride, tf32_split=False):
     """Bytes each kernel class has to move per Parle round (all n replicas), from the data it must
-    touch once: parameter-state vectors at 4 B (fp32) or 2 B (bf16 copy) per element, plus GEMM operands."""
+    touch once: parameter-state vectors at 4 B (fp32) or 2 B (bf16 copy) per element, plus GEMM operands.
+    tf32_split: the fp32 update also writes the tf32 hi/lo copy of y (8 B per element)."""
     n, B, L, dims = cfg.n, cfg.batch, cfg.L, cfg.dims
     nl = len(dims) - 1
     Pw = sum(dims[l] * dims[l + 1] for l in range(nl))
@@ -147,7 +148,7 @@ def algorithmic_bytes_per_round(cfg, stride):
     act = lambda l: B * dims[l]                          # elements of one replica's activation at level l
     out = {}
     # separate update: read g, y, x, z, write y, z (+2 B bf16 copy); first step of a round reads x for y and z
-    out["inner_update"] = n * stride * ((24 + (2 if bf else 0)) * L - 8)
+    out["inner_update"] = n * stride * ((24 + (2 if bf else 0) + (8 if tf32_split else 0)) * L - 8)
     out["outer_mean"] = stride * (12 * n + 8)
     if bf:
         opnd = sum(2 * (act(l) + act(l + 1)) for l in range(nl))             # dH^T and H^T, bf16
@@ -272,7 +273,8 @@ def run_ours(args):
     total_ms = sum(v[0] for v in prof.values()) or 1.0
     shares = {k: {"ms_per_round": v[0] / K, "launches_per_round": v[1] / K, "share": v[0] / total_ms} for k, v in prof.items()}
     dom = max(prof, key=lambda k: prof[k][0])
-    alg = algorithmic_bytes_per_round(cfg, model.stride)
+    t3 = cfg.gemm_dtype == 0 and model.fp32_tensor_cores_active
+    alg = algorithmic_bytes_per_round(cfg, model.stride, tf32_split=t3)
     rooflines = {}
     for k, (ms_k, cnt_k) in prof.items():
         if k not in alg:
@@ -283,6 +285,24 @@ def run_ours(args):
                         "peak_source": peaks["source"], "bytes_per_launch": alg[k] * K / cnt_k,
                         "ms_per_launch": ms_k / cnt_k, "launches_per_round": cnt_k / K}
     flops = gemm_flops_per_round(cfg)
+    if cfg.gemm_dtype == 0:
+        # fp32 configurations.  Tensor cores: every fp32 product is three tf32 products (hi/lo operand split), so the
+        # useful rate can reach a third of the tf32 peak at most; tf32 peak = measured bf16 peak x nominal ratio 1.1 / 2.25.
+        # FMA pipes: 148 SMs x 128 lanes x 2 flop x the maximum SM clock.
+        sm_max = (clocks or {}).get("sm_max_mhz") or 1965.0
+        tf32_peak = peaks["bf16_tflops"] * 1.1 / 2.25
+        alu_peak = 148 * 128 * 2 * sm_max * 1e6 / 1e12
+        for k, f in flops.items():
+            if k not in prof or k == "wgrad_gemm_fused_update":
+                continue
+            tf = f * K / (prof[k][0] * 1e-3) / 1e12
+            rooflines[k] = {"kernel": k, "bound": "tensor" if t3 else "alu", "achieved": tf,
+                            "peak": tf32_peak if t3 else alu_peak, "unit": "TFLOP/s", "frac": tf / (tf32_peak if t3 else alu_peak),
+                            "traffic": None, "peak_source": (peaks["source"] + " bf16 x 1.1/2.25 (tf32)") if t3 else "148 SMs x 128 FMA lanes x max SM clock",
+                            "note": ("useful fp32 flops; the kernel executes 3 tf32 products per fp32 product, so frac <= 1/3" if t3 else
+                                     "fp32 FMA pipes"),
+                            "ms_per_launch": prof[k][0] / prof[k][1], "launches_per_round": prof[k][1] / K}
+        flops = {}
     for k, f in flops.items():
         if k in prof and k in rooflines:
             tf = f * K / (prof[k][0] * 1e-3) / 1e12
@@ -297,7 +317,7 @@ def run_ours(args):
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.gemm_dtype == 1 else "f32", "data": "synthetic",
         "config": {"workload": f"{cfg.name}: n={cfg.n} replicas/GPU, MLP {'-'.join(map(str, cfg.dims))}, batch {cfg.batch}, L={cfg.L}, "
-                               f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else 'fp32'}",
+                               f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else ('fp32 (products as 3 x tf32 on the tensor cores)' if t3 else 'fp32 (FMA pipes)')}",
                    "step": "one Parle round (L inner steps + outer step + replica mean)",
                    "l2": "state + gradients per round >> 126 MB L2 (no flush needed)" if cfg.n * model.stride * 16 > 4e8 else "working set may be L2 resident",
                    "launch": "rounds replayed from CUDA graphs (same kernels, same order)" if args.graphs else "one launch per kernel",

@@ -178,6 +178,18 @@ int parle_round_host(parle_ctx *ctx, int L, const float *inputs_host, const int3
  * fp32 rounding).  EUNSUPPORTED on the fp32 path, ESTATE in the middle of a round. */
 int parle_set_fused_update(parle_ctx *ctx, int on);
 
+/* fp32 configurations only: where the forward / backward products run (Section 1.1 / 2.1, the minibatch
+ * gradient).  On an sm_100 device, when the batch and every layer's input width are multiples of 4, they can
+ * run on the tensor cores at fp32 accuracy: every fp32 operand is kept as a pair of tf32-exact arrays
+ * (hi = the value rounded to tf32, lo = the remainder rounded to tf32) in the workspace and every product is the
+ * sum of three tf32 products (lo x hi, hi x lo, hi x hi) with fp32 accumulation; the dropped lo x lo term is
+ * 2^-22 relative.  mode 0: always the FMA pipes; 1 (default): tensor cores when the batch has at least 32 rows
+ * and every layer's input is at least 128 wide; 2: tensor cores whenever the shapes allow.  The two paths
+ * agree to fp32 rounding, not bit for bit.  EINVAL on a bf16 context, ESTATE inside a round.
+ * parle_fp32_tensor_cores_active: 1 if the bound context currently uses the tensor-core path. */
+int parle_set_fp32_tensor_cores(parle_ctx *ctx, int mode);
+int parle_fp32_tensor_cores_active(const parle_ctx *ctx);
+
 /* Change gamma, rho (Eq. scoping changes them between rounds) or the step
  * sizes eta, eta' between calls.  +INFINITY allowed for gamma and rho. */
 int parle_set_coupling(parle_ctx *ctx, double gamma, double rho);
@@ -240,7 +252,16 @@ const char *parle_profile_class_name(int k);
  *   PARLE_DBG_LOGITS  logits                            [n, B, d_last] fp32   (layer ignored)
  *   PARLE_DBG_OPERAND_COPY  bf16 copy of the weights the GEMMs read, stored per layer in 128-row x 64-column
  *                           blocks (row-block major), [n, bytes/(2n)] (bf16 path; layer ignored)
+ * fp32 configurations whose shapes allow the tensor-core path hold tf32-exact hi/lo pairs (kind = hi, kind + 1 = lo):
+ *   PARLE_DBG_T3_PARAMS   the parameters the products read     [n, stride] fp32   (layer ignored)
+ *   PARLE_DBG_T3_INPUT_T  the minibatch, transposed            [n, d_0, B] fp32   (layer ignored)
+ *   PARLE_DBG_T3_ACT_T    output of `layer`, transposed        [n, d, B]   fp32   (not for the last layer)
+ *   PARLE_DBG_T3_DACT_T   gradient w.r.t. it, transposed       [n, d, B]   fp32
  * EINVAL if that buffer does not exist in this configuration. */
+#define PARLE_DBG_T3_PARAMS 6
+#define PARLE_DBG_T3_INPUT_T 8
+#define PARLE_DBG_T3_ACT_T 10
+#define PARLE_DBG_T3_DACT_T 12
 #define PARLE_DBG_ACT 0
 #define PARLE_DBG_ACT_T 1
 #define PARLE_DBG_DACT 2

@@ -71,6 +71,8 @@ def lib() -> C.CDLL:
         "parle_set_coupling": (ci, [vp, cd, cd]),
         "parle_set_lr": (ci, [vp, cd, cd]),
         "parle_set_fused_update": (ci, [vp, ci]),
+        "parle_set_fp32_tensor_cores": (ci, [vp, ci]),
+        "parle_fp32_tensor_cores_active": (ci, [vp]),
         "parle_set_weight_decay": (ci, [vp, cd]),
         "parle_set_wide_tile_threshold": (ci, [vp, ci]),
         "parle_bind_momentum": (ci, [vp, vp, vp]),
@@ -260,6 +262,14 @@ class Parle:
     def set_fused_update(self, on: bool):
         self._check(self._L.parle_set_fused_update(self._h, 1 if on else 0), "parle_set_fused_update")
 
+    def set_fp32_tensor_cores(self, mode: int):
+        """0: FMA pipes, 1: tensor cores (3 x tf32) for wide layers, 2: tensor cores whenever the shapes allow."""
+        self._check(self._L.parle_set_fp32_tensor_cores(self._h, mode), "parle_set_fp32_tensor_cores")
+
+    @property
+    def fp32_tensor_cores_active(self) -> bool:
+        return bool(self._L.parle_fp32_tensor_cores_active(self._h))
+
     def status(self) -> int:
         f = C.c_int()
         self._check(self._L.parle_status(self._h, C.byref(f)), "parle_status")
@@ -269,6 +279,7 @@ class Parle:
         self._check(self._L.parle_clear_status(self._h), "parle_clear_status")
 
     DBG_ACT, DBG_ACT_T, DBG_DACT, DBG_DACT_T, DBG_LOGITS, DBG_OPERAND_COPY = range(6)
+    DBG_T3_PARAMS, DBG_T3_INPUT_T, DBG_T3_ACT_T, DBG_T3_DACT_T = 6, 8, 10, 12      # hi; + 1 = lo
 
     def debug_buffer(self, kind: int, layer: int = 0):
         """View (torch, no copy) of an intermediate of the last inner step inside the workspace."""
@@ -281,6 +292,11 @@ class Parle:
         d = self.dims[layer + 1]
         if kind == self.DBG_LOGITS:
             return raw.view(torch.float32).view(n, B, self.dims[-1])
+        if kind >= self.DBG_T3_PARAMS:
+            t = raw.view(torch.float32)
+            if kind - (kind & 1) == self.DBG_T3_PARAMS:
+                return t.view(n, -1)
+            return t.view(n, self.dims[0] if kind - (kind & 1) == self.DBG_T3_INPUT_T else d, B)
         if kind == self.DBG_OPERAND_COPY:
             return raw.view(torch.bfloat16).view(n, -1)
         if kind in (self.DBG_ACT_T, self.DBG_DACT_T):

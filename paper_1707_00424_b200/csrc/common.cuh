@@ -17,6 +17,19 @@ enum StatusSlot { SLOT_NONFINITE = 0, SLOT_WAIT_LIMIT = 1, SLOT_BAD_LABEL = 2, S
 
 __host__ __device__ inline size_t round_up(size_t v, size_t m) { return (v + m - 1) / m * m; }
 
+// fp32 -> pair of tf32-exact floats (low 13 mantissa bits zero) with v = hi + lo up to 2^-22 |v|:
+// hi = v rounded to tf32 (nearest, ties away from zero), lo = the exact remainder v - hi rounded the same way.
+// Rounding to nearest keeps both errors centred on zero, so they do not add up over a long reduction.
+__device__ __forceinline__ float round_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return __uint_as_float(r);
+}
+__device__ __forceinline__ void split_tf32(float v, float &hi, float &lo) {
+    hi = round_tf32(v);
+    lo = round_tf32(v - hi);
+}
+
 struct LayerPlan {
     int d_in, d_out;
     size_t w_off, b_off;          // element offsets inside one replica's vector

@@ -230,7 +230,8 @@ __global__ void __launch_bounds__((BM / 8) * (BN / 8)) simt_gemm_tiled_kernel(Si
 //   p = softmax(logits) (row max subtracted), dlogits = (p - onehot)/B,
 //   row_loss = logsumexp - logits[label].
 // Writes fp32 dlogits [rows, C] (d32 != NULL) and/or bf16 copies in both
-// layouts: dbf [B, ld_b] per replica and dbfT [C, B] per replica.
+// layouts: dbf [B, ld_b] per replica and dbfT [C, B] per replica, and/or the
+// fp32 copy as a tf32-exact hi/lo pair in both layouts (dhi, dlo: [rows, ld_split]; dThi, dTlo: [C, B] per replica).
 // With parts > 1 the logits arrive as split-K partial sums: logits = bias + sum_s part_s (s in fixed order),
 // formed here first and written back over part 0 (= the logits buffer).
 __global__ void __launch_bounds__(256)
@@ -239,7 +240,8 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
                            __nv_bfloat16 *__restrict__ dbfT, float *__restrict__ row_loss,
                            int rows, int B, int C, int ld_b, int *status,
                            int parts = 1, long long part_stride = 0, const float *__restrict__ bias = nullptr,
-                           long long bias_gs = 0) {
+                           long long bias_gs = 0, float *__restrict__ dThi = nullptr, float *__restrict__ dTlo = nullptr,
+                           float *__restrict__ dhi = nullptr, float *__restrict__ dlo = nullptr, int ld_split = 0) {
     const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const int lane = threadIdx.x % 32;
     if (row >= rows) return;
@@ -275,6 +277,14 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
             const __nv_bfloat16 h = __float2bfloat16_rn(d);
             dbf[((size_t)g * B + i) * ld_b + j] = h;
             dbfT[((size_t)g * C + j) * B + i] = h;
+        }
+        if (dThi) {                                  // tf32-exact hi/lo pair, [B, ld_split] and transposed [C, B] per replica
+            float hi, lo;
+            split_tf32(d, hi, lo);
+            dThi[((size_t)g * C + j) * B + i] = hi;
+            dTlo[((size_t)g * C + j) * B + i] = lo;
+            dhi[(size_t)row * ld_split + j] = hi;
+            dlo[(size_t)row * ld_split + j] = lo;
         }
     }
     if (lane == 0) {

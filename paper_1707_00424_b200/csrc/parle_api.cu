@@ -8,6 +8,7 @@
 #include "mlp_simt.cuh"
 #include "umma_gemm.cuh"
 #include "umma_wgrad_update.cuh"
+#include "umma_tf32x3.cuh"
 #include "update_kernels.cuh"
 
 using namespace parle;
@@ -36,6 +37,12 @@ struct Workspace {
     size_t dhb[PARLE_MAX_LAYERS], dhbT[PARLE_MAX_LAYERS];    // their gradients, both layouts
     int dh_ld[PARLE_MAX_LAYERS];       // row pitch of dhb[l] (d_{l+1} rounded up to 8)
     size_t row_loss;                   // [n,B] fp32
+    // fp32 mode on the tensor cores (3 x tf32): tf32-exact hi/lo pairs, index [0] = hi, [1] = lo
+    size_t w_split[2];                 // parameters [n, stride]
+    size_t wT_split[2];                // transposed weights of layers >= 1, [n, t3_t_stride]
+    size_t xs[2], xT[2];               // inputs [n, B, d_0] and transposed [n, d_0, B]
+    size_t hs[PARLE_MAX_LAYERS][2], hT[PARLE_MAX_LAYERS][2];     // hidden activations [n, B, d_{l+1}] and transposed
+    size_t dhs[PARLE_MAX_LAYERS][2], dhT[PARLE_MAX_LAYERS][2];   // their gradients [n, B, ld_l] (ld_l = d_{l+1} rounded up to 4) and transposed [n, d_{l+1}, B]
     size_t sched;                      // bf16 mode: two ints, the tile counters of the fused weight-gradient kernel (zero between launches)
     size_t stage_in[2], stage_lab[2], stage_loss[2];   // double-buffered staging for the host-buffer entry points
     size_t total;
@@ -87,6 +94,15 @@ struct parle_ctx {
     CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
+    // fp32 configurations on the tensor cores (three tf32 products per GEMM)
+    int t3_mode;                     // 0 = never, 1 = when the layers are wide enough to fill 128-row tiles, 2 = whenever possible
+    bool t3_shapes_ok;               // widths and batch are multiples of 4 (16-byte rows for TMA)
+    bool t3_ready;                   // tensor maps exist for the bound buffers (needs an sm_100 device)
+    size_t t3_t_off[PARLE_MAX_LAYERS], t3_t_stride;   // transposed weight copy: W_l^T [d_in, ld_l] of layers >= 1 inside a replica's copy
+    int t3_bn_fwd[PARLE_MAX_LAYERS], t3_bn_dg[PARLE_MAX_LAYERS], t3_bn_wg[PARLE_MAX_LAYERS];   // tile widths (64 or 128)
+    CUtensorMap t3_fa[PARLE_MAX_LAYERS][2], t3_fb[PARLE_MAX_LAYERS][2];    // forward operands, hi / lo
+    CUtensorMap t3_da[PARLE_MAX_LAYERS][2], t3_db[PARLE_MAX_LAYERS][2];    // data gradient
+    CUtensorMap t3_wa[PARLE_MAX_LAYERS][2], t3_wb[PARLE_MAX_LAYERS][2];    // weight gradient
     WuMaps wu_maps;                  // fused weight-gradient kernel: operands + fp32 W_l segments of x, y, z (32-row boxes)
     WuMaps wu_maps_mom;              // its momentum variant: same + vy, 16-row boxes
     bool mom_maps;
@@ -148,6 +164,22 @@ void plan_workspace(parle_ctx *c) {
     if (c->gemm_dtype == PARLE_GEMM_FP32) {
         for (int l = 0; l < nl; ++l) w.act[l] = take(n * B * c->dims[l + 1] * sizeof(float));
         for (int l = 0; l < nl; ++l) w.dact[l] = take(n * B * c->dims[l + 1] * sizeof(float));
+        if (c->t3_shapes_ok) {
+            for (int h = 0; h < 2; ++h) {
+                w.w_split[h] = take(n * c->stride * sizeof(float));
+                w.wT_split[h] = take(n * c->t3_t_stride * sizeof(float));
+                w.xs[h] = take(n * B * c->dims[0] * sizeof(float));
+                w.xT[h] = take(n * B * c->dims[0] * sizeof(float));
+                for (int l = 0; l + 1 < nl; ++l) {
+                    w.hs[l][h] = take(n * B * c->dims[l + 1] * sizeof(float));
+                    w.hT[l][h] = take(n * B * c->dims[l + 1] * sizeof(float));
+                }
+                for (int l = 0; l < nl; ++l) {
+                    w.dhs[l][h] = take(n * B * round_up(c->dims[l + 1], 4) * sizeof(float));
+                    w.dhT[l][h] = take(n * B * c->dims[l + 1] * sizeof(float));
+                }
+            }
+        }
     } else {
         w.shadow = take(n * c->sh_stride * 2);
         w.xb = take(n * B * c->dims[0] * 2);
@@ -244,6 +276,94 @@ int encode_blocked_map(parle_ctx *c, CUtensorMap *tm, const void *base, int cb, 
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
     return PARLE_OK;
+}
+
+// fp32 tensor [groups][rows][cols] as a tf32 operand: boxes of 32 columns (128 bytes) x box_rows, 128-byte swizzle.
+int encode_tf32_map(parle_ctx *c, CUtensorMap *tm, const void *base, size_t cols, size_t rows, size_t groups,
+                    size_t row_pitch, size_t group_pitch, unsigned box_rows) {
+    EncodeTiledFn enc;
+    PARLE_TRY(get_encoder(c, &enc));
+    cuuint64_t dims[3] = {cols, rows, groups};
+    cuuint64_t strides[2] = {row_pitch * 4, group_pitch * 4};
+    cuuint32_t box[3] = {32, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
+    return PARLE_OK;
+}
+
+// Tile width of a tf32 product: 128 columns, or 64 when 128-wide tiles would leave a quarter of the SMs idle.
+inline int t3_tile_width(const parle_ctx *c, int M, int N) {
+    const long long wide = (long long)c->n * ((M + T3_BM - 1) / T3_BM) * ((N + 127) / 128);
+    return wide * 4 < (long long)c->sm_count * 3 ? 64 : 128;
+}
+
+int build_tf32_maps(parle_ctx *c) {
+    const Workspace &w = c->ws;
+    const size_t n = c->n, B = c->batch, S = c->stride;
+    for (int l = 0; l < c->n_layers; ++l) {
+        const size_t din = c->dims[l], dout = c->dims[l + 1], wo = c->layers[l].w_off;
+        c->t3_bn_fwd[l] = t3_tile_width(c, (int)B, (int)dout);
+        c->t3_bn_dg[l] = t3_tile_width(c, (int)B, (int)din);
+        c->t3_bn_wg[l] = t3_tile_width(c, (int)din, (int)dout);
+        const size_t ld = round_up(dout, 4);
+        for (int h = 0; h < 2; ++h) {
+            const float *in = l == 0 ? ws_ptr<float>(c, w.xs[h]) : ws_ptr<float>(c, w.hs[l - 1][h]);
+            const float *inT = l == 0 ? ws_ptr<float>(c, w.xT[h]) : ws_ptr<float>(c, w.hT[l - 1][h]);
+            const float *W = ws_ptr<float>(c, w.w_split[h]) + wo;
+            // forward: A = input [B, d_in], B = W [d_out, d_in] (K = d_in)
+            PARLE_TRY(encode_tf32_map(c, &c->t3_fa[l][h], in, din, B, n, din, B * din, T3_BM));
+            PARLE_TRY(encode_tf32_map(c, &c->t3_fb[l][h], W, din, dout, n, din, S, c->t3_bn_fwd[l]));
+            if (l > 0) {
+                // data gradient: A = dH [B, d_out] (pitch ld), B = W^T [d_in, d_out] (pitch ld) (K = d_out)
+                const float *WT = ws_ptr<float>(c, w.wT_split[h]) + c->t3_t_off[l];
+                PARLE_TRY(encode_tf32_map(c, &c->t3_da[l][h], ws_ptr<float>(c, w.dhs[l][h]), dout, B, n, ld, B * ld, T3_BM));
+                PARLE_TRY(encode_tf32_map(c, &c->t3_db[l][h], WT, dout, din, n, ld, c->t3_t_stride, c->t3_bn_dg[l]));
+            }
+            // weight gradient (transposed): A = input^T [d_in, B], B = dH^T [d_out, B] (K = batch)
+            PARLE_TRY(encode_tf32_map(c, &c->t3_wa[l][h], inT, B, din, n, B, din * B, T3_BM));
+            PARLE_TRY(encode_tf32_map(c, &c->t3_wb[l][h], ws_ptr<float>(c, w.dhT[l][h]), B, dout, n, B, dout * B, c->t3_bn_wg[l]));
+        }
+    }
+    return PARLE_OK;
+}
+
+template <int EPI, int BN>
+int launch_t3_bn(parle_ctx *c, int cls, const CUtensorMap *a, const CUtensorMap *b, T3Params p) {
+    p.groups = c->n;
+    p.tiles_m = (p.M + T3_BM - 1) / T3_BM;
+    p.tiles_n = (p.N + BN - 1) / BN;
+    p.status = c->status_dev;
+    const int tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    prof_begin(c, cls);
+    umma_tf32x3_kernel<EPI, BN><<<grid, T3_THREADS, T3Shape<BN>::SMEM_BYTES, c->stream>>>(a[0], a[1], b[0], b[1], p);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+template <int EPI>
+int launch_t3(parle_ctx *c, int cls, int bn, const CUtensorMap *a, const CUtensorMap *b, const T3Params &p) {
+    return bn == 64 ? launch_t3_bn<EPI, 64>(c, cls, a, b, p) : launch_t3_bn<EPI, 128>(c, cls, a, b, p);
+}
+template <int EPI>
+cudaError_t allow_t3_smem() {
+    cudaError_t e = cudaFuncSetAttribute(umma_tf32x3_kernel<EPI, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)T3Shape<64>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(umma_tf32x3_kernel<EPI, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)T3Shape<128>::SMEM_BYTES);
+}
+
+// fp32 products on the tensor cores?  Automatic mode wants every layer input at least one 128-wide tile.
+inline bool use_t3(const parle_ctx *c) {
+    if (c->gemm_dtype != PARLE_GEMM_FP32 || !c->t3_ready || c->t3_mode == 0) return false;
+    if (c->t3_mode == 2) return true;
+    if (c->batch < 32) return false;
+    for (int l = 0; l < c->n_layers; ++l)
+        if (c->dims[l] < 128) return false;
+    return true;
 }
 
 int build_tensor_maps(parle_ctx *c) {
@@ -364,29 +484,140 @@ int run_blocked_copy(parle_ctx *c, const float *src) {
     return PARLE_OK;
 }
 
-int run_inner_update(parle_ctx *c, const float *grad, float wd) {
-    const size_t n4 = (size_t)c->n * c->stride / 4;
+int run_split_transpose(parle_ctx *c, const float *src);
+
+template <bool FIRST, bool MOM, bool SPLIT>
+void launch_inner_update(parle_ctx *c, int grid, const float4 *g, float4 *y, const float4 *x, float4 *z, size_t n4, float wd) {
     constexpr int U = 2;
-    const int grid = stream_grid(c, n4, U);
+    inner_update_kernel<FIRST, U, MOM, SPLIT><<<grid, kUpdThreads, 0, c->stream>>>(
+        g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev,
+        MOM ? reinterpret_cast<float4 *>(c->vy) : nullptr, c->momentum,
+        SPLIT ? ws_ptr<float4>(c, c->ws.w_split[0]) : nullptr, SPLIT ? ws_ptr<float4>(c, c->ws.w_split[1]) : nullptr);
+}
+
+// split: also refresh the tf32 hi/lo copy of the parameters from the new y (fp32 products on the tensor cores)
+int run_inner_update(parle_ctx *c, const float *grad, float wd, bool split = false) {
+    const size_t n4 = (size_t)c->n * c->stride / 4;
+    const int grid = stream_grid(c, n4, 2);
     const float4 *g = reinterpret_cast<const float4 *>(grad);
     float4 *y = reinterpret_cast<float4 *>(c->buf.y), *z = reinterpret_cast<float4 *>(c->buf.z);
     const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
     prof_begin(c, KC_INNER_UPDATE);
-    if (c->momentum > 0.f) {
-        float4 *v = reinterpret_cast<float4 *>(c->vy);
-        if (c->fresh)
-            inner_update_kernel<true, U, true><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev, v, c->momentum);
-        else
-            inner_update_kernel<false, U, true><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev, v, c->momentum);
-    } else if (c->fresh)
-        inner_update_kernel<true, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev);
-    else
-        inner_update_kernel<false, U><<<grid, kUpdThreads, 0, c->stream>>>(g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev);
+    const int variant = (c->fresh ? 4 : 0) | (c->momentum > 0.f ? 2 : 0) | (split ? 1 : 0);
+    switch (variant) {
+        case 0: launch_inner_update<false, false, false>(c, grid, g, y, x, z, n4, wd); break;
+        case 1: launch_inner_update<false, false, true>(c, grid, g, y, x, z, n4, wd); break;
+        case 2: launch_inner_update<false, true, false>(c, grid, g, y, x, z, n4, wd); break;
+        case 3: launch_inner_update<false, true, true>(c, grid, g, y, x, z, n4, wd); break;
+        case 4: launch_inner_update<true, false, false>(c, grid, g, y, x, z, n4, wd); break;
+        case 5: launch_inner_update<true, false, true>(c, grid, g, y, x, z, n4, wd); break;
+        case 6: launch_inner_update<true, true, false>(c, grid, g, y, x, z, n4, wd); break;
+        default: launch_inner_update<true, true, true>(c, grid, g, y, x, z, n4, wd); break;
+    }
     PARLE_LAUNCHED(c);
     c->fresh = false;
     c->shadow_is_x = false;
     c->steps_in_round++;
     if (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0) PARLE_TRY(run_blocked_copy(c, c->buf.y));
+    if (split) PARLE_TRY(run_split_transpose(c, c->buf.y));
+    return PARLE_OK;
+}
+
+// Transposed tf32 hi/lo copy of the weights of layers >= 1 (the B operand of the data-gradient products).
+int run_split_transpose(parle_ctx *c, const float *src) {
+    if (c->n_layers < 2) return PARLE_OK;
+    TransposePlan tp = {};
+    int tiles = 0;
+    for (int l = 1; l < c->n_layers; ++l) {
+        const int k = l - 1;
+        tp.w_off[k] = (long long)c->layers[l].w_off; tp.t_off[k] = (long long)c->t3_t_off[l];
+        tp.d_in[k] = c->dims[l]; tp.d_out[k] = c->dims[l + 1]; tp.ld[k] = (int)round_up(c->dims[l + 1], 4);
+        tp.tiles_in[k] = (c->dims[l] + 31) / 32;
+        tp.first_tile[k] = tiles;
+        tiles += tp.tiles_in[k] * ((c->dims[l + 1] + 31) / 32);
+    }
+    tp.n_layers = c->n_layers - 1;
+    tp.first_tile[tp.n_layers] = tiles;
+    prof_begin(c, KC_TO_BF16);
+    split_transpose_kernel<<<dim3(tiles, c->n), 256, 0, c->stream>>>(
+        tp, src, (long long)c->stride, ws_ptr<float>(c, c->ws.wT_split[0]), ws_ptr<float>(c, c->ws.wT_split[1]), (long long)c->t3_t_stride);
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+
+// tf32 hi/lo copies of the parameters from an fp32 vector (x at the start of a round).
+int run_split_copy(parle_ctx *c, const float *src) {
+    const size_t n4 = (size_t)c->n * c->stride / 4;
+    prof_begin(c, KC_TO_BF16);
+    split_tf32_kernel<<<stream_grid(c, n4, 1), 256, 0, c->stream>>>(
+        reinterpret_cast<const float4 *>(src), ws_ptr<float4>(c, c->ws.w_split[0]), ws_ptr<float4>(c, c->ws.w_split[1]), n4);
+    PARLE_LAUNCHED(c);
+    return run_split_transpose(c, src);
+}
+
+// fp32 configuration on the tensor cores: every product as three tf32 products of hi/lo operand pairs.
+int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labels, float *loss_out) {
+    const Workspace &w = c->ws;
+    const int nl = c->n_layers, n = c->n, B = c->batch;
+    const float *params = c->fresh ? c->buf.x : c->buf.y;      // biases come from the fp32 master copy
+    const long long S = (long long)c->stride;
+    {
+        const int d0 = c->dims[0];
+        prof_begin(c, KC_INPUT_CVT);
+        input_split_kernel<<<dim3((d0 + 31) / 32, (B + 31) / 32, n), 256, 0, c->stream>>>(
+            inputs, ws_ptr<float>(c, w.xs[0]), ws_ptr<float>(c, w.xs[1]), ws_ptr<float>(c, w.xT[0]), ws_ptr<float>(c, w.xT[1]), B, d0);
+        PARLE_LAUNCHED(c);
+    }
+    for (int l = 0; l < nl; ++l) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        T3Params p = {};
+        p.M = B; p.N = dout; p.K = din;
+        p.bias = params + c->layers[l].b_off; p.bias_gs = S;
+        if (l + 1 < nl) {
+            p.out_hi = ws_ptr<float>(c, w.hs[l][0]); p.out_lo = ws_ptr<float>(c, w.hs[l][1]);
+            p.out_gs = (long long)B * dout; p.out_ld = dout;
+            p.outT_hi = ws_ptr<float>(c, w.hT[l][0]); p.outT_lo = ws_ptr<float>(c, w.hT[l][1]);
+            p.outT_gs = (long long)B * dout; p.outT_ld = B;
+            PARLE_TRY(launch_t3<T3_FWD_HIDDEN>(c, KC_FWD_GEMM, c->t3_bn_fwd[l], c->t3_fa[l], c->t3_fb[l], p));
+        } else {
+            p.outf = ws_ptr<float>(c, w.act[l]); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
+            PARLE_TRY(launch_t3<T3_FWD_LAST>(c, KC_FWD_GEMM, c->t3_bn_fwd[l], c->t3_fa[l], c->t3_fb[l], p));
+        }
+    }
+    const int C = c->dims[nl], rows = n * B;
+    prof_begin(c, KC_SOFTMAX_CE);
+    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+        ws_ptr<float>(c, w.act[nl - 1]), labels, nullptr, nullptr, nullptr, ws_ptr<float>(c, w.row_loss), rows, B, C, 0,
+        c->status_dev, 1, 0, nullptr, 0, ws_ptr<float>(c, w.dhT[nl - 1][0]), ws_ptr<float>(c, w.dhT[nl - 1][1]),
+        ws_ptr<float>(c, w.dhs[nl - 1][0]), ws_ptr<float>(c, w.dhs[nl - 1][1]), (int)round_up(C, 4));
+    PARLE_LAUNCHED(c);
+    if (loss_out) {
+        prof_begin(c, KC_LOSS_MEAN);
+        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
+        PARLE_LAUNCHED(c);
+    }
+    for (int l = nl - 1; l >= 0; --l) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        T3Params p = {};                                        // dW_l^T = H_{l-1}^T dH_l
+        p.M = din; p.N = dout; p.K = B;
+        p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
+        PARLE_TRY(launch_t3<T3_WGRAD>(c, KC_WGRAD_GEMM, c->t3_bn_wg[l], c->t3_wa[l], c->t3_wb[l], p));
+        prof_begin(c, KC_BIAS_GRAD);
+        bias_grad_split_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
+            ws_ptr<float>(c, w.dhT[l][0]), ws_ptr<float>(c, w.dhT[l][1]), c->buf.grad + c->layers[l].b_off, S, B, dout);
+        PARLE_LAUNCHED(c);
+        if (l > 0) {                                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
+            T3Params d = {};
+            d.M = B; d.N = din; d.K = dout;
+            d.out_hi = ws_ptr<float>(c, w.dhs[l - 1][0]); d.out_lo = ws_ptr<float>(c, w.dhs[l - 1][1]);
+            d.out_gs = (long long)B * din; d.out_ld = din;      // d_in % 4 == 0: no padding
+            d.outT_hi = ws_ptr<float>(c, w.dhT[l - 1][0]); d.outT_lo = ws_ptr<float>(c, w.dhT[l - 1][1]);
+            d.outT_gs = (long long)B * din; d.outT_ld = B;
+            d.mask_hi = ws_ptr<float>(c, w.hT[l - 1][0]); d.mask_lo = ws_ptr<float>(c, w.hT[l - 1][1]);
+            d.mask_gs = (long long)B * din; d.mask_ld = B;
+            PARLE_TRY(launch_t3<T3_DGRAD>(c, KC_DGRAD_GEMM, c->t3_bn_dg[l], c->t3_da[l], c->t3_db[l], d));
+        }
+    }
     return PARLE_OK;
 }
 
@@ -630,6 +861,15 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         c->sh_cb[l] = (c->dims[l] + 63) / 64;
         c->sh_stride += (size_t)c->sh_rb[l] * c->sh_cb[l] * 8192;
     }
+    c->t3_mode = 1;
+    c->t3_shapes_ok = (c->gemm_dtype == PARLE_GEMM_FP32 && c->n_layers > 0 && c->batch % 4 == 0);
+    for (int l = 0; l < c->n_layers; ++l)
+        if (c->dims[l] % 4) c->t3_shapes_ok = false;
+    for (int l = 1; l < c->n_layers; ++l) {
+        c->t3_t_off[l] = c->t3_t_stride;
+        c->t3_t_stride = round_up(c->t3_t_stride + (size_t)c->dims[l] * round_up(c->dims[l + 1], 4), 32);
+    }
+    if (c->t3_t_stride == 0) c->t3_t_stride = 32;
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
     c->wide_tiles_per_sm = 4;
     c->last_ksplit = 1;
@@ -716,6 +956,19 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         // tile counters of the fused weight-gradient kernel: every launch leaves them at zero again
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.sched), 0, 2 * sizeof(int), c->stream));
     }
+    c->t3_ready = false;
+    if (c->t3_shapes_ok) {
+        int major = 0;
+        PARLE_CUDA(c, cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major == 10) {                                      // other devices keep the FMA-pipe products
+            PARLE_CUDA(c, allow_t3_smem<T3_FWD_HIDDEN>());
+            PARLE_CUDA(c, allow_t3_smem<T3_FWD_LAST>());
+            PARLE_CUDA(c, allow_t3_smem<T3_DGRAD>());
+            PARLE_CUDA(c, allow_t3_smem<T3_WGRAD>());
+            PARLE_TRY(build_tf32_maps(c));
+            c->t3_ready = true;
+        }
+    }
     c->bound = true;
     c->round_open = false; c->fresh = false; c->shadow_is_x = false; c->steps_in_round = 0;
     return PARLE_OK;
@@ -725,6 +978,10 @@ int parle_round_begin(parle_ctx *c) {
     PARLE_TRY(check_bound(c));
     if (c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16 && !c->shadow_is_x) {
         PARLE_TRY(run_blocked_copy(c, c->buf.x));
+        c->shadow_is_x = true;
+    }
+    if (use_t3(c) && !c->shadow_is_x) {
+        PARLE_TRY(run_split_copy(c, c->buf.x));
         c->shadow_is_x = true;
     }
     c->round_open = true; c->fresh = true; c->steps_in_round = 0;
@@ -741,6 +998,9 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
             c->fresh = false; c->shadow_is_x = false; c->steps_in_round++;
             return PARLE_OK;
         }
+    } else if (use_t3(c)) {
+        PARLE_TRY(forward_backward_tf32(c, inputs, labels, loss_out));
+        return run_inner_update(c, c->buf.grad, c->weight_decay, true);
     } else {
         PARLE_TRY(forward_backward_fp32(c, inputs, labels, loss_out));
     }
@@ -987,6 +1247,19 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     return PARLE_OK;
 }
 
+int parle_set_fp32_tensor_cores(parle_ctx *c, int mode) {
+    if (!c || mode < 0 || mode > 2) return PARLE_EINVAL;
+    if (c->gemm_dtype != PARLE_GEMM_FP32) return PARLE_EINVAL;
+    if (c->round_open) return PARLE_ESTATE;       // the operand copies of a round belong to one path
+    if (mode != c->t3_mode) {
+        c->t3_mode = mode;
+        c->shadow_is_x = false;
+        drop_round_graphs(c);
+    }
+    return PARLE_OK;
+}
+int parle_fp32_tensor_cores_active(const parle_ctx *c) { return c ? (use_t3(c) ? 1 : 0) : 0; }
+
 int parle_set_wide_tile_threshold(parle_ctx *c, int tiles_per_sm) {
     if (!c || tiles_per_sm < 0) return PARLE_EINVAL;
     c->wide_tiles_per_sm = tiles_per_sm;
@@ -1112,6 +1385,20 @@ int parle_debug_buffer(const parle_ctx *c, int kind, int layer, size_t *byte_off
         if (!bf) return PARLE_EINVAL;
         *byte_offset = w.shadow; *bytes = (size_t)c->n * c->sh_stride * 2;
         return PARLE_OK;
+    }
+    if (kind >= PARLE_DBG_T3_PARAMS && kind <= PARLE_DBG_T3_DACT_T + 1) {
+        if (!c->t3_shapes_ok) return PARLE_EINVAL;
+        const int h = (kind - PARLE_DBG_T3_PARAMS) & 1;            // 0 = hi, 1 = lo
+        switch (kind - h) {
+            case PARLE_DBG_T3_PARAMS: *byte_offset = w.w_split[h]; *bytes = (size_t)c->n * c->stride * 4; return PARLE_OK;
+            case PARLE_DBG_T3_INPUT_T: *byte_offset = w.xT[h]; *bytes = nB * c->dims[0] * 4; return PARLE_OK;
+            case PARLE_DBG_T3_ACT_T:
+                if (layer < 0 || layer >= nl - 1) return PARLE_EINVAL;
+                *byte_offset = w.hT[layer][h]; *bytes = nB * c->dims[layer + 1] * 4; return PARLE_OK;
+            default:
+                if (layer < 0 || layer >= nl) return PARLE_EINVAL;
+                *byte_offset = w.dhT[layer][h]; *bytes = nB * c->dims[layer + 1] * 4; return PARLE_OK;
+        }
     }
     if (layer < 0 || layer >= nl) return PARLE_EINVAL;
     const size_t d = c->dims[layer + 1];

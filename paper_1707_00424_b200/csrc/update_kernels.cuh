@@ -22,12 +22,15 @@ __device__ __forceinline__ bool finite4(const float4 &v) {
 // x is read in place of y and z, which are only written).
 // MOM: Nesterov momentum (Remark, Section 3.1): with d = g + (y - x)/gamma,
 //      v <- mu v + d, y <- y - eta' (d + mu v); v starts from 0 in every round (FIRST: v is only written).
-template <bool FIRST, int UNROLL, bool MOM = false>
+// SPLIT: also store the new y as a tf32-exact pair (hi = y rounded to tf32, lo = y - hi rounded to tf32):
+//      the operands of the fp32-accurate tensor-core products of the next step.
+template <bool FIRST, int UNROLL, bool MOM = false, bool SPLIT = false>
 __global__ void __launch_bounds__(kUpdThreads)
 inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const float4 *__restrict__ x,
                     float4 *__restrict__ z, size_t n4,
                     float eta_p, float inv_gamma, float alpha, float wd, int *status,
-                    float4 *__restrict__ v = nullptr, float mu = 0.f) {
+                    float4 *__restrict__ v = nullptr, float mu = 0.f,
+                    float4 *__restrict__ y_hi = nullptr, float4 *__restrict__ y_lo = nullptr) {
     const size_t tid = (size_t)blockIdx.x * kUpdThreads + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
     const float one_m_alpha = 1.0f - alpha;
@@ -79,6 +82,13 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
                 ok &= finite4(yn);
                 y[i] = yn;
                 z[i] = zn;
+                if (SPLIT) {
+                    float4 h, l;
+                    split_tf32(yn.x, h.x, l.x); split_tf32(yn.y, h.y, l.y);
+                    split_tf32(yn.z, h.z, l.z); split_tf32(yn.w, h.w, l.w);
+                    y_hi[i] = h;
+                    y_lo[i] = l;
+                }
             }
         }
     }

@@ -25,14 +25,19 @@ DEV = "cuda:0"
 TOL = {pb.GEMM_FP32: 1e-4, pb.GEMM_BF16: 2e-2}
 
 
-def make(cfg, fused=None, **over):
+def make(cfg, fused=None, t3=None, **over):
     """fused: None = library default (on for bf16 GEMMs); False = write the gradient to `grad`
-    and run the separate update kernel (needed by the tests that read the gradient)."""
+    and run the separate update kernel (needed by the tests that read the gradient).
+    t3: fp32 configurations only, where the products run (parle_set_fp32_tensor_cores): None = library
+    default, 0 = FMA pipes, 2 = tensor cores (three tf32 products) whatever the widths."""
     hyper = dict(gamma=cfg.gamma, rho=cfg.rho, alpha=cfg.alpha, eta=cfg.eta, eta_prime=cfg.eta_prime)
     hyper.update(over)
     m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, **hyper).alloc(DEV)
     if fused is not None and cfg.gemm_dtype == pb.GEMM_BF16:
         m.set_fused_update(fused)
+    if t3 is not None and cfg.gemm_dtype == pb.GEMM_FP32:
+        m.set_fp32_tensor_cores(t3)
+        assert m.fp32_tensor_cores_active == (t3 == 2)
     x0 = np.stack([po.pack(si.init_replica(cfg, a)) for a in range(cfg.n)])
     m.x.copy_(torch.from_numpy(to_padded(m, x0)))
     m.mean(); torch.cuda.synchronize()
@@ -40,8 +45,8 @@ def make(cfg, fused=None, **over):
     return m, x0, xbar0, po.Hyper(hyper["eta"], hyper["eta_prime"], hyper["alpha"], hyper["gamma"], hyper["rho"])
 
 
-def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False, fused=None):
-    m, xo, xb, hp = make(cfg, fused=fused)
+def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False, fused=None, t3=None):
+    m, xo, xb, hp = make(cfg, fused=fused, t3=t3)
     tol = TOL[cfg.gemm_dtype]
     pad = torch.from_numpy(padding_mask(m)).to(DEV)
     for r in range(rounds):
@@ -83,7 +88,7 @@ def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False, fused=None):
     return m
 
 
-def grad_check(cfg, tol, loose=None, outliers=0):
+def grad_check(cfg, tol, loose=None, outliers=0, t3=None):
     """One inner step: the gradient buffer against the oracle's gradient, layer by layer.
 
     bf16 GEMMs: a ReLU unit whose pre-activation lies within operand rounding of
@@ -95,7 +100,7 @@ def grad_check(cfg, tol, loose=None, outliers=0):
     fp32 GEMMs at full width: one unit within fp32 rounding of zero (probability
     ~1e-7 per unit and sample, ~1e6 units per step) switches now and then; up to
     `outliers` replicas may exceed `tol` and must then stay within 1e-2."""
-    m, xo, xb, hp = make(cfg, fused=False)
+    m, xo, xb, hp = make(cfg, fused=False, t3=t3)
     X, c = si.round_batches(cfg.scaled(L=1), 0)
     loss = torch.zeros(cfg.n, device=DEV)
     m.round_begin(); m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV), loss)
@@ -225,12 +230,55 @@ def test_host_buffer_round_matches_device_round(dtype_dims):
         assert torch.equal(a.x, b.x)
 
 
-def test_c2_gradient_full_shape_fp32():
-    grad_check(si.C2, 1e-5, outliers=1)
+@pytest.mark.parametrize("t3", [0, 2])
+def test_c2_gradient_full_shape_fp32(t3):
+    grad_check(si.C2, 1e-5, outliers=1, t3=t3)
 
 
-def test_c2_one_round_fp32():
-    run_rounds(si.C2, 1)
+@pytest.mark.parametrize("t3", [0, None])
+def test_c2_one_round_fp32(t3):
+    m = run_rounds(si.C2, 1, t3=t3)
+    assert m.fp32_tensor_cores_active == (t3 is None)      # the default puts this shape on the tensor cores
+
+
+# ------------------------------------------------------------------ fp32 configurations on the tensor cores (3 x tf32)
+def test_c1_fp32_tensor_cores():
+    """Every tile is mostly out of range (widths 64-32-10, batch 16, k-blocks shorter than 32)."""
+    assert not make(si.C1)[0].fp32_tensor_cores_active     # narrow layers stay on the FMA pipes by default
+    grad_check(si.C1, 1e-5, t3=2)
+    run_rounds(si.C1, si.C1.rounds, disp_tol=1e-4, t3=2)
+
+
+@pytest.mark.parametrize("n,dims,batch", [(3, (200, 264, 136, 12), 72), (2, (132, 388, 4), 260), (1, (36, 20, 8, 8, 4), 4),
+                                          (5, (520, 72, 300, 100), 136)])
+def test_ragged_shapes_fp32_tensor_cores(n, dims, batch):
+    """Several tiles with ragged edges along the batch, both widths and the reduction length; 64- and 128-wide tiles."""
+    cfg = si.C1.scaled(name="ragged-t3", n=n, dims=dims, batch=batch, L=3)
+    grad_check(cfg, 1e-5, t3=2)
+    run_rounds(cfg, 2, disp_tol=1e-4, t3=2)
+    run_rounds(cfg, 1, disp_tol=1e-4, use_round_call=True, t3=2)
+
+
+def test_tensor_core_and_fma_paths_agree_fp32():
+    """Same step on both paths: gradients agree to fp32 rounding (a few 1e-7), far inside the 1e-5 either has to the oracle."""
+    cfg = si.C1.scaled(name="both", n=2, dims=(256, 384, 128, 16), batch=128, L=1)
+    grads = []
+    for t3 in (0, 2):
+        m, *_ = make(cfg, t3=t3)
+        X, c = si.round_batches(cfg, 0)
+        m.round_begin(); m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV))
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        grads.append(to_dense(m, m.grad.cpu().numpy()))
+    assert rel_l2(grads[1], grads[0]) < 2e-6, rel_l2(grads[1], grads[0])
+
+
+def test_shapes_not_multiples_of_four_stay_on_fma_pipes():
+    cfg = si.C1.scaled(name="odd", n=2, dims=(130, 140, 10), batch=128, L=2)
+    m, *_ = make(cfg)
+    m.set_fp32_tensor_cores(2)
+    assert not m.fp32_tensor_cores_active
+    run_rounds(cfg, 1, disp_tol=1e-4)
 
 
 # ------------------------------------------------------------------ bf16 GEMMs (tcgen05)
