@@ -532,9 +532,9 @@ int run_split_transpose(parle_ctx *c, const float *src) {
         const int k = l - 1;
         tp.w_off[k] = (long long)c->layers[l].w_off; tp.t_off[k] = (long long)c->t3_t_off[l];
         tp.d_in[k] = c->dims[l]; tp.d_out[k] = c->dims[l + 1]; tp.ld[k] = (int)round_up(c->dims[l + 1], 4);
-        tp.tiles_in[k] = (c->dims[l] + 31) / 32;
+        tp.tiles_in[k] = (c->dims[l] + 63) / 64;
         tp.first_tile[k] = tiles;
-        tiles += tp.tiles_in[k] * ((c->dims[l + 1] + 31) / 32);
+        tiles += tp.tiles_in[k] * ((c->dims[l + 1] + 63) / 64);
     }
     tp.n_layers = c->n_layers - 1;
     tp.first_tile[tp.n_layers] = tiles;

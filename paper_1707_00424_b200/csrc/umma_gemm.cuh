@@ -459,9 +459,22 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (EPI == UEPI_FWD_LAST) {
                     if (m_ok) {
                         float *o = p.outf + (long long)split * p.part_ss + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
+                        if ((p.outf_ld & 3) == 0) {          // rows start 16-byte aligned: four columns per store
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < p.N) o[j] = v[j];
+                            for (int j = 0; j < 32; j += 4) {
+                                if (nb + j + 3 < p.N) {
+                                    *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                                } else {
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k)
+                                        if (nb + j + k < p.N) o[j + k] = v[j + k];
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + j < p.N) o[j] = v[j];
+                        }
                     }
                 }
                 if (EPI == UEPI_WGRAD) {

@@ -349,7 +349,7 @@ input_split_kernel(const float *__restrict__ X, float *__restrict__ Xhi, float *
 }
 
 // Transposed hi/lo copy of the weights of the layers that have a data-gradient product (l >= 1):
-// W_l [d_out, d_in] fp32 inside a replica's vector -> W_l^T [d_in, ld] (ld = d_out rounded up to 4), 32 x 32 tiles.
+// W_l [d_out, d_in] fp32 inside a replica's vector -> W_l^T [d_in, ld] (ld = d_out rounded up to 4), 64 x 64 tiles, 16-byte accesses.
 struct TransposePlan {
     int n_layers;                                   // entries used (layers 1 .. of the network)
     long long w_off[PARLE_MAX_LAYERS], t_off[PARLE_MAX_LAYERS];
@@ -360,29 +360,33 @@ struct TransposePlan {
 __global__ void __launch_bounds__(256)
 split_transpose_kernel(const TransposePlan tp, const float *__restrict__ src, long long stride,
                        float *__restrict__ Thi, float *__restrict__ Tlo, long long t_stride) {
-    __shared__ float tile[32][33];
+    __shared__ float tile[64][65];
     const int g = blockIdx.y;
     int l = 0;
     while (l + 1 < tp.n_layers && (int)blockIdx.x >= tp.first_tile[l + 1]) ++l;
     const int t = blockIdx.x - tp.first_tile[l];
-    const int r0 = (t / tp.tiles_in[l]) * 32, c0 = (t % tp.tiles_in[l]) * 32;      // rows = d_out, columns = d_in
+    const int r0 = (t / tp.tiles_in[l]) * 64, c0 = (t % tp.tiles_in[l]) * 64;      // rows = d_out, columns = d_in
+    const int d_in = tp.d_in[l], d_out = tp.d_out[l], ld = tp.ld[l];
     const float *W = src + (long long)g * stride + tp.w_off[l];
-    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    const int q4 = (threadIdx.x % 16) * 4, rr = threadIdx.x / 16;                  // 16 threads x 4 floats = one 64-float row
 #pragma unroll
-    for (int r = ty; r < 32; r += 8) {
-        const int row = r0 + r, col = c0 + tx;
-        tile[r][tx] = (row < tp.d_out[l] && col < tp.d_in[l]) ? W[(long long)row * tp.d_in[l] + col] : 0.f;
+    for (int r = rr; r < 64; r += 16) {
+        const int row = r0 + r, col = c0 + q4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < d_out && col < d_in) v = *reinterpret_cast<const float4 *>(W + (long long)row * d_in + col);   // d_in % 4 == 0
+        tile[r][q4] = v.x; tile[r][q4 + 1] = v.y; tile[r][q4 + 2] = v.z; tile[r][q4 + 3] = v.w;
     }
     __syncthreads();
     float *oh = Thi + (long long)g * t_stride + tp.t_off[l], *ol = Tlo + (long long)g * t_stride + tp.t_off[l];
 #pragma unroll
-    for (int r = ty; r < 32; r += 8) {
-        const int col = c0 + r, row = r0 + tx;                                      // element (col of W, row of W)
-        if (col < tp.d_in[l] && row < tp.d_out[l]) {
-            float h, lo;
-            split_tf32(tile[tx][r], h, lo);
-            oh[(long long)col * tp.ld[l] + row] = h;
-            ol[(long long)col * tp.ld[l] + row] = lo;
+    for (int r = rr; r < 64; r += 16) {
+        const int col = c0 + r, row = r0 + q4;                // W column (row of W^T), first of four W rows
+        if (col < d_in && row < ld) {                         // ld % 4 == 0: the four are inside the padded row; rows >= d_out hold 0
+            float4 h, lo;
+            split_tf32(tile[q4][r], h.x, lo.x); split_tf32(tile[q4 + 1][r], h.y, lo.y);
+            split_tf32(tile[q4 + 2][r], h.z, lo.z); split_tf32(tile[q4 + 3][r], h.w, lo.w);
+            *reinterpret_cast<float4 *>(oh + (long long)col * ld + row) = h;
+            *reinterpret_cast<float4 *>(ol + (long long)col * ld + row) = lo;
         }
     }
 }
