@@ -11,7 +11,7 @@
 // 2^-24 of the running sum per instruction (1e-5 relative at K = 784, measured).  So the accumulator in tensor
 // memory only ever holds ONE 32-deep k-block (the eight small products first, then the four hi x hi ones); the
 // epilogue warps read it back after every k-block and add it to fp32 register accumulators with round-to-nearest.
-// Two accumulator buffers alternate, so the MMAs of the next k-block run meanwhile.
+// Four accumulator buffers rotate, so the MMAs of the next k-blocks run meanwhile.
 //
 // kind::tf32 takes K-major operands only (an MN-major descriptor yields zeros), so every operand exists in the
 // layout whose contiguous direction is the reduction index of the product that reads it:
@@ -37,6 +37,7 @@ constexpr int T3_BM = 128, T3_BK = 32;                     // 32 fp32 = one 128-
 constexpr int T3_A_BYTES = T3_BM * T3_BK * 4;              // 16 KiB per hi (or lo) tile of A
 constexpr int T3_RING_BYTES = 192 * 1024;
 constexpr int T3_EPI_WARPS = 8;
+constexpr int T3_ACC_BUFS = 4;                             // accumulator buffers of 128 columns: all 512 columns of tensor memory
 constexpr int T3_THREADS = 32 * (2 + T3_EPI_WARPS);
 
 template <int BN>
@@ -92,17 +93,17 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                    const T3Params p) {
     using SH = T3Shape<BN>;
     constexpr int STAGES = SH::STAGES, B_BYTES = SH::B_BYTES, STAGE_BYTES = SH::STAGE_BYTES;
-    constexpr uint32_t TMEM_COLS = 256;                                  // two accumulators of BN <= 128 columns
+    constexpr uint32_t TMEM_COLS = 128 * T3_ACC_BUFS;                   // accumulator buffers of BN <= 128 columns
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;
     uint8_t *ctl = smem_raw + (tiles_base - raw) + (size_t)STAGES * STAGE_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);                  // full[S], empty[S], tfull[2], tempty[2]
-    constexpr int NBARS = 2 * STAGES + 4;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);                  // full[S], empty[S], tfull[T3_ACC_BUFS], tempty[T3_ACC_BUFS]
+    constexpr int NBARS = 2 * STAGES + 2 * T3_ACC_BUFS;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 8 * NBARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
-    const uint32_t bar_tfull = bar_empty + 8 * STAGES, bar_tempty = bar_tfull + 16;
+    const uint32_t bar_tfull = bar_empty + 8 * STAGES, bar_tempty = bar_tfull + 8 * T3_ACC_BUFS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per_g = p.tiles_m * p.tiles_n;
@@ -111,7 +112,7 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, T3_EPI_WARPS); }
+        for (int s = 0; s < T3_ACC_BUFS; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, T3_EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -189,7 +190,7 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                     tc_commit(bar_empty + 8 * stage);
                     tc_commit(bar_tfull + 8 * acc);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                    if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                    if (++acc == T3_ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
                 }
             }
         }
@@ -224,7 +225,7 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                if (++acc == T3_ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
             }
             if (!ok) break;
 #pragma unroll
