@@ -137,10 +137,11 @@ def ncu_traffic(workload: str, kernel: str):
     return rec["bytes"]
 
 
-def algorithmic_bytes_per_round(cfg, stride, tf32_split=False):
+def algorithmic_bytes_per_round(cfg, stride, tf32_split=False, paired_z=True):
     """Bytes each kernel class has to move per Parle round (all n replicas), from the data it must
     touch once: parameter-state vectors at 4 B (fp32) or 2 B (bf16 copy) per element, plus GEMM operands.
-    tf32_split: the fp32 update also writes the tf32 hi/lo copy of y (8 B per element)."""
+    tf32_split: the fp32 update also writes the tf32 hi/lo copy of y (8 B per element).
+    paired_z: the fused bf16 kernel touches z on every other step only (parle_set_paired_z_update)."""
     n, B, L, dims = cfg.n, cfg.batch, cfg.L, cfg.dims
     nl = len(dims) - 1
     Pw = sum(dims[l] * dims[l + 1] for l in range(nl))
@@ -152,8 +153,10 @@ def algorithmic_bytes_per_round(cfg, stride, tf32_split=False):
     out["outer_mean"] = stride * (12 * n + 8)
     if bf:
         opnd = sum(2 * (act(l) + act(l + 1)) for l in range(nl))             # dH^T and H^T, bf16
-        # fused: read y, x, z (12 B), write y, z, bf16 copy (10 B); first step reads only x
-        out["wgrad_gemm_fused_update"] = n * (Pw * (22 * (L - 1) + 14) + opnd * L)
+        # fused: read y, x, z (12 B), write y, z, bf16 copy (10 B); first step reads only x (14 B); with Eq. (parle_z)
+        # applied two steps at a time the other steps alternate between 14 B (z untouched) and 22 B
+        pairs, single = ((L - 1) // 2, (L - 1) % 2) if paired_z else (0, L - 1)
+        out["wgrad_gemm_fused_update"] = n * (Pw * (14 + pairs * (14 + 22) + single * 22) + opnd * L)
         out["wgrad_gemm"] = n * L * (4 * Pw + opnd)
         out["fwd_gemm"] = n * L * (2 * Pw + sum(2 * act(l) + 4 * act(l + 1) for l in range(nl)))
         out["to_bf16"] = n * Pw * 6                                          # blocked bf16 weight copy from x, once per round
@@ -201,6 +204,8 @@ def run_ours(args):
         model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
     model.mean()
     model.set_round_graphs(bool(args.graphs))
+    if cfg.gemm_dtype == 1:
+        model.set_paired_z_update(bool(args.paired_z))
     sets = 2
     Xh, ch = make_round_inputs(cfg, sets)
     Xd, cd = torch.from_numpy(Xh).to(dev), torch.from_numpy(ch).to(dev)
@@ -274,7 +279,7 @@ def run_ours(args):
     shares = {k: {"ms_per_round": v[0] / K, "launches_per_round": v[1] / K, "share": v[0] / total_ms} for k, v in prof.items()}
     dom = max(prof, key=lambda k: prof[k][0])
     t3 = cfg.gemm_dtype == 0 and model.fp32_tensor_cores_active
-    alg = algorithmic_bytes_per_round(cfg, model.stride, tf32_split=t3)
+    alg = algorithmic_bytes_per_round(cfg, model.stride, tf32_split=t3, paired_z=bool(args.paired_z))
     rooflines = {}
     for k, (ms_k, cnt_k) in prof.items():
         if k not in alg:
@@ -318,7 +323,8 @@ def run_ours(args):
         "dtype": "bf16" if cfg.gemm_dtype == 1 else "f32", "data": "synthetic",
         "config": {"workload": f"{cfg.name}: n={cfg.n} replicas/GPU, MLP {'-'.join(map(str, cfg.dims))}, batch {cfg.batch}, L={cfg.L}, "
                                f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else ('fp32 (products as 3 x tf32 on the tensor cores)' if t3 else 'fp32 (FMA pipes)')}",
-                   "step": "one Parle round (L inner steps + outer step + replica mean)",
+                   "step": "one Parle round (L inner steps + outer step + replica mean)" +
+                           ("; z updated every other inner step with the two-step form of Eq. (parle_z)" if cfg.gemm_dtype == 1 and args.paired_z else ""),
                    "l2": "state + gradients per round >> 126 MB L2 (no flush needed)" if cfg.n * model.stride * 16 > 4e8 else "working set may be L2 resident",
                    "launch": "rounds replayed from CUDA graphs (same kernels, same order)" if args.graphs else "one launch per kernel",
                    "parallelism": f"{world} x {cfg.n} replicas, one all-reduce of xbar per round" if world > 1 else "single GPU"},
@@ -407,6 +413,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))
     ap.add_argument("--graphs", type=int, default=1, help="replay rounds from CUDA graphs (parle_set_round_graphs)")
+    ap.add_argument("--paired-z", type=int, default=1, help="bf16 workloads: Eq. (parle_z) two steps at a time inside a round (parle_set_paired_z_update)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -57,6 +57,7 @@ struct RoundKey {
     const void *inputs, *labels, *loss;
     float scal[7];                   // 1/gamma, 1/rho, alpha, eta, eta', weight decay, momentum
     int fused, wide_thr, shadow_is_x, fresh;   // L == 0: a single inner step (fresh = first of its round)
+    int paired_z, z_mode;            // whole rounds: Eq. (parle_z) in pairs or not; single steps: how this step treats z
     const void *ptrs[9];             // x, y, z, grad, xbar, workspace, vy, vx, stream
 };
 struct RoundGraph {
@@ -86,6 +87,8 @@ struct parle_ctx {
     cudaStream_t stream;
     int *status_host, *status_dev;
     bool round_open, fresh, shadow_is_x;
+    bool paired_z;                   // fused bf16 path, whole rounds: Eq. (parle_z) applied two steps at a time
+    int z_mode;                      // how the next fused step treats z (WU_Z_*); set per step by the round drivers
     bool fused_update;               // bf16 path: apply Eq. (parle_y)/(parle_z) inside the weight-gradient GEMM
     int steps_in_round;
     long long launches;
@@ -763,16 +766,23 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     p.sched = ws_ptr<int>(c, w.sched);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     prof_begin(c, KC_WGRAD_UPDATE);
+    const int zm = c->fresh ? WU_Z_SINGLE : c->z_mode;
+    if (mom) { p.v = c->vy; p.mu = c->momentum; }
+    const WuMaps &maps = mom ? c->wu_maps_mom : c->wu_maps;
+#define PARLE_WU_LAUNCH(FIRST, SH, MOM, ZM) \
+    umma_wgrad_update_kernel<FIRST, SH, MOM, ZM><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p)
     if (mom) {
-        p.v = c->vy; p.mu = c->momentum;
-        if (c->fresh)
-            umma_wgrad_update_kernel<true, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(c->wu_maps_mom, p);
-        else
-            umma_wgrad_update_kernel<false, WuMomentum, true><<<grid, WuMomentum::THREADS, WuMomentum::SMEM_BYTES, c->stream>>>(c->wu_maps_mom, p);
-    } else if (c->fresh)
-        umma_wgrad_update_kernel<true, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(c->wu_maps, p);
-    else
-        umma_wgrad_update_kernel<false, WuDefault><<<grid, WuDefault::THREADS, WuDefault::SMEM_BYTES, c->stream>>>(c->wu_maps, p);
+        if (c->fresh) PARLE_WU_LAUNCH(true, WuMomentum, true, WU_Z_SINGLE);
+        else if (zm == WU_Z_SKIP) PARLE_WU_LAUNCH(false, WuMomentum, true, WU_Z_SKIP);
+        else if (zm == WU_Z_DOUBLE) PARLE_WU_LAUNCH(false, WuMomentum, true, WU_Z_DOUBLE);
+        else PARLE_WU_LAUNCH(false, WuMomentum, true, WU_Z_SINGLE);
+    } else {
+        if (c->fresh) PARLE_WU_LAUNCH(true, WuDefault, false, WU_Z_SINGLE);
+        else if (zm == WU_Z_SKIP) PARLE_WU_LAUNCH(false, WuDefault, false, WU_Z_SKIP);
+        else if (zm == WU_Z_DOUBLE) PARLE_WU_LAUNCH(false, WuDefault, false, WU_Z_DOUBLE);
+        else PARLE_WU_LAUNCH(false, WuDefault, false, WU_Z_SINGLE);
+    }
+#undef PARLE_WU_LAUNCH
     PARLE_LAUNCHED(c);
     TailPlan tp = {};
     tp.n_layers = nl; tp.batch = B;
@@ -871,6 +881,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
     }
     if (c->t3_t_stride == 0) c->t3_t_stride = 32;
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
+    c->paired_z = true;
     c->wide_tiles_per_sm = 4;
     c->last_ksplit = 1;
     if (c->fused_update) {
@@ -944,10 +955,13 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, UB_BLOCKED_K>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, UB_BLOCKED_K>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, UB_ROWMAJOR_K>()));
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false, WuDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuDefault::SMEM_BYTES));
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<true, WuMomentum, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuMomentum::SMEM_BYTES));
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<false, WuMomentum, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WuMomentum::SMEM_BYTES));
+#define PARLE_WU_SMEM(FIRST, SH, MOM, ZM) \
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES))
+        PARLE_WU_SMEM(true, WuDefault, false, WU_Z_SINGLE); PARLE_WU_SMEM(false, WuDefault, false, WU_Z_SINGLE);
+        PARLE_WU_SMEM(false, WuDefault, false, WU_Z_SKIP); PARLE_WU_SMEM(false, WuDefault, false, WU_Z_DOUBLE);
+        PARLE_WU_SMEM(true, WuMomentum, true, WU_Z_SINGLE); PARLE_WU_SMEM(false, WuMomentum, true, WU_Z_SINGLE);
+        PARLE_WU_SMEM(false, WuMomentum, true, WU_Z_SKIP); PARLE_WU_SMEM(false, WuMomentum, true, WU_Z_DOUBLE);
+#undef PARLE_WU_SMEM
         c->mom_maps = false;
         PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, UB_BLOCKED_MN>()));
         PARLE_TRY(build_tensor_maps(c));
@@ -1073,6 +1087,7 @@ static RoundKey make_round_key(const parle_ctx *c, int L, const void *in, const 
     const float sc[7] = {c->inv_gamma, c->inv_rho, c->alpha, c->eta, c->eta_prime, c->weight_decay, c->momentum};
     memcpy(k.scal, sc, sizeof(sc));
     k.fused = c->fused_update; k.wide_thr = c->wide_tiles_per_sm; k.shadow_is_x = c->shadow_is_x; k.fresh = c->fresh;
+    k.paired_z = c->paired_z; k.z_mode = c->z_mode;
     const void *pt[9] = {c->buf.x, c->buf.y, c->buf.z, c->buf.grad, c->buf.xbar, c->buf.workspace, c->vy, c->vx, c->stream};
     memcpy(k.ptrs, pt, sizeof(pt));
     return k;
@@ -1178,12 +1193,26 @@ int parle_set_round_graphs(parle_ctx *c, int on) {
     return PARLE_OK;
 }
 
+// How step l (0-based) of an L-step round treats z when Eq. (parle_z) is applied two steps at a time (fused bf16
+// path): the first step forms z from x; the remaining L - 1 steps go in (skip, two-step) pairs, with a one-step
+// update at the end when L - 1 is odd.
+static int paired_z_mode(const parle_ctx *c, int l, int L) {
+    if (!c->paired_z || !c->fused_update || c->gemm_dtype != PARLE_GEMM_BF16 || l == 0) return WU_Z_SINGLE;
+    const int rest = L - 1, idx = l - 1;
+    if ((rest & 1) && idx == rest - 1) return WU_Z_SINGLE;
+    return (idx & 1) ? WU_Z_DOUBLE : WU_Z_SKIP;
+}
+
 static int round_direct(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
     PARLE_TRY(parle_round_begin(c));
     const size_t nb = (size_t)c->n * c->batch;
-    for (int l = 0; l < L; ++l)
-        PARLE_TRY(parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
-                                   loss_out ? loss_out + (size_t)l * c->n : nullptr));
+    for (int l = 0; l < L; ++l) {
+        c->z_mode = paired_z_mode(c, l, L);
+        const int rc = parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
+                                        loss_out ? loss_out + (size_t)l * c->n : nullptr);
+        c->z_mode = WU_Z_SINGLE;
+        PARLE_TRY(rc);
+    }
     return parle_outer_step(c);
 }
 
@@ -1219,12 +1248,16 @@ int parle_round_host(parle_ctx *c, int L, const float *inputs_host, const int32_
         if (l + 1 < L) PARLE_TRY(upload(l + 1));
         PARLE_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
         float *dloss = ws_ptr<float>(c, c->ws.stage_loss[b]);
+        c->z_mode = paired_z_mode(c, l, L);
+        int rc;
         if (c->graphs_on && !c->prof_on)       // the step's kernels as one cached graph (staging buffers have fixed addresses)
-            PARLE_TRY(round_graphed(c, 0, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
-                                    loss_out_host ? dloss : nullptr));
+            rc = round_graphed(c, 0, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
+                               loss_out_host ? dloss : nullptr);
         else
-            PARLE_TRY(parle_inner_step(c, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
-                                       loss_out_host ? dloss : nullptr));
+            rc = parle_inner_step(c, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
+                                  loss_out_host ? dloss : nullptr);
+        c->z_mode = WU_Z_SINGLE;
+        PARLE_TRY(rc);
         if (loss_out_host)
             PARLE_CUDA(c, cudaMemcpyAsync(loss_out_host + (size_t)l * c->n, dloss, c->n * sizeof(float),
                                           cudaMemcpyDeviceToHost, c->stream));
@@ -1244,6 +1277,13 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->fused_update = on != 0;
+    return PARLE_OK;
+}
+
+int parle_set_paired_z_update(parle_ctx *c, int on) {
+    if (!c) return PARLE_EINVAL;
+    if (c->round_open) return PARLE_ESTATE;
+    c->paired_z = on != 0;
     return PARLE_OK;
 }
 

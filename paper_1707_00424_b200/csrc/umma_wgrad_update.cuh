@@ -33,6 +33,13 @@
 // the other roles read it from there.  The last CTA to leave resets the counter
 // pair, so consecutive launches on one stream can share it.  Which CTA runs a
 // tile does not change what is computed for it: results stay bit-identical.
+//
+// Eq. (parle_z) two steps at a time (ZMODE).  z is only needed by the outer step, and
+//     z_{k+2} = alpha z_{k+1} + (1-alpha) y_{k+2} = alpha^2 z_k + (1-alpha) (alpha y_{k+1} + y_{k+2})
+// needs, besides z_k, exactly the two y values the kernel of step k+2 holds anyway (the y it reads and the y it
+// writes).  So inside a whole round z is read and written every other step only: ZMODE 1 leaves z alone (14 bytes
+// per weight instead of 22), ZMODE 2 applies the two-step form, ZMODE 0 the one-step form (single steps, and the last
+// step of a round with an even number of steps).  Same recurrence, different fp32 rounding of z (1e-7 relative).
 // All waits are bounded.
 #pragma once
 
@@ -108,7 +115,9 @@ struct WuMaps {
 
 // MOM: Nesterov momentum on the y step (see inner_update_kernel): v <- mu v + d, y <- y - eta' (d + mu v),
 // v = 0 at the start of a round (FIRST: v is only written).
-template <bool FIRST, class SH, bool MOM = false>
+// ZMODE (ignored when FIRST): 0 = z <- alpha z + (1-alpha) y_new; 1 = z untouched; 2 = z <- alpha^2 z + (1-alpha)(alpha y_old + y_new).
+constexpr int WU_Z_SINGLE = 0, WU_Z_SKIP = 1, WU_Z_DOUBLE = 2;
+template <bool FIRST, class SH, bool MOM = false, int ZMODE = WU_Z_SINGLE>
 __global__ void __launch_bounds__(SH::THREADS, 1)
 umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_constant__ WgradUpdateParams p) {
     constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
@@ -250,11 +259,12 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     if (!mbar_wait(bar_sempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t dst = st_base + stage * WU_STATE_BYTES;
                     const uint32_t fb = bar_sfull + 8 * stage;
-                    mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES);   // STATE_BYTES counts v when MOM
+                    constexpr bool LOAD_Z = !FIRST && ZMODE != WU_Z_SKIP;
+                    mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES - (LOAD_Z ? 0 : WU_ARRAY_BYTES));   // STATE_BYTES counts v when MOM
                     tma_load_3d(dst, &maps.x[l], fb, m0, nb, g);
                     if (!FIRST) {
                         tma_load_3d(dst + WU_ARRAY_BYTES, &maps.y[l], fb, m0, nb, g);
-                        tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &maps.z[l], fb, m0, nb, g);
+                        if (LOAD_Z) tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &maps.z[l], fb, m0, nb, g);
                         if (MOM) tma_load_3d(dst + 3 * WU_ARRAY_BYTES, &maps.v[l], fb, m0, nb, g);
                     }
                     if (++stage == WU_STATE_STAGES) { stage = 0; phase ^= 1u; }
@@ -272,8 +282,9 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
         // ------------------------------------------------ epilogue groups
         const int q = warp & 3;                              // tensor-memory lane quarter of this warp
         const int grp = (warp - 3) >> 2;                     // rows grp*RPG .. of every chunk
-        const float one_m_alpha = 1.0f - p.alpha;
+        const float one_m_alpha = 1.0f - p.alpha, alpha_sq = p.alpha * p.alpha;
         const float neg_eta_p = -p.eta_p;
+        constexpr bool USE_Z = FIRST || ZMODE != WU_Z_SKIP;
         int acc = 0; uint32_t acc_phase = 0;
         int stage = 0; uint32_t sphase = 0;                  // state ring position: every warp walks every chunk
         float chk = 0.f;                                     // 0 * y summed: turns NaN as soon as a y is NaN or Inf
@@ -319,7 +330,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     xv[j] = sx[j * UM_BM];
                     if (!FIRST) {
                         yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
-                        zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
+                        if (USE_Z) zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                         if (MOM) vv[j] = sx[3 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                     }
                 }
@@ -335,7 +346,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                 float *yr = yp, *zr = zp, *vr = vp;
                 __nv_bfloat16 *sr = sp;
                 auto update_row = [&](int j) {
-                    const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : zv[j];
+                    const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : (USE_Z ? zv[j] : 0.f);
                     float d = fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j])));
                     if (MOM) {
                         const float vn = FIRST ? d : fmaf(p.mu, vv[j], d);      // v = 0 before the first step of a round
@@ -343,10 +354,13 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                         d = fmaf(p.mu, vn, d);
                     }
                     const float yn = fmaf(neg_eta_p, d, yo);
-                    const float zn = fmaf(p.alpha, zo, one_m_alpha * yn);
                     chk = fmaf(yn, 0.f, chk);
                     *yr = yn;
-                    *zr = zn;
+                    if (USE_Z) {
+                        const float zn = (!FIRST && ZMODE == WU_Z_DOUBLE) ? fmaf(alpha_sq, zo, one_m_alpha * fmaf(p.alpha, yo, yn))
+                                                                           : fmaf(p.alpha, zo, one_m_alpha * yn);
+                        *zr = zn;
+                    }
                     *sr = __float2bfloat16_rn(yn);
                 };
                 if (rows >= RPG) {                           // common case: no per-row bounds checks

@@ -35,6 +35,7 @@ def make(cfg, fused=None, t3=None, **over):
     m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, **hyper).alloc(DEV)
     if fused is not None and cfg.gemm_dtype == pb.GEMM_BF16:
         m.set_fused_update(fused)
+        m.set_paired_z_update(False)      # tests that name the path compare it bit for bit with the other one: z step by step in both
     if t3 is not None and cfg.gemm_dtype == pb.GEMM_FP32:
         m.set_fp32_tensor_cores(t3)
         assert m.fp32_tensor_cores_active == (t3 == 2)
@@ -621,7 +622,40 @@ def test_graph_rounds_equal_plain_rounds(gemm_dtype, dims):
         for r in range(3):
             m.round_host(cfg.L, Xh, ch, lh)
         torch.cuda.synchronize()
-        assert m.round_graph_count == (3 if graphs else -1)
+        # step graphs: first step / later step with either staging buffer; on the fused bf16 path the later steps are
+        # "z untouched" (odd steps, buffer 1), "two-step z" (even steps, buffer 0) and the closing one-step update
+        assert m.round_graph_count == ((3 if gemm_dtype == 0 else 4) if graphs else -1)
         outs.append((m.x.clone(), m.xbar.clone(), lh.clone()))
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("L", [1, 2, 5, 6])
+@pytest.mark.parametrize("mu", [0.0, 0.9])
+def test_paired_z_update_is_the_same_recurrence_bf16(L, mu):
+    """Whole rounds apply Eq. (parle_z) two steps at a time (z touched every other step).  Against rounds that update
+    z at every step: y is bit-identical (z does not enter it), z and x agree to fp32 rounding, for odd and even L."""
+    cfg = si.C1.scaled(name="pairz", n=3, dims=(200, 328, 136, 101), batch=136, gemm_dtype=1, L=L)
+    res = []
+    for paired in (True, False):
+        m, *_ = make(cfg)
+        m.set_paired_z_update(paired)
+        if mu:
+            m.set_momentum(mu)
+        snaps = []
+        for r in range(2):
+            X, c = si.round_batches(cfg, r)
+            m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV))
+            torch.cuda.synchronize()
+            assert m.status() == 0
+            snaps.append([t.cpu().numpy().astype(np.float64) for t in (m.y, m.z, m.x, m.xbar)])
+        res.append(snaps)
+    (y1, z1, x1, b1), (y0, z0, x0, b0) = res[0][0], res[1][0]
+    assert np.array_equal(y1, y0)                    # first round: the same y trajectory, bit for bit
+    assert rel_l2(z1, z0) < 5e-7 and rel_l2(x1, x0) < 5e-7 and rel_l2(b1, b0) < 5e-7
+    if L > 2:
+        assert not np.array_equal(z1, z0)            # the two-step form did run
+    # second round: it starts from x values that differ in the last bit, a few of which round to another bf16 operand
+    # (and momentum amplifies that): a tenth of the bf16 parity bound
+    for a, b in zip(res[0][1], res[1][1]):
+        assert rel_l2(a, b) < 2e-3
