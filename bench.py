@@ -112,13 +112,14 @@ def dense_to_padded(model, cfg, replica_layers):
     return out
 
 
-# DRAM bytes per launch (mean over the four launches of an inner step) of the dominant kernel from the committed
-# ncu capture (profiles/ncu_full_gemms_and_fused_update_C3.md), valid only while the kernel source is unchanged.
+# DRAM bytes per launch of the dominant kernel from the committed ncu capture
+# (profiles/ncu_full_gemms_and_fused_update_C3.md), valid only while the kernel source is unchanged.
 NCU_TRAFFIC = {("C3", "wgrad_gemm_fused_update"): {
-    # dram__bytes_read.sum + dram__bytes_write.sum, mean over the four layers' launches of one inner step
-    "bytes": 2479.96e6 / 4,
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch (all layers, all replicas): mean of the two variants
+    # that alternate inside a round, "z untouched" (984.4 + 663.6 MB) and "two-step z" (1462.5 + 1135.8 MB)
+    "bytes": (984.443e6 + 663.629e6 + 1462.463e6 + 1135.813e6) / 2,
     "sources": ("paper_1707_00424_b200/csrc/umma_wgrad_update.cuh", "paper_1707_00424_b200/csrc/umma_gemm.cuh"),
-    "sources_sha256_16": "9d3a29e7efb49222"}}
+    "sources_sha256_16": "72d91c0118922456"}}
 
 
 def sources_digest(sources):
@@ -134,7 +135,7 @@ def ncu_traffic(workload: str, kernel: str):
     rec = NCU_TRAFFIC.get((workload, kernel))
     if not rec or sources_digest(rec["sources"]) != rec["sources_sha256_16"]:
         return None             # no capture, or the kernel changed since the counters were taken
-    return rec["bytes"]
+    return rec["bytes"]         # (taken with the default settings: z updated every other step)
 
 
 def algorithmic_bytes_per_round(cfg, stride, tf32_split=False, paired_z=True):
@@ -286,7 +287,7 @@ def run_ours(args):
             continue
         ach = alg[k] * K / (ms_k * 1e-3) / 1e9          # bytes of K rounds / device time of the class over K rounds
         rooflines[k] = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, k),
+                        "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, k) if args.paired_z else None,
                         "peak_source": peaks["source"], "bytes_per_launch": alg[k] * K / cnt_k,
                         "ms_per_launch": ms_k / cnt_k, "launches_per_round": cnt_k / K}
     flops = gemm_flops_per_round(cfg)

@@ -38,6 +38,7 @@ struct Workspace {
     int dh_ld[PARLE_MAX_LAYERS];       // row pitch of dhb[l] (d_{l+1} rounded up to 8)
     size_t row_loss;                   // [n,B] fp32
     // fp32 mode on the tensor cores (3 x tf32): tf32-exact hi/lo pairs, index [0] = hi, [1] = lo
+    size_t t3_logits;                  // fp32 logits [n, B, C] x t3_ksplit partial sums
     size_t w_split[2];                 // parameters [n, stride]
     size_t wT_split[2];                // transposed weights of layers >= 1, [n, t3_t_stride]
     size_t xs[2], xT[2];               // inputs [n, B, d_0] and transposed [n, d_0, B]
@@ -102,6 +103,7 @@ struct parle_ctx {
     bool t3_shapes_ok;               // widths and batch are multiples of 4 (16-byte rows for TMA)
     bool t3_ready;                   // tensor maps exist for the bound buffers (needs an sm_100 device)
     size_t t3_t_off[PARLE_MAX_LAYERS], t3_t_stride;   // transposed weight copy: W_l^T [d_in, ld_l] of layers >= 1 inside a replica's copy
+    int t3_ksplit;                   // split-K factor of the last forward layer on this path (1 = off)
     int t3_bn_fwd[PARLE_MAX_LAYERS], t3_bn_dg[PARLE_MAX_LAYERS], t3_bn_wg[PARLE_MAX_LAYERS];   // tile widths (64 or 128)
     CUtensorMap t3_fa[PARLE_MAX_LAYERS][2], t3_fb[PARLE_MAX_LAYERS][2];    // forward operands, hi / lo
     CUtensorMap t3_da[PARLE_MAX_LAYERS][2], t3_db[PARLE_MAX_LAYERS][2];    // data gradient
@@ -168,6 +170,7 @@ void plan_workspace(parle_ctx *c) {
         for (int l = 0; l < nl; ++l) w.act[l] = take(n * B * c->dims[l + 1] * sizeof(float));
         for (int l = 0; l < nl; ++l) w.dact[l] = take(n * B * c->dims[l + 1] * sizeof(float));
         if (c->t3_shapes_ok) {
+            w.t3_logits = take(n * B * C * sizeof(float) * (size_t)c->t3_ksplit);
             for (int h = 0; h < 2; ++h) {
                 w.w_split[h] = take(n * c->stride * sizeof(float));
                 w.wT_split[h] = take(n * c->t3_t_stride * sizeof(float));
@@ -339,7 +342,7 @@ int launch_t3_bn(parle_ctx *c, int cls, const CUtensorMap *a, const CUtensorMap 
     p.tiles_m = (p.M + T3_BM - 1) / T3_BM;
     p.tiles_n = (p.N + BN - 1) / BN;
     p.status = c->status_dev;
-    const int tiles = p.groups * p.tiles_m * p.tiles_n;
+    const int tiles = p.groups * p.tiles_m * p.tiles_n * ((EPI == T3_FWD_LAST && p.ksplit > 1) ? p.ksplit : 1);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     prof_begin(c, cls);
     umma_tf32x3_kernel<EPI, BN><<<grid, T3_THREADS, T3Shape<BN>::SMEM_BYTES, c->stream>>>(a[0], a[1], b[0], b[1], p);
@@ -583,15 +586,17 @@ int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labe
             p.outT_gs = (long long)B * dout; p.outT_ld = B;
             PARLE_TRY(launch_t3<T3_FWD_HIDDEN>(c, KC_FWD_GEMM, c->t3_bn_fwd[l], c->t3_fa[l], c->t3_fb[l], p));
         } else {
-            p.outf = ws_ptr<float>(c, w.act[l]); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
+            p.outf = ws_ptr<float>(c, w.t3_logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
+            p.ksplit = c->t3_ksplit; p.part_ss = (long long)n * B * dout;
             PARLE_TRY(launch_t3<T3_FWD_LAST>(c, KC_FWD_GEMM, c->t3_bn_fwd[l], c->t3_fa[l], c->t3_fb[l], p));
         }
     }
     const int C = c->dims[nl], rows = n * B;
     prof_begin(c, KC_SOFTMAX_CE);
     softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
-        ws_ptr<float>(c, w.act[nl - 1]), labels, nullptr, nullptr, nullptr, ws_ptr<float>(c, w.row_loss), rows, B, C, 0,
-        c->status_dev, 1, 0, nullptr, 0, ws_ptr<float>(c, w.dhT[nl - 1][0]), ws_ptr<float>(c, w.dhT[nl - 1][1]),
+        ws_ptr<float>(c, w.t3_logits), labels, nullptr, nullptr, nullptr, ws_ptr<float>(c, w.row_loss), rows, B, C, 0,
+        c->status_dev, c->t3_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
+        ws_ptr<float>(c, w.dhT[nl - 1][0]), ws_ptr<float>(c, w.dhT[nl - 1][1]),
         ws_ptr<float>(c, w.dhs[nl - 1][0]), ws_ptr<float>(c, w.dhs[nl - 1][1]), (int)round_up(C, 4));
     PARLE_LAUNCHED(c);
     if (loss_out) {
@@ -616,7 +621,7 @@ int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labe
             d.out_gs = (long long)B * din; d.out_ld = din;      // d_in % 4 == 0: no padding
             d.outT_hi = ws_ptr<float>(c, w.dhT[l - 1][0]); d.outT_lo = ws_ptr<float>(c, w.dhT[l - 1][1]);
             d.outT_gs = (long long)B * din; d.outT_ld = B;
-            d.mask_hi = ws_ptr<float>(c, w.hT[l - 1][0]); d.mask_lo = ws_ptr<float>(c, w.hT[l - 1][1]);
+            d.mask_hi = ws_ptr<float>(c, w.hT[l - 1][0]);
             d.mask_gs = (long long)B * din; d.mask_ld = B;
             PARLE_TRY(launch_t3<T3_DGRAD>(c, KC_DGRAD_GEMM, c->t3_bn_dg[l], c->t3_da[l], c->t3_db[l], d));
         }
@@ -880,6 +885,18 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         c->t3_t_stride = round_up(c->t3_t_stride + (size_t)c->dims[l] * round_up(c->dims[l + 1], 4), 32);
     }
     if (c->t3_t_stride == 0) c->t3_t_stride = 32;
+    c->t3_ksplit = 1;
+    if (c->t3_shapes_ok) {
+        // the last forward layer usually has one tile per replica: split its k-blocks over several CTAs (partial sums,
+        // added up with the bias by the softmax kernel in fixed order)
+        const int nl = c->n_layers;
+        const int tiles = c->n * ((c->batch + 127) / 128) * ((c->dims[nl] + 63) / 64);
+        const int num_kb = (c->dims[nl - 1] + 31) / 32;
+        int s = 148 / (tiles > 0 ? tiles : 1);
+        if (s > 8) s = 8;
+        if (s > num_kb / 2) s = num_kb / 2;
+        if (s >= 2) c->t3_ksplit = s;
+    }
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
     c->paired_z = true;
     c->wide_tiles_per_sm = 4;
@@ -1417,7 +1434,7 @@ int parle_debug_buffer(const parle_ctx *c, int kind, int layer, size_t *byte_off
     const bool bf = c->gemm_dtype == PARLE_GEMM_BF16;
     const size_t es = bf ? 2 : 4;
     if (kind == PARLE_DBG_LOGITS) {
-        *byte_offset = bf ? w.logits : w.act[nl - 1];
+        *byte_offset = bf ? w.logits : (use_t3(c) ? w.t3_logits : w.act[nl - 1]);
         *bytes = nB * c->dims[nl] * 4;
         return PARLE_OK;
     }

@@ -63,7 +63,11 @@ struct T3Params {
     float *out_hi, *out_lo; long long out_gs; int out_ld;          // row-major pair (out_ld % 4 == 0)
     float *outT_hi, *outT_lo; long long outT_gs; int outT_ld;       // transposed pair
     float *outf; long long outf_gs; int outf_ld;
-    const float *mask_hi, *mask_lo; long long mask_gs; int mask_ld;   // transposed pair of the layer input: [n * mask_ld + m]
+    const float *mask_hi; long long mask_gs; int mask_ld;   // hi part of the layer input, transposed: [n * mask_ld + m]
+                                                             // (rounding to tf32 keeps the sign: H > 0 exactly when its hi part is)
+    // split-K (T3_FWD_LAST only): each tile's k-blocks are divided among ksplit work items, each of which stores its raw
+    // partial sums (no bias) at outf + split * part_ss; the softmax kernel adds them up in fixed order
+    int ksplit; long long part_ss;
     int *status;
 };
 
@@ -107,8 +111,9 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per_g = p.tiles_m * p.tiles_n;
-    const int total_tiles = p.groups * per_g;
     const int num_kb = (p.K + T3_BK - 1) / T3_BK;
+    const int ksplit = (EPI == T3_FWD_LAST && p.ksplit > 1) ? p.ksplit : 1;
+    const int total_items = p.groups * per_g * ksplit;     // work item = (tile, k range)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -138,9 +143,11 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+                const int t = it / ksplit, split = it - t * ksplit;
+                const int kb_lo = split * num_kb / ksplit, kb_hi = (split + 1) * num_kb / ksplit;
                 int g, m0, n0; coords(t, g, m0, n0);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sa = tiles_base + stage * STAGE_BYTES, sb = sa + 2 * T3_A_BYTES;
                     const uint32_t fb = bar_full + 8 * stage;
@@ -167,8 +174,10 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_tf32(false, false, BN);
             int stage = 0; uint32_t phase = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                for (int kb = 0; kb < num_kb; ++kb) {
+            for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+                const int split = it % ksplit;
+                const int kb_lo = split * num_kb / ksplit, kb_hi = (split + 1) * num_kb / ksplit;
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     // one k-block per accumulator buffer
                     if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
@@ -201,7 +210,9 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
         constexpr int CPW = BN / 64;                         // 32-column chunks per warp
         int acc = 0; uint32_t acc_phase = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        for (int it = blockIdx.x; it < total_items && ok; it += gridDim.x) {
+            const int t = it / ksplit, split = it - t * ksplit;
+            const int kb_lo = split * num_kb / ksplit, kb_hi = (split + 1) * num_kb / ksplit;
             int g, m0, n0; coords(t, g, m0, n0);
             const int m = m0 + q * 32 + lane;                // accumulator row of this thread
             const bool m_ok = m < p.M;
@@ -210,7 +221,7 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
             for (int cc = 0; cc < CPW; ++cc)
 #pragma unroll
                 for (int j = 0; j < 32; ++j) sum[cc][j] = 0.f;
-            for (int kb = 0; kb < num_kb; ++kb) {
+            for (int kb = kb_lo; kb < kb_hi; ++kb) {
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
@@ -235,14 +246,16 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                 const float (&r)[32] = sum[cc];
                 float bias_lane = 0.f;
                 if (EPI == T3_FWD_HIDDEN || EPI == T3_FWD_LAST)
-                    bias_lane = (nb + lane < p.N) ? __ldg(p.bias + (long long)g * p.bias_gs + nb + lane) : 0.f;
+                    bias_lane = (nb + lane < p.N && ksplit == 1) ? __ldg(p.bias + (long long)g * p.bias_gs + nb + lane) : 0.f;
                 if (EPI == T3_FWD_HIDDEN || EPI == T3_DGRAD) {
                     float *th = p.outT_hi + (long long)g * p.outT_gs + (long long)nb * p.outT_ld + m;
                     float *tl = p.outT_lo + (long long)g * p.outT_gs + (long long)nb * p.outT_ld + m;
-                    const float *mh = nullptr, *ml = nullptr;
+                    float mk[32];                                        // ReLU mask source: all 32 loads in flight at once
                     if (EPI == T3_DGRAD) {
-                        mh = p.mask_hi + (long long)g * p.mask_gs + (long long)nb * p.mask_ld + m;
-                        ml = p.mask_lo + (long long)g * p.mask_gs + (long long)nb * p.mask_ld + m;
+                        const float *mh = p.mask_hi + (long long)g * p.mask_gs + (long long)nb * p.mask_ld + m;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            mk[j] = (m_ok && nb + j < p.N) ? __ldg(mh + (long long)j * p.mask_ld) : 0.f;
                     }
                     float hi[32], lo[32];
 #pragma unroll
@@ -251,10 +264,7 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                         if (EPI == T3_FWD_HIDDEN) v = fmaxf(v + __shfl_sync(0xffffffffu, bias_lane, j), 0.f);
                         hi[j] = 0.f; lo[j] = 0.f;
                         if (m_ok && nb + j < p.N) {
-                            if (EPI == T3_DGRAD) {
-                                const float h = __ldg(mh + (long long)j * p.mask_ld), l = __ldg(ml + (long long)j * p.mask_ld);
-                                if (!(h > 0.f || l > 0.f)) v = 0.f;
-                            }
+                            if (EPI == T3_DGRAD && !(mk[j] > 0.f)) v = 0.f;
                             split_tf32(v, hi[j], lo[j]);
                             th[(long long)j * p.outT_ld] = hi[j];         // lanes = consecutive batch rows: coalesced
                             tl[(long long)j * p.outT_ld] = lo[j];
@@ -273,7 +283,7 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                     }
                 }
                 if (EPI == T3_FWD_LAST) {
-                    float *o = p.outf + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
+                    float *o = p.outf + (long long)split * p.part_ss + (long long)g * p.outf_gs + (long long)m * p.outf_ld + nb;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const float v = r[j] + __shfl_sync(0xffffffffu, bias_lane, j);
