@@ -150,7 +150,9 @@ def algorithmic_bytes_per_round(cfg, stride, tf32_split=False, paired_z=True):
     act = lambda l: B * dims[l]                          # elements of one replica's activation at level l
     out = {}
     # separate update: read g, y, x, z, write y, z (+2 B bf16 copy); first step of a round reads x for y and z
-    out["inner_update"] = n * stride * ((24 + (2 if bf else 0) + (8 if tf32_split else 0)) * L - 8)
+    # with Eq. (parle_z) applied two steps at a time, half of the later steps leave z alone (8 B less)
+    skipped = (L - 1) // 2 if paired_z else 0
+    out["inner_update"] = n * stride * ((24 + (2 if bf else 0) + (8 if tf32_split else 0)) * L - 8 - 8 * skipped)
     out["outer_mean"] = stride * (12 * n + 8)
     if bf:
         opnd = sum(2 * (act(l) + act(l + 1)) for l in range(nl))             # dH^T and H^T, bf16
@@ -205,8 +207,7 @@ def run_ours(args):
         model.x.copy_(torch.from_numpy(dense_to_padded(model, cfg, [si.init_replica(cfg, a) for a in range(cfg.n)])))
     model.mean()
     model.set_round_graphs(bool(args.graphs))
-    if cfg.gemm_dtype == 1:
-        model.set_paired_z_update(bool(args.paired_z))
+    model.set_paired_z_update(bool(args.paired_z))
     sets = 2
     Xh, ch = make_round_inputs(cfg, sets)
     Xd, cd = torch.from_numpy(Xh).to(dev), torch.from_numpy(ch).to(dev)
@@ -325,7 +326,7 @@ def run_ours(args):
         "config": {"workload": f"{cfg.name}: n={cfg.n} replicas/GPU, MLP {'-'.join(map(str, cfg.dims))}, batch {cfg.batch}, L={cfg.L}, "
                                f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else ('fp32 (products as 3 x tf32 on the tensor cores)' if t3 else 'fp32 (FMA pipes)')}",
                    "step": "one Parle round (L inner steps + outer step + replica mean)" +
-                           ("; z updated every other inner step with the two-step form of Eq. (parle_z)" if cfg.gemm_dtype == 1 and args.paired_z else ""),
+                           ("; z updated every other inner step with the two-step form of Eq. (parle_z)" if args.paired_z else ""),
                    "l2": "state + gradients per round >> 126 MB L2 (no flush needed)" if cfg.n * model.stride * 16 > 4e8 else "working set may be L2 resident",
                    "launch": "rounds replayed from CUDA graphs (same kernels, same order)" if args.graphs else "one launch per kernel",
                    "parallelism": f"{world} x {cfg.n} replicas, one all-reduce of xbar per round" if world > 1 else "single GPU"},
@@ -414,7 +415,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))
     ap.add_argument("--graphs", type=int, default=1, help="replay rounds from CUDA graphs (parle_set_round_graphs)")
-    ap.add_argument("--paired-z", type=int, default=1, help="bf16 workloads: Eq. (parle_z) two steps at a time inside a round (parle_set_paired_z_update)")
+    ap.add_argument("--paired-z", type=int, default=1, help="Eq. (parle_z) two steps at a time inside a round (parle_set_paired_z_update)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

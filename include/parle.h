@@ -178,13 +178,14 @@ int parle_round_host(parle_ctx *ctx, int L, const float *inputs_host, const int3
  * fp32 rounding).  EUNSUPPORTED on the fp32 path, ESTATE in the middle of a round. */
 int parle_set_fused_update(parle_ctx *ctx, int on);
 
-/* bf16 path with the fused update, whole rounds only (parle_round, parle_round_host).  on (the default): z^a, which
+/* Whole rounds only (parle_round, parle_round_host).  on (the default): z^a, which
  * only the outer step reads, is updated every other inner step, with Eq. (parle_z) applied twice at once,
  *     z_{k+2} = alpha^2 z_k + (1 - alpha) (alpha y_{k+1} + y_{k+2}),
  * from the two y values the step's kernel holds anyway; the first step of a round and, when L is even, the last
  * one use the one-step form.  The same recurrence, so z and x^a agree with the step-by-step form to fp32 rounding
- * (not bit for bit); y^a is unchanged.  It saves the read and the write of z on half of the steps (14 instead of
- * 22 bytes per weight).  parle_inner_step always applies the one-step form: z is current after every call.
+ * (not bit for bit); y^a is unchanged.  It saves the read and the write of z on half of the steps (8 of the 22 bytes
+ * per weight of the fused bf16 kernel, 8 of the 24 of the separate update kernel).  parle_inner_step and
+ * parle_inner_update always apply the one-step form: z is current after every call.
  * off: every step of a round updates z.  ESTATE inside a round. */
 int parle_set_paired_z_update(parle_ctx *ctx, int on);
 

@@ -88,7 +88,7 @@ struct parle_ctx {
     cudaStream_t stream;
     int *status_host, *status_dev;
     bool round_open, fresh, shadow_is_x;
-    bool paired_z;                   // fused bf16 path, whole rounds: Eq. (parle_z) applied two steps at a time
+    bool paired_z;                   // whole rounds: Eq. (parle_z) applied two steps at a time
     int z_mode;                      // how the next fused step treats z (WU_Z_*); set per step by the round drivers
     bool fused_update;               // bf16 path: apply Eq. (parle_y)/(parle_z) inside the weight-gradient GEMM
     int steps_in_round;
@@ -492,34 +492,36 @@ int run_blocked_copy(parle_ctx *c, const float *src) {
 
 int run_split_transpose(parle_ctx *c, const float *src);
 
-template <bool FIRST, bool MOM, bool SPLIT>
+template <bool FIRST, bool MOM, bool SPLIT, int ZMODE>
 void launch_inner_update(parle_ctx *c, int grid, const float4 *g, float4 *y, const float4 *x, float4 *z, size_t n4, float wd) {
     constexpr int U = 2;
-    inner_update_kernel<FIRST, U, MOM, SPLIT><<<grid, kUpdThreads, 0, c->stream>>>(
+    inner_update_kernel<FIRST, U, MOM, SPLIT, ZMODE><<<grid, kUpdThreads, 0, c->stream>>>(
         g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev,
         MOM ? reinterpret_cast<float4 *>(c->vy) : nullptr, c->momentum,
         SPLIT ? ws_ptr<float4>(c, c->ws.w_split[0]) : nullptr, SPLIT ? ws_ptr<float4>(c, c->ws.w_split[1]) : nullptr);
 }
+template <bool MOM, bool SPLIT>
+void launch_inner_update_z(parle_ctx *c, int zm, int grid, const float4 *g, float4 *y, const float4 *x, float4 *z, size_t n4, float wd) {
+    if (c->fresh) launch_inner_update<true, MOM, SPLIT, UPD_Z_SINGLE>(c, grid, g, y, x, z, n4, wd);
+    else if (zm == UPD_Z_SKIP) launch_inner_update<false, MOM, SPLIT, UPD_Z_SKIP>(c, grid, g, y, x, z, n4, wd);
+    else if (zm == UPD_Z_DOUBLE) launch_inner_update<false, MOM, SPLIT, UPD_Z_DOUBLE>(c, grid, g, y, x, z, n4, wd);
+    else launch_inner_update<false, MOM, SPLIT, UPD_Z_SINGLE>(c, grid, g, y, x, z, n4, wd);
+}
 
 // split: also refresh the tf32 hi/lo copy of the parameters from the new y (fp32 products on the tensor cores)
-int run_inner_update(parle_ctx *c, const float *grad, float wd, bool split = false) {
+// zm: how this step treats z (UPD_Z_*; the round drivers pair the steps, single calls use the one-step form)
+int run_inner_update(parle_ctx *c, const float *grad, float wd, bool split = false, int zm = UPD_Z_SINGLE) {
     const size_t n4 = (size_t)c->n * c->stride / 4;
     const int grid = stream_grid(c, n4, 2);
     const float4 *g = reinterpret_cast<const float4 *>(grad);
     float4 *y = reinterpret_cast<float4 *>(c->buf.y), *z = reinterpret_cast<float4 *>(c->buf.z);
     const float4 *x = reinterpret_cast<const float4 *>(c->buf.x);
     prof_begin(c, KC_INNER_UPDATE);
-    const int variant = (c->fresh ? 4 : 0) | (c->momentum > 0.f ? 2 : 0) | (split ? 1 : 0);
-    switch (variant) {
-        case 0: launch_inner_update<false, false, false>(c, grid, g, y, x, z, n4, wd); break;
-        case 1: launch_inner_update<false, false, true>(c, grid, g, y, x, z, n4, wd); break;
-        case 2: launch_inner_update<false, true, false>(c, grid, g, y, x, z, n4, wd); break;
-        case 3: launch_inner_update<false, true, true>(c, grid, g, y, x, z, n4, wd); break;
-        case 4: launch_inner_update<true, false, false>(c, grid, g, y, x, z, n4, wd); break;
-        case 5: launch_inner_update<true, false, true>(c, grid, g, y, x, z, n4, wd); break;
-        case 6: launch_inner_update<true, true, false>(c, grid, g, y, x, z, n4, wd); break;
-        default: launch_inner_update<true, true, true>(c, grid, g, y, x, z, n4, wd); break;
-    }
+    const bool mom = c->momentum > 0.f;
+    if (mom && split) launch_inner_update_z<true, true>(c, zm, grid, g, y, x, z, n4, wd);
+    else if (mom) launch_inner_update_z<true, false>(c, zm, grid, g, y, x, z, n4, wd);
+    else if (split) launch_inner_update_z<false, true>(c, zm, grid, g, y, x, z, n4, wd);
+    else launch_inner_update_z<false, false>(c, zm, grid, g, y, x, z, n4, wd);
     PARLE_LAUNCHED(c);
     c->fresh = false;
     c->shadow_is_x = false;
@@ -1031,11 +1033,11 @@ int parle_inner_step(parle_ctx *c, const float *inputs, const int32_t *labels, f
         }
     } else if (use_t3(c)) {
         PARLE_TRY(forward_backward_tf32(c, inputs, labels, loss_out));
-        return run_inner_update(c, c->buf.grad, c->weight_decay, true);
+        return run_inner_update(c, c->buf.grad, c->weight_decay, true, c->z_mode);
     } else {
         PARLE_TRY(forward_backward_fp32(c, inputs, labels, loss_out));
     }
-    return run_inner_update(c, c->buf.grad, c->weight_decay);
+    return run_inner_update(c, c->buf.grad, c->weight_decay, false, c->z_mode);
 }
 
 int parle_inner_step_host(parle_ctx *c, const float *inputs_host, const int32_t *labels_host, float *loss_out_host) {
@@ -1210,11 +1212,12 @@ int parle_set_round_graphs(parle_ctx *c, int on) {
     return PARLE_OK;
 }
 
-// How step l (0-based) of an L-step round treats z when Eq. (parle_z) is applied two steps at a time (fused bf16
-// path): the first step forms z from x; the remaining L - 1 steps go in (skip, two-step) pairs, with a one-step
-// update at the end when L - 1 is odd.
+// How step l (0-based) of an L-step round treats z when Eq. (parle_z) is applied two steps at a time: the first
+// step forms z from x; the remaining L - 1 steps go in (skip, two-step) pairs, with a one-step update at the end
+// when L - 1 is odd.  (WU_Z_* and UPD_Z_* have the same values.)
+static_assert(WU_Z_SINGLE == UPD_Z_SINGLE && WU_Z_SKIP == UPD_Z_SKIP && WU_Z_DOUBLE == UPD_Z_DOUBLE, "z modes");
 static int paired_z_mode(const parle_ctx *c, int l, int L) {
-    if (!c->paired_z || !c->fused_update || c->gemm_dtype != PARLE_GEMM_BF16 || l == 0) return WU_Z_SINGLE;
+    if (!c->paired_z || l == 0) return WU_Z_SINGLE;
     const int rest = L - 1, idx = l - 1;
     if ((rest & 1) && idx == rest - 1) return WU_Z_SINGLE;
     return (idx & 1) ? WU_Z_DOUBLE : WU_Z_SKIP;

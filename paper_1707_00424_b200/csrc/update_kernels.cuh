@@ -24,7 +24,11 @@ __device__ __forceinline__ bool finite4(const float4 &v) {
 //      v <- mu v + d, y <- y - eta' (d + mu v); v starts from 0 in every round (FIRST: v is only written).
 // SPLIT: also store the new y as a tf32-exact pair (hi = y rounded to tf32, lo = y - hi rounded to tf32):
 //      the operands of the fp32-accurate tensor-core products of the next step.
-template <bool FIRST, int UNROLL, bool MOM = false, bool SPLIT = false>
+// ZMODE (ignored when FIRST): Eq. (parle_z) may be applied two steps at a time inside a round, since
+//      z_{k+2} = alpha^2 z_k + (1-alpha)(alpha y_{k+1} + y_{k+2}) needs only the y this step reads and the y it writes:
+//      0 = one-step form, 1 = z untouched (neither read nor written), 2 = two-step form.
+constexpr int UPD_Z_SINGLE = 0, UPD_Z_SKIP = 1, UPD_Z_DOUBLE = 2;
+template <bool FIRST, int UNROLL, bool MOM = false, bool SPLIT = false, int ZMODE = UPD_Z_SINGLE>
 __global__ void __launch_bounds__(kUpdThreads)
 inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const float4 *__restrict__ x,
                     float4 *__restrict__ z, size_t n4,
@@ -33,7 +37,9 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
                     float4 *__restrict__ y_hi = nullptr, float4 *__restrict__ y_lo = nullptr) {
     const size_t tid = (size_t)blockIdx.x * kUpdThreads + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * kUpdThreads;
-    const float one_m_alpha = 1.0f - alpha;
+    const float one_m_alpha = 1.0f - alpha, alpha_sq = alpha * alpha;
+    constexpr bool USE_Z = FIRST || ZMODE != UPD_Z_SKIP;
+    constexpr bool DOUBLE_Z = !FIRST && ZMODE == UPD_Z_DOUBLE;
     bool ok = true;
     for (size_t base = tid; base < n4; base += nthreads * UNROLL) {
         float4 gv[UNROLL], yv[UNROLL], xv[UNROLL], zv[UNROLL], vv[UNROLL];
@@ -45,7 +51,7 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
                 xv[u] = __ldg(x + i);
                 if (!FIRST) {
                     yv[u] = y[i];
-                    zv[u] = z[i];
+                    if (USE_Z) zv[u] = z[i];
                     if (MOM) vv[u] = v[i];
                 }
             }
@@ -55,7 +61,7 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
             const size_t i = base + (size_t)u * nthreads;
             if (i < n4) {
                 float4 yo = FIRST ? xv[u] : yv[u];
-                float4 zo = FIRST ? xv[u] : zv[u];
+                float4 zo = FIRST ? xv[u] : (USE_Z ? zv[u] : make_float4(0.f, 0.f, 0.f, 0.f));
                 float4 yn, zn, d;
                 d.x = fmaf(inv_gamma, yo.x - xv[u].x, fmaf(wd, yo.x, gv[u].x));
                 d.y = fmaf(inv_gamma, yo.y - xv[u].y, fmaf(wd, yo.y, gv[u].y));
@@ -75,13 +81,20 @@ inner_update_kernel(const float4 *__restrict__ g, float4 *__restrict__ y, const 
                 yn.y = yo.y - eta_p * d.y;
                 yn.z = yo.z - eta_p * d.z;
                 yn.w = yo.w - eta_p * d.w;
-                zn.x = fmaf(alpha, zo.x, one_m_alpha * yn.x);
-                zn.y = fmaf(alpha, zo.y, one_m_alpha * yn.y);
-                zn.z = fmaf(alpha, zo.z, one_m_alpha * yn.z);
-                zn.w = fmaf(alpha, zo.w, one_m_alpha * yn.w);
+                if (DOUBLE_Z) {
+                    zn.x = fmaf(alpha_sq, zo.x, one_m_alpha * fmaf(alpha, yo.x, yn.x));
+                    zn.y = fmaf(alpha_sq, zo.y, one_m_alpha * fmaf(alpha, yo.y, yn.y));
+                    zn.z = fmaf(alpha_sq, zo.z, one_m_alpha * fmaf(alpha, yo.z, yn.z));
+                    zn.w = fmaf(alpha_sq, zo.w, one_m_alpha * fmaf(alpha, yo.w, yn.w));
+                } else {
+                    zn.x = fmaf(alpha, zo.x, one_m_alpha * yn.x);
+                    zn.y = fmaf(alpha, zo.y, one_m_alpha * yn.y);
+                    zn.z = fmaf(alpha, zo.z, one_m_alpha * yn.z);
+                    zn.w = fmaf(alpha, zo.w, one_m_alpha * yn.w);
+                }
                 ok &= finite4(yn);
                 y[i] = yn;
-                z[i] = zn;
+                if (USE_Z) z[i] = zn;
                 if (SPLIT) {
                     float4 h, l;
                     split_tf32(yn.x, h.x, l.x); split_tf32(yn.y, h.y, l.y);
