@@ -271,6 +271,14 @@ def run_ours(args):
     e2e_value = world * cfg.n * cfg.L * K / (ms_e2e * 1e-3)
     h2d = cfg.L * (cfg.n * cfg.batch * cfg.dims[0] * 4 + cfg.n * cfg.batch * 4)
     d2h = cfg.L * cfg.n * 4
+    # 4. for comparison: the same rounds with z read and written at every inner step (Eq. parle_z one step at a time)
+    every_step = None
+    if args.paired_z:
+        model.set_paired_z_update(False)
+        ms_u, _, _ = timed(round_device, min(W, 2), K)
+        model.set_paired_z_update(True)
+        every_step = {"value": world * cfg.n * cfg.L * K / (ms_u * 1e-3), "unit": UNIT, "ms_per_step": ms_u / K,
+                      "what": "same rounds with parle_set_paired_z_update(0): z updated at every inner step"}
 
     if rank != 0:
         if world > 1:
@@ -335,6 +343,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e / K},
         "roofline": roofline, "roofline_other_kernels": {k: v for k, v in rooflines.items() if k != dom},
         "kernel_shares": shares, "profile_dropped": dropped,
+        "z_every_step": every_step,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
