@@ -97,3 +97,19 @@ def test_scoping_schedule_host_function():
     m.set_weight_decay(1e-3)
     with pytest.raises(pb.ParleError):
         m.set_weight_decay(-1.0)
+
+
+def test_path_switches_check_their_arguments_without_a_gpu():
+    m = pb.Parle(2, (256, 256, 8), 64)                   # fp32: the tensor-core path exists for it, but nothing is bound yet
+    assert not m.fp32_tensor_cores_active
+    for mode in (0, 1, 2):
+        m.set_fp32_tensor_cores(mode)
+    with pytest.raises(pb.ParleError) as e:
+        m.set_fp32_tensor_cores(3)
+    assert e.value.code == -1
+    with pytest.raises(pb.ParleError):
+        pb.Parle(2, (64, 64, 8), 64, pb.GEMM_BF16).set_fp32_tensor_cores(1)     # a bf16 context has no such switch
+    m.set_paired_z_update(False); m.set_paired_z_update(True)
+    # the workspace of an fp32 context whose shapes allow the tensor-core path holds the hi/lo operand pairs too
+    odd = pb.Parle(2, (254, 256, 8), 64)                 # 254 is not a multiple of 4: FMA pipes only
+    assert m.workspace_bytes > odd.workspace_bytes + 2 * 2 * m.stride * 4
