@@ -138,7 +138,7 @@ def ncu_traffic(workload: str, kernel: str):
     return rec["bytes"]         # (taken with the default settings: z updated every other step)
 
 
-def algorithmic_bytes_per_round(cfg, stride, tf32_split=False, paired_z=True):
+def algorithmic_bytes_per_round(cfg, stride, tf32_split=False, paired_z=True, split_y=True):
     """Bytes each kernel class has to move per Parle round (all n replicas), from the data it must
     touch once: parameter-state vectors at 4 B (fp32) or 2 B (bf16 copy) per element, plus GEMM operands.
     tf32_split: the fp32 update also writes the tf32 hi/lo copy of y (8 B per element).
@@ -159,7 +159,10 @@ def algorithmic_bytes_per_round(cfg, stride, tf32_split=False, paired_z=True):
         # fused: read y, x, z (12 B), write y, z, bf16 copy (10 B); first step reads only x (14 B); with Eq. (parle_z)
         # applied two steps at a time the other steps alternate between 14 B (z untouched) and 22 B
         pairs, single = ((L - 1) // 2, (L - 1) % 2) if paired_z else (0, L - 1)
-        out["wgrad_gemm_fused_update"] = n * (Pw * (14 + pairs * (14 + 22) + single * 22) + opnd * L)
+        # y as two 16-bit planes inside a round: every step moves 2 B less (no separate operand copy), the last one
+        # stores the fp32 y once more
+        ys = 2 if split_y else 0
+        out["wgrad_gemm_fused_update"] = n * (Pw * (14 - ys + pairs * (14 + 22 - 2 * ys) + single * (22 - ys) + (4 if split_y else 0)) + opnd * L)
         out["wgrad_gemm"] = n * L * (4 * Pw + opnd)
         out["fwd_gemm"] = n * L * (2 * Pw + sum(2 * act(l) + 4 * act(l + 1) for l in range(nl)))
         out["to_bf16"] = n * Pw * 6                                          # blocked bf16 weight copy from x, once per round
@@ -208,6 +211,8 @@ def run_ours(args):
     model.mean()
     model.set_round_graphs(bool(args.graphs))
     model.set_paired_z_update(bool(args.paired_z))
+    if cfg.gemm_dtype == 1:
+        model.set_split_y(bool(args.split_y))
     sets = 2
     Xh, ch = make_round_inputs(cfg, sets)
     Xd, cd = torch.from_numpy(Xh).to(dev), torch.from_numpy(ch).to(dev)
@@ -275,10 +280,14 @@ def run_ours(args):
     every_step = None
     if args.paired_z:
         model.set_paired_z_update(False)
+        if cfg.gemm_dtype == 1:
+            model.set_split_y(False)
         ms_u, _, _ = timed(round_device, min(W, 2), K)
         model.set_paired_z_update(True)
+        if cfg.gemm_dtype == 1:
+            model.set_split_y(bool(args.split_y))
         every_step = {"value": world * cfg.n * cfg.L * K / (ms_u * 1e-3), "unit": UNIT, "ms_per_step": ms_u / K,
-                      "what": "same rounds with parle_set_paired_z_update(0): z updated at every inner step"}
+                      "what": "same rounds with parle_set_paired_z_update(0) and parle_set_split_y(0): z and fp32 y read and written at every inner step"}
 
     if rank != 0:
         if world > 1:
@@ -289,14 +298,14 @@ def run_ours(args):
     shares = {k: {"ms_per_round": v[0] / K, "launches_per_round": v[1] / K, "share": v[0] / total_ms} for k, v in prof.items()}
     dom = max(prof, key=lambda k: prof[k][0])
     t3 = cfg.gemm_dtype == 0 and model.fp32_tensor_cores_active
-    alg = algorithmic_bytes_per_round(cfg, model.stride, tf32_split=t3, paired_z=bool(args.paired_z))
+    alg = algorithmic_bytes_per_round(cfg, model.stride, tf32_split=t3, paired_z=bool(args.paired_z), split_y=bool(args.split_y))
     rooflines = {}
     for k, (ms_k, cnt_k) in prof.items():
         if k not in alg:
             continue
         ach = alg[k] * K / (ms_k * 1e-3) / 1e9          # bytes of K rounds / device time of the class over K rounds
         rooflines[k] = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, k) if args.paired_z else None,
+                        "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(cfg.name, k) if (args.paired_z and args.split_y) else None,
                         "peak_source": peaks["source"], "bytes_per_launch": alg[k] * K / cnt_k,
                         "ms_per_launch": ms_k / cnt_k, "launches_per_round": cnt_k / K}
     flops = gemm_flops_per_round(cfg)
@@ -424,6 +433,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(si.CONFIGS))
     ap.add_argument("--graphs", type=int, default=1, help="replay rounds from CUDA graphs (parle_set_round_graphs)")
+    ap.add_argument("--split-y", type=int, default=1, help="bf16 workloads: y as bf16 copy + lower-half plane inside a round (parle_set_split_y)")
     ap.add_argument("--paired-z", type=int, default=1, help="Eq. (parle_z) two steps at a time inside a round (parle_set_paired_z_update)")
     args = ap.parse_args()
     if args.impl == "reference":

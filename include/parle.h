@@ -189,6 +189,16 @@ int parle_set_fused_update(parle_ctx *ctx, int on);
  * off: every step of a round updates z.  ESTATE inside a round. */
 int parle_set_paired_z_update(parle_ctx *ctx, int on);
 
+/* bf16 path with the fused update, whole rounds only (parle_round, parle_round_host).  on (the default): between the
+ * first and the last inner step of a round the y^a of the weights is not kept as fp32 words but as the bf16 operand copy
+ * the GEMMs read (the rounded upper halves) plus a plane of the lower halves in the workspace -- together the same 32
+ * bits, moved as 2 + 2 bytes with no separate operand copy to write (12 / 20 instead of 14 / 22 bytes per weight and
+ * step).  The last step of the round stores the fp32 y^a again, so y is current when the call returns.  One detail: an
+ * fp32 value whose lower half is exactly 0x8000 under an odd upper half is stored one fp32 ulp higher (that makes the
+ * rounding direction of the bf16 copy recoverable from the lower half alone); this touches 2^-17 of the elements.
+ * Biases are not affected.  off: y^a is read and written as fp32 at every step.  ESTATE inside a round. */
+int parle_set_split_y(parle_ctx *ctx, int on);
+
 /* fp32 configurations only: where the forward / backward products run (Section 1.1 / 2.1, the minibatch
  * gradient).  On an sm_100 device, when the batch and every layer's input width are multiples of 4, they can
  * run on the tensor cores at fp32 accuracy: every fp32 operand is kept as a pair of tf32-exact arrays

@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
         "parle_set_fused_update": (ci, [vp, ci]),
         "parle_set_fp32_tensor_cores": (ci, [vp, ci]),
         "parle_set_paired_z_update": (ci, [vp, ci]),
+        "parle_set_split_y": (ci, [vp, ci]),
         "parle_fp32_tensor_cores_active": (ci, [vp]),
         "parle_set_weight_decay": (ci, [vp, cd]),
         "parle_set_wide_tile_threshold": (ci, [vp, ci]),
@@ -266,6 +267,10 @@ class Parle:
     def set_paired_z_update(self, on: bool):
         """Whole rounds on the fused bf16 path: update z every other inner step with the two-step form of Eq. (parle_z)."""
         self._check(self._L.parle_set_paired_z_update(self._h, 1 if on else 0), "parle_set_paired_z_update")
+
+    def set_split_y(self, on: bool):
+        """Whole rounds on the fused bf16 path: keep y of the weights as bf16 operand copy + lower-half plane between steps."""
+        self._check(self._L.parle_set_split_y(self._h, 1 if on else 0), "parle_set_split_y")
 
     def set_fp32_tensor_cores(self, mode: int):
         """0: FMA pipes, 1: tensor cores (3 x tf32) for wide layers, 2: tensor cores whenever the shapes allow."""

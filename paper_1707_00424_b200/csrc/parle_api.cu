@@ -44,6 +44,7 @@ struct Workspace {
     size_t xs[2], xT[2];               // inputs [n, B, d_0] and transposed [n, d_0, B]
     size_t hs[PARLE_MAX_LAYERS][2], hT[PARLE_MAX_LAYERS][2];     // hidden activations [n, B, d_{l+1}] and transposed
     size_t dhs[PARLE_MAX_LAYERS][2], dhT[PARLE_MAX_LAYERS][2];   // their gradients [n, B, ld_l] (ld_l = d_{l+1} rounded up to 4) and transposed [n, d_{l+1}, B]
+    size_t ylo;                        // bf16 mode: low 16 bits of the fp32 words of y, [n, stride] uint16 (whole rounds keep y as bf16 copy + this)
     size_t sched;                      // bf16 mode: two ints, the tile counters of the fused weight-gradient kernel (zero between launches)
     size_t stage_in[2], stage_lab[2], stage_loss[2];   // double-buffered staging for the host-buffer entry points
     size_t total;
@@ -59,6 +60,7 @@ struct RoundKey {
     float scal[7];                   // 1/gamma, 1/rho, alpha, eta, eta', weight decay, momentum
     int fused, wide_thr, shadow_is_x, fresh;   // L == 0: a single inner step (fresh = first of its round)
     int paired_z, z_mode;            // whole rounds: Eq. (parle_z) in pairs or not; single steps: how this step treats z
+    int split_y, y_step;             // whole rounds: y in two 16-bit planes or not; single steps: bit 0 = in that mode, bit 1 = stores fp32 y
     const void *ptrs[9];             // x, y, z, grad, xbar, workspace, vy, vx, stream
 };
 struct RoundGraph {
@@ -89,6 +91,8 @@ struct parle_ctx {
     int *status_host, *status_dev;
     bool round_open, fresh, shadow_is_x;
     bool paired_z;                   // whole rounds: Eq. (parle_z) applied two steps at a time
+    bool split_y;                    // fused bf16 path, whole rounds: y of the weights kept as bf16 copy + low-half plane
+    bool y_split_step, y_write_step; // this step runs in that mode / also stores the fp32 y (set per step by the round drivers)
     int z_mode;                      // how the next fused step treats z (WU_Z_*); set per step by the round drivers
     bool fused_update;               // bf16 path: apply Eq. (parle_y)/(parle_z) inside the weight-gradient GEMM
     int steps_in_round;
@@ -200,6 +204,7 @@ void plan_workspace(parle_ctx *c) {
             w.dhb[l] = take(n * B * w.dh_ld[l] * 2);
             w.dhbT[l] = take(n * B * c->dims[l + 1] * 2);
         }
+        w.ylo = take(n * c->stride * sizeof(uint16_t));
         w.sched = take(2 * sizeof(int));
     }
     w.row_loss = take(n * B * sizeof(float));
@@ -306,6 +311,37 @@ inline int t3_tile_width(const parle_ctx *c, int M, int N) {
     return wide * 4 < (long long)c->sm_count * 3 ? 64 : 128;
 }
 
+// The two 16-bit planes of y for the fused kernel: boxes of 64 columns x box_rows of the blocked bf16 copy (5-D, no
+// swizzle: they are read back element by element), and boxes of 128 columns x box_rows of the uint16 lo plane.
+int encode_yhi_map(parle_ctx *c, CUtensorMap *tm, const void *base, int cb, int rb, size_t groups, size_t group_pitch,
+                   unsigned box_rows) {
+    EncodeTiledFn enc;
+    PARLE_TRY(get_encoder(c, &enc));
+    cuuint64_t dims[5] = {64, 128, (cuuint64_t)cb, (cuuint64_t)rb, groups};
+    cuuint64_t strides[4] = {128, 16384, (cuuint64_t)cb * 16384, group_pitch * 2};
+    cuuint32_t box[5] = {64, box_rows, 1, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
+    return PARLE_OK;
+}
+int encode_ylo_map(parle_ctx *c, CUtensorMap *tm, const void *base, size_t cols, size_t rows, size_t groups,
+                   size_t row_pitch, size_t group_pitch, unsigned box_rows) {
+    EncodeTiledFn enc;
+    PARLE_TRY(get_encoder(c, &enc));
+    cuuint64_t dims[3] = {cols, rows, groups};
+    cuuint64_t strides[2] = {row_pitch * 2, group_pitch * 2};
+    cuuint32_t box[3] = {(cuuint32_t)UM_BM, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { c->last_cuda = (int)r; return PARLE_ECUDA; }
+    return PARLE_OK;
+}
+
 int build_tf32_maps(parle_ctx *c) {
     const Workspace &w = c->ws;
     const size_t n = c->n, B = c->batch, S = c->stride;
@@ -395,6 +431,8 @@ int build_tensor_maps(parle_ctx *c) {
         PARLE_TRY(encode_f32_map(c, &c->wu_maps.z[l], c->buf.z + wo, din, dout, n, din, c->stride, UM_BM, WU_CHUNK_ROWS));
         c->wu_maps.v[l] = c->wu_maps.z[l];                                   // not read without momentum
         c->wu_maps.a[l] = c->tm_wg_a[l]; c->wu_maps.b[l] = c->tm_wg_b[l];
+        PARLE_TRY(encode_yhi_map(c, &c->wu_maps.yhi[l], W, c->sh_cb[l], c->sh_rb[l], n, c->sh_stride, WU_CHUNK_ROWS));
+        PARLE_TRY(encode_ylo_map(c, &c->wu_maps.ylo[l], ws_ptr<uint16_t>(c, w.ylo) + wo, din, dout, n, din, c->stride, WU_CHUNK_ROWS));
         if (l > 0) {
             // data gradient: A = dH [B, dout] K-major (K = dout); B = W [dout (K), din (N)] MN-major,
             // fetched as 64 k-rows x 64 n-columns boxes
@@ -776,8 +814,11 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     const int zm = c->fresh ? WU_Z_SINGLE : c->z_mode;
     if (mom) { p.v = c->vy; p.mu = c->momentum; }
     const WuMaps &maps = mom ? c->wu_maps_mom : c->wu_maps;
-#define PARLE_WU_LAUNCH(FIRST, SH, MOM, ZM) \
-    umma_wgrad_update_kernel<FIRST, SH, MOM, ZM><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p)
+#define PARLE_WU_LAUNCH(FIRST, SH, MOM, ZM) do { \
+        if (ys) umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); \
+        else umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); } while (0)
+    const bool ys = c->y_split_step;
+    p.ylo = ws_ptr<uint16_t>(c, w.ylo); p.write_y = c->y_write_step ? 1 : 0;
     if (mom) {
         if (c->fresh) PARLE_WU_LAUNCH(true, WuMomentum, true, WU_Z_SINGLE);
         else if (zm == WU_Z_SKIP) PARLE_WU_LAUNCH(false, WuMomentum, true, WU_Z_SKIP);
@@ -901,6 +942,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
     }
     c->fused_update = (c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0);
     c->paired_z = true;
+    c->split_y = true;
     c->wide_tiles_per_sm = 4;
     c->last_ksplit = 1;
     if (c->fused_update) {
@@ -975,7 +1017,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, UB_BLOCKED_K>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, UB_ROWMAJOR_K>()));
 #define PARLE_WU_SMEM(FIRST, SH, MOM, ZM) \
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES))
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES)); \
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES))
         PARLE_WU_SMEM(true, WuDefault, false, WU_Z_SINGLE); PARLE_WU_SMEM(false, WuDefault, false, WU_Z_SINGLE);
         PARLE_WU_SMEM(false, WuDefault, false, WU_Z_SKIP); PARLE_WU_SMEM(false, WuDefault, false, WU_Z_DOUBLE);
         PARLE_WU_SMEM(true, WuMomentum, true, WU_Z_SINGLE); PARLE_WU_SMEM(false, WuMomentum, true, WU_Z_SINGLE);
@@ -1107,6 +1150,7 @@ static RoundKey make_round_key(const parle_ctx *c, int L, const void *in, const 
     memcpy(k.scal, sc, sizeof(sc));
     k.fused = c->fused_update; k.wide_thr = c->wide_tiles_per_sm; k.shadow_is_x = c->shadow_is_x; k.fresh = c->fresh;
     k.paired_z = c->paired_z; k.z_mode = c->z_mode;
+    k.split_y = c->split_y; k.y_step = (c->y_split_step ? 1 : 0) | (c->y_write_step ? 2 : 0);
     const void *pt[9] = {c->buf.x, c->buf.y, c->buf.z, c->buf.grad, c->buf.xbar, c->buf.workspace, c->vy, c->vx, c->stream};
     memcpy(k.ptrs, pt, sizeof(pt));
     return k;
@@ -1223,14 +1267,21 @@ static int paired_z_mode(const parle_ctx *c, int l, int L) {
     return (idx & 1) ? WU_Z_DOUBLE : WU_Z_SKIP;
 }
 
+// Whole rounds on the fused bf16 path keep the y of the weights as bf16 copy + low-half plane (the last step also
+// stores the fp32 y).
+static bool split_y_round(const parle_ctx *c) {
+    return c->split_y && c->fused_update && c->gemm_dtype == PARLE_GEMM_BF16;
+}
+
 static int round_direct(parle_ctx *c, int L, const float *inputs, const int32_t *labels, float *loss_out) {
     PARLE_TRY(parle_round_begin(c));
     const size_t nb = (size_t)c->n * c->batch;
     for (int l = 0; l < L; ++l) {
         c->z_mode = paired_z_mode(c, l, L);
+        c->y_split_step = split_y_round(c); c->y_write_step = (l == L - 1);
         const int rc = parle_inner_step(c, inputs + (size_t)l * nb * c->dims[0], labels + (size_t)l * nb,
                                         loss_out ? loss_out + (size_t)l * c->n : nullptr);
-        c->z_mode = WU_Z_SINGLE;
+        c->z_mode = WU_Z_SINGLE; c->y_split_step = false; c->y_write_step = false;
         PARLE_TRY(rc);
     }
     return parle_outer_step(c);
@@ -1269,6 +1320,7 @@ int parle_round_host(parle_ctx *c, int L, const float *inputs_host, const int32_
         PARLE_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[b], 0));
         float *dloss = ws_ptr<float>(c, c->ws.stage_loss[b]);
         c->z_mode = paired_z_mode(c, l, L);
+        c->y_split_step = split_y_round(c); c->y_write_step = (l == L - 1);
         int rc;
         if (c->graphs_on && !c->prof_on)       // the step's kernels as one cached graph (staging buffers have fixed addresses)
             rc = round_graphed(c, 0, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
@@ -1276,7 +1328,7 @@ int parle_round_host(parle_ctx *c, int L, const float *inputs_host, const int32_
         else
             rc = parle_inner_step(c, ws_ptr<float>(c, c->ws.stage_in[b]), ws_ptr<int32_t>(c, c->ws.stage_lab[b]),
                                   loss_out_host ? dloss : nullptr);
-        c->z_mode = WU_Z_SINGLE;
+        c->z_mode = WU_Z_SINGLE; c->y_split_step = false; c->y_write_step = false;
         PARLE_TRY(rc);
         if (loss_out_host)
             PARLE_CUDA(c, cudaMemcpyAsync(loss_out_host + (size_t)l * c->n, dloss, c->n * sizeof(float),
@@ -1297,6 +1349,13 @@ int parle_set_fused_update(parle_ctx *c, int on) {
     if (on && !(c->gemm_dtype == PARLE_GEMM_BF16 && c->n_layers > 0)) return PARLE_EUNSUPPORTED;
     if (c->round_open && c->steps_in_round > 0) return PARLE_ESTATE;
     c->fused_update = on != 0;
+    return PARLE_OK;
+}
+
+int parle_set_split_y(parle_ctx *c, int on) {
+    if (!c) return PARLE_EINVAL;
+    if (c->round_open) return PARLE_ESTATE;
+    c->split_y = on != 0;
     return PARLE_OK;
 }
 
@@ -1340,6 +1399,10 @@ int parle_bind_momentum(parle_ctx *c, float *vy, float *vx) {
             for (int k = 0; k < 4; ++k)
                 PARLE_TRY(encode_f32_map(c, tm[k], base[k], din, dout, c->n, din, c->stride, UM_BM, WU_CHUNK_ROWS_MOM));
             c->wu_maps_mom.a[l] = c->tm_wg_a[l]; c->wu_maps_mom.b[l] = c->tm_wg_b[l];
+            PARLE_TRY(encode_yhi_map(c, &c->wu_maps_mom.yhi[l], ws_ptr<__nv_bfloat16>(c, c->ws.shadow) + c->sh_off[l], c->sh_cb[l],
+                                     c->sh_rb[l], c->n, c->sh_stride, WU_CHUNK_ROWS_MOM));
+            PARLE_TRY(encode_ylo_map(c, &c->wu_maps_mom.ylo[l], ws_ptr<uint16_t>(c, c->ws.ylo) + wo, din, dout, c->n, din, c->stride,
+                                     WU_CHUNK_ROWS_MOM));
         }
         c->mom_maps = true;
     }

@@ -40,6 +40,14 @@
 // writes).  So inside a whole round z is read and written every other step only: ZMODE 1 leaves z alone (14 bytes
 // per weight instead of 22), ZMODE 2 applies the two-step form, ZMODE 0 the one-step form (single steps, and the last
 // step of a round with an even number of steps).  Same recurrence, different fp32 rounding of z (1e-7 relative).
+//
+// y in two 16-bit planes (YSPLIT).  Inside a whole round nobody but this kernel reads the fp32 y of the weights, and the
+// kernel writes bf16(y) for the GEMMs anyway.  So y is kept as that bf16 copy (the "hi" plane) plus the low 16 bits of
+// its fp32 word (the "lo" plane, workspace): together exactly the fp32 value, read and written as 2 + 2 bytes, and the
+// separate 2-byte operand copy comes for free: 12 / 20 bytes per weight and step instead of 14 / 22.  Decoding:
+// bf16 round-to-nearest-even went up exactly when lo > 0x8000, or lo == 0x8000 with an odd upper half; in that last
+// (tie) case the encoder stores 0x8001, i.e. moves y by one fp32 ulp (2^-17 of the elements), so that "went up" is
+// simply lo > 0x8000.  The last step of a round also writes the fp32 y, so y is current again when the round returns.
 // All waits are bounded.
 #pragma once
 
@@ -102,6 +110,8 @@ struct WgradUpdateParams {
     long long shadow_gs;         // replica pitch of the copy (elements)
     long long gs;
     float eta_p, inv_gamma, alpha, wd;
+    uint16_t *ylo;               // YSPLIT: low halves of the fp32 words of y (same addressing as y); the high halves are `shadow`
+    int write_y;                 // YSPLIT: also store the fp32 y (last step of a round)
     float *v; float mu;          // Nesterov momentum buffer of y (same addressing as y), used by the MOM variant
     int *sched;                  // sched[0]: tiles claimed beyond the first of every CTA, sched[1]: CTAs that have left; both 0 between launches
     int *status;
@@ -111,13 +121,17 @@ struct WgradUpdateParams {
 struct WuMaps {
     CUtensorMap a[PARLE_MAX_LAYERS], b[PARLE_MAX_LAYERS];
     CUtensorMap x[PARLE_MAX_LAYERS], y[PARLE_MAX_LAYERS], z[PARLE_MAX_LAYERS], v[PARLE_MAX_LAYERS];
+    // YSPLIT: y as its two 16-bit planes -- boxes of 64 columns x chunk rows of the blocked bf16 copy (no swizzle),
+    // and boxes of 128 columns x chunk rows of the lo plane
+    CUtensorMap yhi[PARLE_MAX_LAYERS], ylo[PARLE_MAX_LAYERS];
 };
 
 // MOM: Nesterov momentum on the y step (see inner_update_kernel): v <- mu v + d, y <- y - eta' (d + mu v),
 // v = 0 at the start of a round (FIRST: v is only written).
 // ZMODE (ignored when FIRST): 0 = z <- alpha z + (1-alpha) y_new; 1 = z untouched; 2 = z <- alpha^2 z + (1-alpha)(alpha y_old + y_new).
 constexpr int WU_Z_SINGLE = 0, WU_Z_SKIP = 1, WU_Z_DOUBLE = 2;
-template <bool FIRST, class SH, bool MOM = false, int ZMODE = WU_Z_SINGLE>
+// YSPLIT: y is read and written as two 16-bit planes (see the head of this file).
+template <bool FIRST, class SH, bool MOM = false, int ZMODE = WU_Z_SINGLE, bool YSPLIT = false>
 __global__ void __launch_bounds__(SH::THREADS, 1)
 umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_constant__ WgradUpdateParams p) {
     constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
@@ -263,7 +277,15 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES - (LOAD_Z ? 0 : WU_ARRAY_BYTES));   // STATE_BYTES counts v when MOM
                     tma_load_3d(dst, &maps.x[l], fb, m0, nb, g);
                     if (!FIRST) {
-                        tma_load_3d(dst + WU_ARRAY_BYTES, &maps.y[l], fb, m0, nb, g);
+                        if (YSPLIT) {
+                            // hi plane: rows nb % 128 .. of the two 64-column blocks under this tile; lo plane: one box
+                            const uint32_t yd = dst + WU_ARRAY_BYTES;
+                            tma_load_5d(yd, &maps.yhi[l], fb, 0, nb & 127, m0 >> 6, nb >> 7, g);
+                            tma_load_5d(yd + WU_ARRAY_BYTES / 4, &maps.yhi[l], fb, 0, nb & 127, (m0 >> 6) + 1, nb >> 7, g);
+                            tma_load_3d(yd + WU_ARRAY_BYTES / 2, &maps.ylo[l], fb, m0, nb, g);
+                        } else {
+                            tma_load_3d(dst + WU_ARRAY_BYTES, &maps.y[l], fb, m0, nb, g);
+                        }
                         if (LOAD_Z) tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &maps.z[l], fb, m0, nb, g);
                         if (MOM) tma_load_3d(dst + 3 * WU_ARRAY_BYTES, &maps.v[l], fb, m0, nb, g);
                     }
@@ -309,6 +331,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
             const long long tile_e0 = (long long)g * p.gs + p.layer[l].w_off + (long long)(n0 + grp * RPG) * ld + m;
             const long long chunk_step = (long long)WU_CHUNK_ROWS * ld;
             float *yp = p.y + tile_e0, *zp = p.z + tile_e0;
+            uint16_t *lp = YSPLIT ? p.ylo + tile_e0 : nullptr;
             float *vp = MOM ? p.v + tile_e0 : nullptr;
             // blocked copy: W row r, column m live in block (r/128, m/64) at (r%128)*64 + m%64; n0 % 128 == 0
             __nv_bfloat16 *sp = p.shadow + (long long)g * p.shadow_gs + p.layer[l].shadow_off +
@@ -317,6 +340,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
 #pragma unroll 1
             for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
                 if (MOM && c > 0) vp += chunk_step;
+                if (YSPLIT && c > 0) lp += chunk_step;
                 const int nb0 = n0 + c * WU_CHUNK_ROWS;
                 if (nb0 >= N) break;                         // same rule as the loader
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
@@ -329,7 +353,15 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                 for (int j = 0; j < RPG; ++j) {
                     xv[j] = sx[j * UM_BM];
                     if (!FIRST) {
-                        yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
+                        if (YSPLIT) {
+                            const uint16_t *sy = reinterpret_cast<const uint16_t *>(st_ptr + (size_t)stage * WU_STATE_BYTES + WU_ARRAY_BYTES);
+                            const int rr = grp * RPG + j;
+                            const uint32_t hi = sy[(col >> 6) * (WU_CHUNK_ROWS * 64) + rr * 64 + (col & 63)];
+                            const uint32_t lo = sy[WU_CHUNK_ROWS * 128 + rr * UM_BM + col];
+                            yv[j] = __uint_as_float(((hi - (lo > 0x8000u ? 1u : 0u)) << 16) | lo);
+                        } else {
+                            yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
+                        }
                         if (USE_Z) zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                         if (MOM) vv[j] = sx[3 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                     }
@@ -344,6 +376,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                 if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
                 const int rows = m_ok ? (N - nb) : 0;        // rows of this thread that exist
                 float *yr = yp, *zr = zp, *vr = vp;
+                uint16_t *lr = lp;
                 __nv_bfloat16 *sr = sp;
                 auto update_row = [&](int j) {
                     const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : (USE_Z ? zv[j] : 0.f);
@@ -355,7 +388,15 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     }
                     const float yn = fmaf(neg_eta_p, d, yo);
                     chk = fmaf(yn, 0.f, chk);
-                    *yr = yn;
+                    if (YSPLIT) {
+                        const uint32_t u = __float_as_uint(yn);
+                        uint32_t lo = u & 0xFFFFu;
+                        if (lo == 0x8000u && ((u >> 16) & 1u)) lo = 0x8001u;     // tie that rounds up: see the head of this file
+                        *lr = (uint16_t)lo;
+                        if (p.write_y) *yr = __uint_as_float((u & 0xFFFF0000u) | lo);
+                    } else {
+                        *yr = yn;
+                    }
                     if (USE_Z) {
                         const float zn = (!FIRST && ZMODE == WU_Z_DOUBLE) ? fmaf(alpha_sq, zo, one_m_alpha * fmaf(p.alpha, yo, yn))
                                                                            : fmaf(p.alpha, zo, one_m_alpha * yn);
@@ -368,12 +409,14 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     for (int j = 0; j < RPG; ++j, yr += ld, zr += ld, sr += 64) {
                         update_row(j);
                         if (MOM) vr += ld;
+                        if (YSPLIT) lr += ld;
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < RPG; ++j, yr += ld, zr += ld, sr += 64) {
                         if (j < rows) update_row(j);
                         if (MOM) vr += ld;
+                        if (YSPLIT) lr += ld;
                     }
                 }
             }

@@ -36,6 +36,7 @@ def make(cfg, fused=None, t3=None, **over):
     if fused is not None and cfg.gemm_dtype == pb.GEMM_BF16:
         m.set_fused_update(fused)
         m.set_paired_z_update(False)      # tests that name the path compare it bit for bit with the other one: z step by step in both
+        m.set_split_y(False)              # ... and y as fp32 words at every step
     if t3 is not None and cfg.gemm_dtype == pb.GEMM_FP32:
         m.set_fp32_tensor_cores(t3)
         assert m.fp32_tensor_cores_active == (t3 == 2)
@@ -661,3 +662,34 @@ def test_paired_z_update_is_the_same_recurrence(L, mu, gemm_dtype, t3):
     # (and momentum amplifies that): a tenth of the bf16 parity bound
     for a, b in zip(res[0][1], res[1][1]):
         assert rel_l2(a, b) < (2e-3 if gemm_dtype == 1 else 2e-5)
+
+
+@pytest.mark.parametrize("L", [1, 2, 5])
+@pytest.mark.parametrize("mu", [0.0, 0.9])
+@pytest.mark.parametrize("dims,batch", [((200, 328, 136, 101), 136), ((64, 128, 72, 10), 16)])
+def test_split_y_rounds_keep_y_exactly_bf16(L, mu, dims, batch):
+    """Inside a whole round the fused kernel keeps y of the weights as bf16 operand copy + lower-half plane and stores the
+    fp32 y again at the last step.  Against rounds with fp32 y at every step, after the first round: the same y up to the
+    documented one-ulp move of tie values (lower half 0x8000 under an odd upper half), hence z, x, xbar to fp32 rounding."""
+    cfg = si.C1.scaled(name="splity", n=3, dims=dims, batch=batch, gemm_dtype=1, L=L)
+    res = []
+    for split in (True, False):
+        m, *_ = make(cfg)
+        m.set_split_y(split)
+        if mu:
+            m.set_momentum(mu)
+        X, c = si.round_batches(cfg, 0)
+        m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV))
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        res.append([t.cpu().numpy() for t in (m.y, m.z, m.x, m.xbar)])
+        X, c = si.round_batches(cfg, 1)                 # a second round starts from x again: must still run clean
+        m.round(cfg.L, torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV))
+        torch.cuda.synchronize()
+        assert m.status() == 0
+    (y1, z1, x1, b1), (y0, z0, x0, b0) = res
+    diff = y1 != y0
+    assert diff.mean() < 1e-3, diff.mean()
+    assert np.all(np.abs(y1.astype(np.float64) - y0) <= 4 * np.spacing(np.abs(y0)))
+    for a, b in ((z1, z0), (x1, x0), (b1, b0)):
+        assert rel_l2(a, b) < 1e-6
