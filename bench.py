@@ -116,10 +116,10 @@ def dense_to_padded(model, cfg, replica_layers):
 # (profiles/ncu_full_gemms_and_fused_update_C3.md), valid only while the kernel source is unchanged.
 NCU_TRAFFIC = {("C3", "wgrad_gemm_fused_update"): {
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch (all layers, all replicas): mean of the two variants
-    # that alternate inside a round, "z untouched" (984.4 + 663.6 MB) and "two-step z" (1462.5 + 1135.8 MB)
-    "bytes": (984.443e6 + 663.629e6 + 1462.463e6 + 1135.813e6) / 2,
+    # that alternate inside a round, "z untouched" (985.3 + 433.0 MB) and "two-step z" (1462.6 + 900.7 MB)
+    "bytes": (985.298e6 + 432.966e6 + 1462.564e6 + 900.722e6) / 2,
     "sources": ("paper_1707_00424_b200/csrc/umma_wgrad_update.cuh", "paper_1707_00424_b200/csrc/umma_gemm.cuh"),
-    "sources_sha256_16": "72d91c0118922456"}}
+    "sources_sha256_16": "45c6fe3d686ff3ef"}}
 
 
 def sources_digest(sources):
