@@ -343,7 +343,8 @@ def run_ours(args):
         "config": {"workload": f"{cfg.name}: n={cfg.n} replicas/GPU, MLP {'-'.join(map(str, cfg.dims))}, batch {cfg.batch}, L={cfg.L}, "
                                f"{'bf16 GEMM operands, fp32 master state' if cfg.gemm_dtype == 1 else ('fp32 (products as 3 x tf32 on the tensor cores)' if t3 else 'fp32 (FMA pipes)')}",
                    "step": "one Parle round (L inner steps + outer step + replica mean)" +
-                           ("; z updated every other inner step with the two-step form of Eq. (parle_z)" if args.paired_z else ""),
+                           ("; z updated every other inner step with the two-step form of Eq. (parle_z)" if args.paired_z else "") +
+                           ("; y of the weights kept as bf16 operand copy + lower-half plane inside the round" if cfg.gemm_dtype == 1 and args.split_y else ""),
                    "l2": "state + gradients per round >> 126 MB L2 (no flush needed)" if cfg.n * model.stride * 16 > 4e8 else "working set may be L2 resident",
                    "launch": "rounds replayed from CUDA graphs (same kernels, same order)" if args.graphs else "one launch per kernel",
                    "parallelism": f"{world} x {cfg.n} replicas, one all-reduce of xbar per round" if world > 1 else "single GPU"},
