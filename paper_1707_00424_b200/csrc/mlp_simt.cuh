@@ -246,32 +246,23 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
     const int lane = threadIdx.x % 32;
     if (row >= rows) return;
     float *lg = logits + (size_t)row * C;
-    if (parts > 1) {
-        const float *bg = bias + (long long)(row / B) * bias_gs;
-        for (int j = lane; j < C; j += 32) {
-            float pv[8];                             // parts <= 8: all loads in flight before the fixed-order sum
-#pragma unroll
-            for (int q = 0; q < 8; ++q) pv[q] = (q < parts) ? lg[(long long)q * part_stride + j] : 0.f;
-            float s = pv[0];
-#pragma unroll
-            for (int q = 1; q < 8; ++q) s += pv[q];
-            lg[j] = s + bg[j];                       // read back below by the same lane
-        }
-    }
-    float mx = -INFINITY;
-    for (int j = lane; j < C; j += 32) mx = fmaxf(mx, lg[j]);
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float s = 0.f;
-    for (int j = lane; j < C; j += 32) s += __expf(lg[j] - mx);
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     const int label = labels[row];
     const bool label_ok = (label >= 0 && label < C);
-    const float inv_s = 1.f / s, inv_B = 1.f / (float)B;
+    const float inv_B = 1.f / (float)B;
     const int g = row / B, i = row % B;
-    for (int j = lane; j < C; j += 32) {
-        float d = __expf(lg[j] - mx) * inv_s;
-        if (j == label) d -= 1.f;
-        d *= inv_B;
+    const float *bg = parts > 1 ? bias + (long long)g * bias_gs : nullptr;
+    // logit j of this row: with split-K partial sums, bias + sum_s part_s in fixed order (all loads in flight first)
+    auto logit = [&](int j) -> float {
+        if (parts <= 1) return lg[j];
+        float pv[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) pv[q] = (q < parts) ? lg[(long long)q * part_stride + j] : 0.f;
+        float s = pv[0];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) s += pv[q];
+        return s + bg[j];
+    };
+    auto emit = [&](int j, float d) {                // d = dlogits[row, j]
         if (d32) d32[(size_t)row * C + j] = d;
         if (dbf) {
             const __nv_bfloat16 h = __float2bfloat16_rn(d);
@@ -286,9 +277,53 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
             dhi[(size_t)row * ld_split + j] = hi;
             dlo[(size_t)row * ld_split + j] = lo;
         }
+    };
+    constexpr int VR = 4;                            // up to 128 classes: the row stays in registers (one pass over memory)
+    float mx = -INFINITY, s = 0.f, label_logit = 0.f;
+    if (C <= 32 * VR) {
+        float v[VR];
+#pragma unroll
+        for (int k = 0; k < VR; ++k) {
+            const int j = lane + 32 * k;
+            v[k] = j < C ? logit(j) : -INFINITY;
+            if (parts > 1 && j < C) lg[j] = v[k];    // the logits buffer then holds the complete logits
+            mx = fmaxf(mx, v[k]);
+        }
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+        for (int k = 0; k < VR; ++k)
+            if (lane + 32 * k < C) s += __expf(v[k] - mx);
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float inv_s = 1.f / s;
+        float cand = 0.f;
+#pragma unroll
+        for (int k = 0; k < VR; ++k) {
+            const int j = lane + 32 * k;
+            if (k == (label >> 5)) cand = v[k];
+            if (j < C) {
+                float d = __expf(v[k] - mx) * inv_s;
+                if (j == label) d -= 1.f;
+                emit(j, d * inv_B);
+            }
+        }
+        label_logit = __shfl_sync(0xffffffffu, cand, label & 31);
+    } else {
+        if (parts > 1)
+            for (int j = lane; j < C; j += 32) lg[j] = logit(j);      // read back below by the same lane
+        for (int j = lane; j < C; j += 32) mx = fmaxf(mx, lg[j]);
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        for (int j = lane; j < C; j += 32) s += __expf(lg[j] - mx);
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float inv_s = 1.f / s;
+        for (int j = lane; j < C; j += 32) {
+            float d = __expf(lg[j] - mx) * inv_s;
+            if (j == label) d -= 1.f;
+            emit(j, d * inv_B);
+        }
+        if (lane == 0 && label_ok) label_logit = lg[label];
     }
     if (lane == 0) {
-        row_loss[row] = label_ok ? (mx + __logf(s) - lg[label]) : 0.f;
+        row_loss[row] = label_ok ? (mx + __logf(s) - label_logit) : 0.f;
         if (!label_ok) status[SLOT_BAD_LABEL] = 1;
     }
 }
