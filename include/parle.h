@@ -230,7 +230,8 @@ int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
  * parle_bind_momentum attaches the two caller-owned buffers, dev [n, stride] fp32, 128-byte aligned;
  * vx must be zero before the first round (vy needs no initialisation).  parle_set_momentum(mu), mu in
  * [0, 1): 0 switches momentum off; ENOTBOUND if mu > 0 without buffers, ESTATE in the middle of a round.
- * Call parle_bind_momentum after parle_bind (and again after every later parle_bind).  On the bf16 path the
+ * Call parle_bind_momentum after parle_bind.  A later parle_bind detaches the momentum buffers and sets mu back to 0:
+ * call parle_bind_momentum and parle_set_momentum again after it.  On the bf16 path the
  * fused weight-gradient kernel has a momentum variant (vy is staged with x, y, z: 30 bytes per weight and step). */
 int parle_bind_momentum(parle_ctx *ctx, float *vy, float *vx);
 int parle_set_momentum(parle_ctx *ctx, double mu);
@@ -242,7 +243,7 @@ int parle_set_momentum(parle_ctx *ctx, double mu);
 int parle_scoping(double gamma0, double rho0, long long minibatches_per_epoch, long long round,
                   double gamma_floor, double rho_floor, double *gamma, double *rho);
 
-/* Weight-decay regulariser of f (Section 1.1: "along with a regularization term (say weight decay)"):
+/* Weight-decay regulariser of f (Section 1.1 allows f a regularisation term and names weight decay):
  * parle_inner_step uses grad f(y) + lambda * y in Eq. (parle_y), for every parameter.  Default 0.
  * loss_out stays the data term alone.  parle_inner_update applies its gradient argument as given. */
 int parle_set_weight_decay(parle_ctx *ctx, double lambda);

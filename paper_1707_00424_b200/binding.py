@@ -205,6 +205,7 @@ class Parle:
         with torch.cuda.device(x.device):
             self._check(self._L.parle_bind(self._h, C.byref(b), C.c_void_p(sp)), "parle_bind")
         self.x, self.y, self.z, self.grad, self.xbar, self.workspace = x, y, z, grad, xbar, workspace
+        self._momentum_bound = False          # parle_bind detaches the momentum buffers
 
     # -- the round --------------------------------------------------------
     def round_begin(self):
@@ -249,10 +250,12 @@ class Parle:
     def set_momentum(self, mu: float, vy=None, vx=None):
         """Nesterov momentum on the y and x^a steps; allocates (zeroed) vy, vx with torch when not given."""
         import torch
-        if mu > 0 and getattr(self, "vy", None) is None:
-            self.vy = vy if vy is not None else torch.zeros_like(self.x)
-            self.vx = vx if vx is not None else torch.zeros_like(self.x)
+        if mu > 0 and not getattr(self, "_momentum_bound", False):
+            have = getattr(self, "vy", None) is not None
+            self.vy = vy if vy is not None else (self.vy if have else torch.zeros_like(self.x))
+            self.vx = vx if vx is not None else (self.vx if have else torch.zeros_like(self.x))
             self._check(self._L.parle_bind_momentum(self._h, _ptr(self.vy), _ptr(self.vx)), "parle_bind_momentum")
+            self._momentum_bound = True
         self._check(self._L.parle_set_momentum(self._h, mu), "parle_set_momentum")
 
     def set_wide_tile_threshold(self, tiles_per_sm: int):

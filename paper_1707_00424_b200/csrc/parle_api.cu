@@ -17,6 +17,10 @@ namespace {
 
 constexpr size_t kWsAlign = 1024;
 constexpr int kProfCapacity = 65536;       // launches recorded between two parle_profile_read calls
+// SM count the split-K factors of the last forward layer are planned for.  They are fixed at parle_init (the size
+// of the workspace depends on them) where no device is known yet; the launches themselves use the bound device's
+// count.  On a part with another count the split is merely sized for 148.
+constexpr int kPlanSmCount = 148;
 
 enum KernelClass {
     KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_LOSS_MEAN, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
@@ -935,7 +939,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         const int nl = c->n_layers;
         const int tiles = c->n * ((c->batch + 127) / 128) * ((c->dims[nl] + 63) / 64);
         const int num_kb = (c->dims[nl - 1] + 31) / 32;
-        int s = 148 / (tiles > 0 ? tiles : 1);
+        int s = kPlanSmCount / (tiles > 0 ? tiles : 1);
         if (s > 8) s = 8;
         if (s > num_kb / 2) s = num_kb / 2;
         if (s >= 2) c->t3_ksplit = s;
@@ -951,7 +955,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         const int nl = c->n_layers;
         const int tiles = c->n * ((c->batch + 127) / 128) * ((c->dims[nl] + 127) / 128);
         const int num_kb = (c->dims[nl - 1] + 63) / 64;
-        int s = 148 / (tiles > 0 ? tiles : 1);
+        int s = kPlanSmCount / (tiles > 0 ? tiles : 1);
         if (s > 8) s = 8;
         if (s > num_kb / 2) s = num_kb / 2;
         if (s >= 2) c->last_ksplit = s;
@@ -1009,6 +1013,9 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
     }
     c->buf = *b;
     c->stream = static_cast<cudaStream_t>(cuda_stream);
+    // the momentum buffers (and the tensor maps over them) belonged to the previous binding: momentum is off until
+    // parle_bind_momentum and parle_set_momentum are called again
+    c->momentum = 0.f; c->vy = nullptr; c->vx = nullptr; c->mom_maps = false;
     if (c->n_layers > 0 && c->gemm_dtype == PARLE_GEMM_BF16) {
         int major = 0;
         PARLE_CUDA(c, cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
@@ -1106,7 +1113,8 @@ int parle_inner_update(parle_ctx *c, const float *grad) {
     if (!grad) return PARLE_EINVAL;
     if (reinterpret_cast<uintptr_t>(grad) % 16) return PARLE_EALIGN;
     if (!c->round_open) return PARLE_ESTATE;
-    return run_inner_update(c, grad, 0.f);
+    // the operand copies of the active GEMM path follow y: a later parle_inner_step of the same round reads them
+    return run_inner_update(c, grad, 0.f, use_t3(c));
 }
 
 int parle_outer_step(parle_ctx *c) {

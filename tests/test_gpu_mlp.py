@@ -1,13 +1,14 @@
 """GPU parity of the whole round (forward/backward, Eq. parle_y .. parle_x)
 against the fp64 oracle on seeded inputs, through the C ABI.
 
-Bounds: relative L2 error of every parameter tensor (x^a, xbar) after a round
-<= 1e-4 for fp32 GEMMs and <= 2e-2 for bf16 GEMM operands.  The inner iterates
-y^a, z^a are compared too; at the MNIST-shaped workload the inner loop runs at
-the edge of stability (eta' = 0.1 against a large top Hessian eigenvalue from
-the all-positive inputs), which amplifies fp32 rounding of *any* fp32
-implementation by up to ~1e4 over 25 steps, so y and z get 10x the fp32 bound;
-the per-step gradient check at the same shape shows the kernels themselves
+Bounds: relative L2 error of every parameter tensor (x^a, xbar) and of the inner
+iterates y^a, z^a after a round <= 1e-4 for fp32 GEMMs and <= 2e-2 for bf16 GEMM
+operands.  One exception: at the MNIST-shaped workload (C2) y^a and z^a get 1e-3.
+There the fp64 trajectory passes within 6e-8 of a ReLU kink, either side of which
+an fp32 evaluation may land, and the inner loop (at the edge of stability with
+all-positive inputs) enlarges the difference to 3.5e-4 in y^a;
+tests/test_fp32_relu_kink_sensitivity.py shows this on the CPU with the oracle
+alone.  The per-step gradient check at the same shape shows the kernels themselves
 are accurate to 1e-5."""
 import math
 
@@ -57,7 +58,9 @@ def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False, fused=None, t3=
         loss = torch.zeros(cfg.L, cfg.n, device=DEV)
         if use_round_call:
             m.round(cfg.L, Xd, cd, loss)
-            y_gpu = z_gpu = None
+            torch.cuda.synchronize()
+            # the outer step leaves y and z alone: they still hold the inner loop's last values
+            y_gpu, z_gpu = to_dense(m, m.y.cpu().numpy()), to_dense(m, m.z.cpu().numpy())
         else:
             m.round_begin()
             for l in range(cfg.L):
@@ -71,10 +74,9 @@ def run_rounds(cfg, rounds, disp_tol=None, use_round_call=False, fused=None, t3=
         errs = {"xbar": rel_l2(xb_gpu, out["xbar"])}
         for a in range(cfg.n):
             errs[f"x{a}"] = rel_l2(x_gpu[a], out["x"][a])
-            if y_gpu is not None:
-                errs[f"y{a}"] = rel_l2(y_gpu[a], out["y"][a])
-                errs[f"z{a}"] = rel_l2(z_gpu[a], out["z"][a])
-        tol_inner = tol * (10 if cfg.gemm_dtype == pb.GEMM_FP32 else 1)
+            errs[f"y{a}"] = rel_l2(y_gpu[a], out["y"][a])
+            errs[f"z{a}"] = rel_l2(z_gpu[a], out["z"][a])
+        tol_inner = tol * (10 if cfg.name == "C2" else 1)      # see the head of this file
         bad = {k: v for k, v in errs.items() if v > (tol_inner if k[0] in "yz" else tol)}
         assert not bad, (bad, errs)
         # stricter, on the displacement of the round (what the round actually computed)
@@ -239,7 +241,9 @@ def test_c2_gradient_full_shape_fp32(t3):
 
 @pytest.mark.parametrize("t3", [0, None])
 def test_c2_one_round_fp32(t3):
-    m = run_rounds(si.C2, 1, t3=t3)
+    # displacement: one ReLU unit landing on the other side of its kink moves a replica's displacement by 2e-2
+    # (tests/test_fp32_relu_kink_sensitivity.py); over all 8 replicas that is 7e-3
+    m = run_rounds(si.C2, 1, disp_tol=3e-2, t3=t3)
     assert m.fp32_tensor_cores_active == (t3 is None)      # the default puts this shape on the tensor cores
 
 
@@ -403,7 +407,8 @@ def test_layerwise_teacher_forced_ragged_bf16():
 def test_c5_widths_div8_round_bf16():
     """Same depth, replica count and batch as the largest workload, widths / 8 (a full fp64 round at
     full width is ~1e17 flop): whole-round parity, fused update."""
-    cfg = si.C5.scaled(name="C5/8", dims=(512, 1024, 1024, 1024, 1024, 125), L=5)
+    cfg = si.C5.scaled(name="C5/8", dims=(512, 1024, 1024, 1024, 1024, 125))
+    assert cfg.L == 25 and cfg.n == 16 and cfg.batch == 256
     run_rounds(cfg, 1, disp_tol=5e-2, use_round_call=True)
 
 
@@ -693,3 +698,50 @@ def test_split_y_rounds_keep_y_exactly_bf16(L, mu, dims, batch):
     assert np.all(np.abs(y1.astype(np.float64) - y0) <= 4 * np.spacing(np.abs(y0)))
     for a, b in ((z1, z0), (x1, x0), (b1, b0)):
         assert rel_l2(a, b) < 1e-6
+
+
+@pytest.mark.parametrize("t3", [0, 2])
+def test_inner_update_then_inner_step_in_one_round_fp32(t3):
+    """parle_inner_update followed by parle_inner_step inside the same round: the step's forward/backward must see
+    the y the update produced (on the tensor-core path that means its tf32 operand copies were refreshed too)."""
+    cfg = si.C1.scaled(name="mixed", n=2, dims=(64, 128, 72, 12), batch=16, L=2)
+    m, xo, xb, hp = make(cfg, t3=t3)
+    X, c = si.round_batches(cfg, 0)
+    g0 = np.stack([po.mlp_loss_grad(xo[a], cfg.dims, X[0, a], c[0, a])[1] for a in range(cfg.n)])   # oracle gradient at x
+    m.round_begin()
+    m.inner_update(torch.from_numpy(to_padded(m, g0)).to(DEV))
+    m.inner_step(torch.from_numpy(X[1]).to(DEV), torch.from_numpy(c[1]).to(DEV))
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    y_gpu, z_gpu = to_dense(m, m.y.cpu().numpy()), to_dense(m, m.z.cpu().numpy())
+    for a in range(cfg.n):
+        y, z = po.inner_step(xo[a], xo[a], xo[a], g0[a], hp)
+        _, g1 = po.mlp_loss_grad(y, cfg.dims, X[1, a], c[1, a])
+        y2, z2 = po.inner_step(y, z, xo[a], g1, hp)
+        assert rel_l2(y_gpu[a], y2) <= 1e-6 and rel_l2(z_gpu[a], z2) <= 1e-6
+        assert rel_l2(y_gpu[a] - y, y2 - y) <= 1e-4              # the second step alone: a stale operand copy gives ~1
+
+
+def test_rebinding_detaches_momentum_bf16():
+    """After a second parle_bind the momentum buffers of the first binding are gone: momentum is off, switching it on
+    needs parle_bind_momentum again, and the rounds that follow equal those of a context bound once."""
+    cfg = si.C1.scaled(name="rebind", n=2, dims=(64, 128, 72, 10), batch=16, gemm_dtype=1, L=3, eta_prime=0.02)
+    X, c = si.round_batches(cfg, 0)
+    Xd, cd = torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)
+    ref, *_ = make(cfg)
+    ref.set_momentum(0.9)
+    ref.round(cfg.L, Xd, cd); torch.cuda.synchronize()
+    m, *_ = make(cfg)
+    m.set_momentum(0.9)
+    x_start = m.x.clone()
+    m.round(cfg.L, Xd, cd); torch.cuda.synchronize()
+    old = (m.x, m.y, m.z, m.grad, m.xbar, m.workspace, m.vy, m.vx)     # keep the first binding's buffers alive
+    m.alloc(DEV)                                                       # new buffers, bound with parle_bind
+    m.x.copy_(x_start); m.mean()
+    assert pb.lib().parle_set_momentum(m._h, 0.9) == -2                # ENOTBOUND: no momentum buffers on this binding
+    m.vy = m.vx = None
+    m.set_momentum(0.9)                                                # binds fresh (zeroed) buffers, then switches it on
+    m.round(cfg.L, Xd, cd); torch.cuda.synchronize()
+    assert m.status() == 0
+    assert torch.equal(m.x, ref.x) and torch.equal(m.vx, ref.vx) and torch.equal(m.xbar, ref.xbar)
+    del old

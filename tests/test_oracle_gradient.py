@@ -150,3 +150,67 @@ def test_bf16_rounding_helper_and_rounded_mode():
     assert abs(l0 - l1) < 1e-14 and np.allclose(g0, g1, rtol=1e-13, atol=1e-15)
     l2, g2 = po.mlp_loss_grad(vec, dims, X, c, operand_rounding=po.round_to_bf16)
     assert 0 < np.linalg.norm(g2 - g0) / np.linalg.norm(g0) < 0.05
+
+
+def _wd_fd_ok(vec, dims, X, c, lam):
+    _, g = po.mlp_loss_grad(vec, dims, X, c, weight_decay=lam)
+    h = 1e-6
+    for i in range(vec.size):
+        e = np.zeros_like(vec); e[i] = h
+        fd = (po.mlp_loss_grad(vec + e, dims, X, c, weight_decay=lam)[0]
+              - po.mlp_loss_grad(vec - e, dims, X, c, weight_decay=lam)[0]) / (2 * h)
+        if abs(fd - g[i]) > 1e-6 * max(1.0, abs(g[i])):
+            return False
+    return True
+
+
+def test_weight_decay_term_of_f():
+    """Section 1.1 lets f carry a regulariser besides the average loss and names weight decay as the example.  The
+    reading taken is f(y) = data term + (lambda/2) |y|^2 over every parameter: the loss grows by exactly that amount,
+    the gradient by lambda y, central differences of the regularised loss give the regularised gradient, and the
+    regulariser's own second derivative is lambda."""
+    dims, B, lam = (5, 4, 3), 3, 0.37
+    vec, X, c = _rand_problem(dims, B, seed=21)
+    l0, g0 = po.mlp_loss_grad(vec, dims, X, c)
+    l1, g1 = po.mlp_loss_grad(vec, dims, X, c, weight_decay=lam)
+    assert abs((l1 - l0) - 0.5 * lam * sum(v * v for v in vec.tolist())) < 1e-13     # the sum written out in Python
+    np.testing.assert_allclose(g1 - g0, lam * vec, rtol=1e-13, atol=1e-15)
+    assert _wd_fd_ok(vec, dims, X, c, lam)
+    # second derivative of the regulariser alone, by differencing the gradient: lambda on the diagonal
+    e = np.zeros_like(vec); e[7] = 1e-5
+    gp = po.mlp_loss_grad(vec + e, dims, X, c, weight_decay=lam)[1] - po.mlp_loss_grad(vec + e, dims, X, c)[1]
+    gm = po.mlp_loss_grad(vec - e, dims, X, c, weight_decay=lam)[1] - po.mlp_loss_grad(vec - e, dims, X, c)[1]
+    np.testing.assert_allclose((gp - gm)[7] / 2e-5, lam, rtol=1e-9)
+
+
+def test_planted_weight_decay_mistakes_are_caught(monkeypatch):
+    """A dropped 1/2 in the regulariser's loss, a flipped sign of its gradient, or decay applied to the weights but
+    not the biases each break the pin above."""
+    dims, B, lam = (5, 4, 3), 3, 0.37
+    vec, X, c = _rand_problem(dims, B, seed=21)
+    assert _wd_fd_ok(vec, dims, X, c, lam)
+    real = po.mlp_loss_grad
+
+    def no_half(v, d, X_, c_, weight_decay=0.0, operand_rounding=None):
+        loss, g = real(v, d, X_, c_, weight_decay, operand_rounding)
+        return loss + 0.5 * weight_decay * float(np.dot(v, v)), g
+    monkeypatch.setattr(po, "mlp_loss_grad", no_half)
+    assert not _wd_fd_ok(vec, dims, X, c, lam)
+
+    def wrong_sign(v, d, X_, c_, weight_decay=0.0, operand_rounding=None):
+        loss, g = real(v, d, X_, c_, weight_decay, operand_rounding)
+        return loss, g - 2.0 * weight_decay * np.asarray(v)
+    monkeypatch.setattr(po, "mlp_loss_grad", wrong_sign)
+    assert not _wd_fd_ok(vec, dims, X, c, lam)
+
+    def weights_only(v, d, X_, c_, weight_decay=0.0, operand_rounding=None):
+        loss, g = real(v, d, X_, c_, weight_decay, operand_rounding)
+        g = g.copy()
+        o = 0
+        for l in range(len(d) - 1):
+            o += d[l + 1] * d[l]
+            g[o:o + d[l + 1]] -= weight_decay * np.asarray(v)[o:o + d[l + 1]]
+            o += d[l + 1]
+        return loss, g
+    monkeypatch.setattr(po, "mlp_loss_grad", weights_only)
+    assert not _wd_fd_ok(vec, dims, X, c, lam)

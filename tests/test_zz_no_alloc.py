@@ -57,6 +57,14 @@ def test_static_loss_matches_inner_step_twice_in_a_row():
         np.testing.assert_allclose(got_d.cpu().numpy(), want_d.cpu().numpy(), rtol=1e-6, atol=1e-7)
         np.testing.assert_allclose(got_loss.cpu().numpy(), want_loss.cpu().numpy(), rtol=1e-6, atol=1e-7)
         assert flags.item() == 0
+        # and against the oracle's softmax cross-entropy on the same logits, replica by replica
+        lg = logits.cpu().numpy().astype(np.float64).reshape(cfg.n, cfg.batch, C)
+        lab = labels.cpu().numpy().reshape(cfg.n, cfg.batch)
+        gd = got_d.cpu().numpy().reshape(cfg.n, cfg.batch, -1)[:, :, :C]
+        for a in range(cfg.n):
+            want_l, want_dl = po.softmax_ce(lg[a], lab[a])
+            np.testing.assert_allclose(gd[a], want_dl, rtol=1e-5, atol=1e-7)
+            assert abs(got_loss[a].item() - want_l) <= 1e-5 * max(1.0, abs(want_l))
 
 
 def test_static_loss_flags_bad_labels_and_then_clears():
