@@ -85,12 +85,12 @@ def test_flat_vectors_past_2_to_31_elements_match_oracle_on_slices():
 
 
 def test_network_past_2_to_31_elements_fused_equals_separate_update_bf16():
-    """The 243 M-parameter shape with nine replicas: the last replica's parameters start beyond element 2^31.
-    Two inner steps (the first of a round and a later one): the fused kernel's y, z and bf16 operand copy of the
-    last replica equal, bit for bit, what the weight-gradient product + separate update kernel give; sampled
+    """The 243 M-parameter shape with ten replicas: element 2^31 falls inside replica 8, replica 9 lies wholly beyond it.
+    Two inner steps (the first of a round and a later one): the fused kernel's y, z (last two replicas) and bf16 operand
+    copy (last replica) equal, bit for bit, what the weight-gradient product + separate update kernel give; sampled
     entries of that replica's weight gradient are recomputed in fp64 from the operands the GPU used."""
-    cfg = si.C5.scaled(name="C5x9", n=9, L=2)
-    _need(60)
+    cfg = si.C5.scaled(name="C5x10", n=10, L=2)
+    _need(70)
     last = cfg.n - 1
     X, c = si.round_batches(cfg, 0)
     Xd, cd = torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)
@@ -98,7 +98,7 @@ def test_network_past_2_to_31_elements_fused_equals_separate_update_bf16():
     keep = []
     for fused in (False, True):
         m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype).alloc(DEV)
-        assert last * m.stride > (1 << 31)
+        assert last * m.stride > (1 << 31) > (last - 1) * m.stride
         m.set_fused_update(fused)
         gen = torch.Generator(device=DEV).manual_seed(77)
         for a in range(cfg.n):
@@ -123,7 +123,7 @@ def test_network_past_2_to_31_elements_fused_equals_separate_update_bf16():
         m.inner_step(Xd[1], cd[1]); torch.cuda.synchronize()
         assert m.status() == 0
         keep.append((m.y[last].clone(), m.z[last].clone(), m.debug_buffer(m.DBG_OPERAND_COPY)[last].clone(),
-                     m.y[0, :1 << 20].clone()))
+                     m.y[last - 1].clone(), m.z[last - 1].clone(), m.y[0, :1 << 20].clone()))
         del m
         torch.cuda.empty_cache()
     for a, b in zip(*keep):
