@@ -819,10 +819,11 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     if (mom) { p.v = c->vy; p.mu = c->momentum; }
     const WuMaps &maps = mom ? c->wu_maps_mom : c->wu_maps;
 #define PARLE_WU_LAUNCH(FIRST, SH, MOM, ZM) do { \
-        if (ys) umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); \
-        else umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); } while (0)
-    const bool ys = c->y_split_step;
-    p.ylo = ws_ptr<uint16_t>(c, w.ylo); p.write_y = c->y_write_step ? 1 : 0;
+        if (ys && yw) umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true, true><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); \
+        else if (ys) umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true, false><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); \
+        else umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false, false><<<grid, SH::THREADS, SH::SMEM_BYTES, c->stream>>>(maps, p); } while (0)
+    const bool ys = c->y_split_step, yw = c->y_write_step;
+    p.ylo = ws_ptr<uint16_t>(c, w.ylo);
     if (mom) {
         if (c->fresh) PARLE_WU_LAUNCH(true, WuMomentum, true, WU_Z_SINGLE);
         else if (zm == WU_Z_SKIP) PARLE_WU_LAUNCH(false, WuMomentum, true, WU_Z_SKIP);
@@ -1024,8 +1025,9 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, UB_BLOCKED_K>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, UB_ROWMAJOR_K>()));
 #define PARLE_WU_SMEM(FIRST, SH, MOM, ZM) \
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES)); \
-        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES))
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES)); \
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES)); \
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES))
         PARLE_WU_SMEM(true, WuDefault, false, WU_Z_SINGLE); PARLE_WU_SMEM(false, WuDefault, false, WU_Z_SINGLE);
         PARLE_WU_SMEM(false, WuDefault, false, WU_Z_SKIP); PARLE_WU_SMEM(false, WuDefault, false, WU_Z_DOUBLE);
         PARLE_WU_SMEM(true, WuMomentum, true, WU_Z_SINGLE); PARLE_WU_SMEM(false, WuMomentum, true, WU_Z_SINGLE);

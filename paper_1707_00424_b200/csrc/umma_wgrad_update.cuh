@@ -111,7 +111,6 @@ struct WgradUpdateParams {
     long long gs;
     float eta_p, inv_gamma, alpha, wd;
     uint16_t *ylo;               // YSPLIT: low halves of the fp32 words of y (same addressing as y); the high halves are `shadow`
-    int write_y;                 // YSPLIT: also store the fp32 y (last step of a round)
     float *v; float mu;          // Nesterov momentum buffer of y (same addressing as y), used by the MOM variant
     int *sched;                  // sched[0]: tiles claimed beyond the first of every CTA, sched[1]: CTAs that have left; both 0 between launches
     int *status;
@@ -130,8 +129,10 @@ struct WuMaps {
 // v = 0 at the start of a round (FIRST: v is only written).
 // ZMODE (ignored when FIRST): 0 = z <- alpha z + (1-alpha) y_new; 1 = z untouched; 2 = z <- alpha^2 z + (1-alpha)(alpha y_old + y_new).
 constexpr int WU_Z_SINGLE = 0, WU_Z_SKIP = 1, WU_Z_DOUBLE = 2;
-// YSPLIT: y is read and written as two 16-bit planes (see the head of this file).
-template <bool FIRST, class SH, bool MOM = false, int ZMODE = WU_Z_SINGLE, bool YSPLIT = false>
+// YSPLIT: y is read and written as two 16-bit planes (see the head of this file); YWRITE: such a step also stores the
+// fp32 y (the last step of a round).
+template <int LD> struct WuPitch { static constexpr int value = LD; };
+template <bool FIRST, class SH, bool MOM = false, int ZMODE = WU_Z_SINGLE, bool YSPLIT = false, bool YWRITE = false>
 __global__ void __launch_bounds__(SH::THREADS, 1)
 umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_constant__ WgradUpdateParams p) {
     constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
@@ -337,88 +338,93 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
             __nv_bfloat16 *sp = p.shadow + (long long)g * p.shadow_gs + p.layer[l].shadow_off +
                                 ((long long)(n0 / UM_BN) * p.layer[l].shadow_cb + (m >> 6)) * (UM_BN * 64) +
                                 (grp * RPG) * 64 + (m & 63);
+            // The rows a thread owns inside a chunk are `ld` elements apart.  For the usual widths the pitch is a
+            // compile-time constant, so every row's address is the chunk pointer plus an immediate offset and the
+            // loop below carries no address arithmetic; other widths take the run-time pitch.
+            auto run_chunks = [&](auto ld_tag) {
+                constexpr int LDC = decltype(ld_tag)::value;
+                const long long ldv = LDC > 0 ? (long long)LDC : (long long)ld;
 #pragma unroll 1
-            for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
-                if (MOM && c > 0) vp += chunk_step;
-                if (YSPLIT && c > 0) lp += chunk_step;
-                const int nb0 = n0 + c * WU_CHUNK_ROWS;
-                if (nb0 >= N) break;                         // same rule as the loader
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
-                if (!ok) break;
-                const int nb = nb0 + grp * RPG;
-                const float *sx = reinterpret_cast<const float *>(st_ptr + (size_t)stage * WU_STATE_BYTES) +
-                                  grp * RPG * UM_BM + col;
-                float xv[RPG], yv[RPG], zv[RPG], vv[RPG];
+                for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
+                    if (MOM && c > 0) vp += chunk_step;
+                    if (YSPLIT && c > 0) lp += chunk_step;
+                    const int nb0 = n0 + c * WU_CHUNK_ROWS;
+                    if (nb0 >= N) break;                         // same rule as the loader
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull + 8 * stage, sphase, abort_flag));
+                    if (!ok) break;
+                    const int nb = nb0 + grp * RPG;
+                    const float *sx = reinterpret_cast<const float *>(st_ptr + (size_t)stage * WU_STATE_BYTES) +
+                                      grp * RPG * UM_BM + col;
+                    float xv[RPG], yv[RPG], zv[RPG], vv[RPG];
 #pragma unroll
-                for (int j = 0; j < RPG; ++j) {
-                    xv[j] = sx[j * UM_BM];
-                    if (!FIRST) {
-                        if (YSPLIT) {
-                            const uint16_t *sy = reinterpret_cast<const uint16_t *>(st_ptr + (size_t)stage * WU_STATE_BYTES + WU_ARRAY_BYTES);
-                            const int rr = grp * RPG + j;
-                            const uint32_t hi = sy[(col >> 6) * (WU_CHUNK_ROWS * 64) + rr * 64 + (col & 63)];
-                            const uint32_t lo = sy[WU_CHUNK_ROWS * 128 + rr * UM_BM + col];
-                            yv[j] = __uint_as_float(((hi - (lo > 0x8000u ? 1u : 0u)) << 16) | lo);
-                        } else {
-                            yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
+                    for (int j = 0; j < RPG; ++j) {
+                        xv[j] = sx[j * UM_BM];
+                        if (!FIRST) {
+                            if (YSPLIT) {
+                                const uint16_t *sy = reinterpret_cast<const uint16_t *>(st_ptr + (size_t)stage * WU_STATE_BYTES + WU_ARRAY_BYTES);
+                                const int rr = grp * RPG + j;
+                                const uint32_t hi = sy[(col >> 6) * (WU_CHUNK_ROWS * 64) + rr * 64 + (col & 63)];
+                                const uint32_t lo = sy[WU_CHUNK_ROWS * 128 + rr * UM_BM + col];
+                                yv[j] = __uint_as_float(((hi - (lo > 0x8000u ? 1u : 0u)) << 16) | lo);
+                            } else {
+                                yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
+                            }
+                            if (USE_Z) zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
+                            if (MOM) vv[j] = sx[3 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                         }
-                        if (USE_Z) zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
-                        if (MOM) vv[j] = sx[3 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                     }
-                }
-                uint32_t r[RPG];
-                tc_ld_cols<RPG>(tmem_base + ((uint32_t)(q * 32) << 16) +
-                                (uint32_t)(acc * UM_BN + c * WU_CHUNK_ROWS + grp * RPG), r);
-                tc_wait_ld();
-                // the values are in registers: hand the stage back to the loader
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
-                if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
-                const int rows = m_ok ? (N - nb) : 0;        // rows of this thread that exist
-                float *yr = yp, *zr = zp, *vr = vp;
-                uint16_t *lr = lp;
-                __nv_bfloat16 *sr = sp;
-                auto update_row = [&](int j) {
-                    const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : (USE_Z ? zv[j] : 0.f);
-                    float d = fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j])));
-                    if (MOM) {
-                        const float vn = FIRST ? d : fmaf(p.mu, vv[j], d);      // v = 0 before the first step of a round
-                        *vr = vn;
-                        d = fmaf(p.mu, vn, d);
-                    }
-                    const float yn = fmaf(neg_eta_p, d, yo);
-                    chk = fmaf(yn, 0.f, chk);
-                    if (YSPLIT) {
-                        const uint32_t u = __float_as_uint(yn);
-                        uint32_t lo = u & 0xFFFFu;
-                        if (lo == 0x8000u && ((u >> 16) & 1u)) lo = 0x8001u;     // tie that rounds up: see the head of this file
-                        *lr = (uint16_t)lo;
-                        if (p.write_y) *yr = __uint_as_float((u & 0xFFFF0000u) | lo);
+                    uint32_t r[RPG];
+                    tc_ld_cols<RPG>(tmem_base + ((uint32_t)(q * 32) << 16) +
+                                    (uint32_t)(acc * UM_BN + c * WU_CHUNK_ROWS + grp * RPG), r);
+                    tc_wait_ld();
+                    // the values are in registers: hand the stage back to the loader
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
+                    if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
+                    const int rows = m_ok ? (N - nb) : 0;        // rows of this thread that exist
+                    auto update_row = [&](int j) {
+                        const long long o = (long long)j * ldv;
+                        const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : (USE_Z ? zv[j] : 0.f);
+                        float d = fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j])));
+                        if (MOM) {
+                            const float vn = FIRST ? d : fmaf(p.mu, vv[j], d);      // v = 0 before the first step of a round
+                            vp[o] = vn;
+                            d = fmaf(p.mu, vn, d);
+                        }
+                        const float yn = fmaf(neg_eta_p, d, yo);
+                        chk = fmaf(yn, 0.f, chk);
+                        if (YSPLIT) {
+                            const uint32_t u = __float_as_uint(yn);
+                            uint32_t lo = u & 0xFFFFu;
+                            if (lo == 0x8000u && ((u >> 16) & 1u)) lo = 0x8001u;     // tie that rounds up: see the head of this file
+                            lp[o] = (uint16_t)lo;
+                            if (YWRITE) yp[o] = __uint_as_float((u & 0xFFFF0000u) | lo);
+                        } else {
+                            yp[o] = yn;
+                        }
+                        if (USE_Z) {
+                            const float zn = (!FIRST && ZMODE == WU_Z_DOUBLE) ? fmaf(alpha_sq, zo, one_m_alpha * fmaf(p.alpha, yo, yn))
+                                                                               : fmaf(p.alpha, zo, one_m_alpha * yn);
+                            zp[o] = zn;
+                        }
+                        sp[j * 64] = __float2bfloat16_rn(yn);
+                    };
+                    if (rows >= RPG) {                           // common case: no per-row bounds checks
+#pragma unroll
+                        for (int j = 0; j < RPG; ++j) update_row(j);
                     } else {
-                        *yr = yn;
-                    }
-                    if (USE_Z) {
-                        const float zn = (!FIRST && ZMODE == WU_Z_DOUBLE) ? fmaf(alpha_sq, zo, one_m_alpha * fmaf(p.alpha, yo, yn))
-                                                                           : fmaf(p.alpha, zo, one_m_alpha * yn);
-                        *zr = zn;
-                    }
-                    *sr = __float2bfloat16_rn(yn);
-                };
-                if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j, yr += ld, zr += ld, sr += 64) {
-                        update_row(j);
-                        if (MOM) vr += ld;
-                        if (YSPLIT) lr += ld;
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < RPG; ++j, yr += ld, zr += ld, sr += 64) {
-                        if (j < rows) update_row(j);
-                        if (MOM) vr += ld;
-                        if (YSPLIT) lr += ld;
+                        for (int j = 0; j < RPG; ++j)
+                            if (j < rows) update_row(j);
                     }
                 }
+            };
+            switch (ld) {
+                case 2048: run_chunks(WuPitch<2048>()); break;
+                case 3072: run_chunks(WuPitch<3072>()); break;
+                case 4096: run_chunks(WuPitch<4096>()); break;
+                case 8192: run_chunks(WuPitch<8192>()); break;
+                default: run_chunks(WuPitch<0>()); break;
             }
             if (!ok) break;
             tc_fence_before();
