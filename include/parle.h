@@ -54,7 +54,9 @@ extern "C" {
 
 #define PARLE_GEMM_FP32 0   /* fp32 operands, fp32 FMA accumulation */
 #define PARLE_GEMM_BF16 1   /* bf16 operands on the tcgen05 tensor cores, fp32 accumulation;
-                               needs batch % 8 == 0 and every d_l % 8 == 0 except the last */
+                               needs batch % 8 == 0 and every d_l % 8 == 0 except the last.
+                               Weights are rounded to bf16 to nearest with ties away from zero,
+                               activations and their gradients to nearest with ties to even */
 
 #define PARLE_MAX_LAYERS 16
 #define PARLE_MAX_REPLICAS 64
@@ -190,13 +192,13 @@ int parle_set_fused_update(parle_ctx *ctx, int on);
 int parle_set_paired_z_update(parle_ctx *ctx, int on);
 
 /* bf16 path with the fused update, whole rounds only (parle_round, parle_round_host).  on (the default): between the
- * first and the last inner step of a round the y^a of the weights is not kept as fp32 words but as the bf16 operand copy
- * the GEMMs read (the rounded upper halves) plus a plane of the lower halves in the workspace -- together the same 32
- * bits, moved as 2 + 2 bytes with no separate operand copy to write (12 / 20 instead of 14 / 22 bytes per weight and
- * step).  The last step of the round stores the fp32 y^a again, so y is current when the call returns.  One detail: an
- * fp32 value whose lower half is exactly 0x8000 under an odd upper half is stored one fp32 ulp higher (that makes the
- * rounding direction of the bf16 copy recoverable from the lower half alone); this touches 2^-17 of the elements.
- * Biases are not affected.  off: y^a is read and written as fp32 at every step.  ESTATE inside a round. */
+ * first and the last inner step of a round the y^a of the weights is not kept as fp32 words but as two 16-bit planes:
+ * the upper and the lower half of (fp32 word + 0x8000).  The upper half is the bf16 operand copy the GEMMs read (y
+ * rounded to nearest, ties away from zero -- the rounding every weight copy of this library uses), the lower half lives
+ * in the workspace; ((upper << 16) | lower) - 0x8000 is the fp32 word again, exactly.  So y moves as 2 + 2 bytes with no
+ * separate operand copy to write (12 / 20 instead of 14 / 22 bytes per weight and step), and every result is bit for bit
+ * what the fp32 form gives.  The last step of the round stores the fp32 y^a again, so y is current when the call
+ * returns.  Biases are not affected.  off: y^a is read and written as fp32 at every step.  ESTATE inside a round. */
 int parle_set_split_y(parle_ctx *ctx, int on);
 
 /* fp32 configurations only: where the forward / backward products run (Section 1.1 / 2.1, the minibatch

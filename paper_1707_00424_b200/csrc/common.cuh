@@ -30,6 +30,14 @@ __device__ __forceinline__ void split_tf32(float v, float &hi, float &lo) {
     lo = round_tf32(v - hi);
 }
 
+// bf16 operand copy of a weight: the upper half of the fp32 word after adding 0x8000, i.e. rounded to nearest with
+// ties away from zero.  Written this way (rather than ties-to-even) because the same addition splits the word into
+// two 16-bit halves from which it can be put together again exactly: word = ((upper << 16) | lower) - 0x8000.
+__device__ __forceinline__ uint32_t bf16_split_word(float v) { return __float_as_uint(v) + 0x8000u; }
+__device__ __forceinline__ __nv_bfloat16 bf16_weight(float v) {
+    return __ushort_as_bfloat16((unsigned short)(bf16_split_word(v) >> 16));
+}
+
 struct LayerPlan {
     int d_in, d_out;
     size_t w_off, b_off;          // element offsets inside one replica's vector

@@ -448,9 +448,9 @@ blocked_bf16_kernel(const BlockedPlan bp, const float *__restrict__ src, long lo
         const int row = rb * 128 + r;
         if (row < bp.d_out[l] && col < bp.d_in[l]) {          // d_in % 8 == 0: the 4 columns are all inside
             const float4 v = *reinterpret_cast<const float4 *>(W + (long long)row * bp.d_in[l] + col);
-            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-            uint2 pk;
-            pk.x = *reinterpret_cast<uint32_t *>(&lo); pk.y = *reinterpret_cast<uint32_t *>(&hi);
+            uint2 pk;                                         // weights: nearest, ties away from zero (bf16_weight)
+            pk.x = (bf16_split_word(v.x) >> 16) | (bf16_split_word(v.y) & 0xFFFF0000u);
+            pk.y = (bf16_split_word(v.z) >> 16) | (bf16_split_word(v.w) & 0xFFFF0000u);
             *reinterpret_cast<uint2 *>(out + r * 64 + c4) = pk;
         }
     }

@@ -42,12 +42,11 @@
 // step of a round with an even number of steps).  Same recurrence, different fp32 rounding of z (1e-7 relative).
 //
 // y in two 16-bit planes (YSPLIT).  Inside a whole round nobody but this kernel reads the fp32 y of the weights, and the
-// kernel writes bf16(y) for the GEMMs anyway.  So y is kept as that bf16 copy (the "hi" plane) plus the low 16 bits of
-// its fp32 word (the "lo" plane, workspace): together exactly the fp32 value, read and written as 2 + 2 bytes, and the
-// separate 2-byte operand copy comes for free: 12 / 20 bytes per weight and step instead of 14 / 22.  Decoding:
-// bf16 round-to-nearest-even went up exactly when lo > 0x8000, or lo == 0x8000 with an odd upper half; in that last
-// (tie) case the encoder stores 0x8001, i.e. moves y by one fp32 ulp (2^-17 of the elements), so that "went up" is
-// simply lo > 0x8000.  The last step of a round also writes the fp32 y, so y is current again when the round returns.
+// kernel writes a bf16 copy of y for the GEMMs anyway.  That copy is the upper half of (fp32 word + 0x8000): y rounded to
+// nearest, ties away from zero.  The lower half of the same sum goes to a second plane (workspace), and
+// word = ((upper << 16) | lower) - 0x8000 gives the fp32 y back exactly.  So y is read and written as 2 + 2 bytes and the
+// separate 2-byte operand copy comes for free: 12 / 20 bytes per weight and step instead of 14 / 22.  The last step of a
+// round also writes the fp32 y, so y is current again when the round returns.
 // All waits are bounded.
 #pragma once
 
@@ -67,13 +66,17 @@ struct WuShape {
     static constexpr int GROUPS = G, CHUNK_ROWS = CR, RPG = CR / G;
     static constexpr int CHUNKS = UM_BN / CR;
     static constexpr int ARRAY_BYTES = CR * UM_BM * 4;          // one fp32 box of x, y, z (or the momentum v)
-    static constexpr int STATE_BYTES = NA * ARRAY_BYTES;        // x | y | z [| v]
-    static constexpr int STAGES = WU_STATE_RING_BYTES / STATE_BYTES;
+    static constexpr int MAX_ARRAYS = NA;                       // x | y | z [| v]
+    // A stage holds only the arrays its kind of step loads (x alone on the first step of a round, no z on the steps
+    // that leave z untouched), so those steps get more, smaller stages out of the same ring: the bytes in flight per
+    // SM stay the same, which is what keeps a step with few bytes per weight from becoming latency-bound.
+    __host__ __device__ static constexpr int stages(int arrays) { return WU_STATE_RING_BYTES / (arrays * ARRAY_BYTES); }
+    static constexpr int MAX_STAGES = stages(1);
     static constexpr int THREADS = 96 + 128 * G;
-    static constexpr size_t SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)STAGES * STATE_BYTES +
+    static constexpr size_t SMEM_BYTES = (size_t)WU_OP_STAGES * UM_STAGE_BYTES + (size_t)WU_STATE_RING_BYTES +
                                          1024 /*alignment slack*/ + WU_CTL_BYTES;
     static_assert(RPG == 4 || RPG == 8 || RPG == 16, "rows per thread must match a tcgen05.ld shape");
-    static_assert(STAGES >= 2 && 8 * (2 * WU_OP_STAGES + 4 + 2 * STAGES + 2 * WU_TILE_SLOTS) + 8 + 4 * WU_TILE_SLOTS <= WU_CTL_BYTES,
+    static_assert(stages(NA) >= 2 && 8 * (2 * WU_OP_STAGES + 4 + 2 * MAX_STAGES + 2 * WU_TILE_SLOTS) + 8 + 4 * WU_TILE_SLOTS <= WU_CTL_BYTES,
                   "stage count");
 };
 using WuDefault = WuShape<4, 32>;
@@ -136,14 +139,18 @@ template <bool FIRST, class SH, bool MOM = false, int ZMODE = WU_Z_SINGLE, bool 
 __global__ void __launch_bounds__(SH::THREADS, 1)
 umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_constant__ WgradUpdateParams p) {
     constexpr int WU_GROUPS = SH::GROUPS, WU_CHUNKS = SH::CHUNKS, WU_ARRAY_BYTES = SH::ARRAY_BYTES;
-    constexpr int WU_STATE_BYTES = SH::STATE_BYTES, WU_STATE_STAGES = SH::STAGES, RPG = SH::RPG;
+    constexpr bool LOADS_Z = !FIRST && ZMODE != WU_Z_SKIP;
+    constexpr int WU_ARRAYS = FIRST ? 1 : 2 + (LOADS_Z ? 1 : 0) + (MOM ? 1 : 0);           // arrays a stage of this step holds
+    constexpr int WU_Z_SLOT = 2, WU_V_SLOT = LOADS_Z ? 3 : 2;                               // x = 0, y = 1
+    constexpr int WU_STATE_BYTES = WU_ARRAYS * WU_ARRAY_BYTES, WU_STATE_STAGES = SH::stages(WU_ARRAYS), RPG = SH::RPG;
+    static_assert(WU_ARRAYS <= SH::MAX_ARRAYS, "stage layout");
     constexpr int WU_CHUNK_ROWS = SH::CHUNK_ROWS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t op_base = (raw + 1023u) & ~1023u;
     const uint32_t st_base = op_base + WU_OP_STAGES * UM_STAGE_BYTES;
     uint8_t *st_ptr = smem_raw + (st_base - raw);
-    uint8_t *ctl = st_ptr + (size_t)WU_STATE_STAGES * WU_STATE_BYTES;
+    uint8_t *ctl = st_ptr + (size_t)WU_STATE_RING_BYTES;
     // barriers: op_full[2], op_empty[2], tfull[2], tempty[2], st_full[S], st_empty[S], tile_full[T], tile_empty[T]
     uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);
     constexpr int NBARS = 2 * WU_OP_STAGES + 4 + 2 * WU_STATE_STAGES + 2 * WU_TILE_SLOTS;
@@ -274,8 +281,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     if (!mbar_wait(bar_sempty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t dst = st_base + stage * WU_STATE_BYTES;
                     const uint32_t fb = bar_sfull + 8 * stage;
-                    constexpr bool LOAD_Z = !FIRST && ZMODE != WU_Z_SKIP;
-                    mbar_expect_tx(fb, FIRST ? WU_ARRAY_BYTES : WU_STATE_BYTES - (LOAD_Z ? 0 : WU_ARRAY_BYTES));   // STATE_BYTES counts v when MOM
+                    mbar_expect_tx(fb, WU_STATE_BYTES);
                     tma_load_3d(dst, &maps.x[l], fb, m0, nb, g);
                     if (!FIRST) {
                         if (YSPLIT) {
@@ -287,8 +293,8 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                         } else {
                             tma_load_3d(dst + WU_ARRAY_BYTES, &maps.y[l], fb, m0, nb, g);
                         }
-                        if (LOAD_Z) tma_load_3d(dst + 2 * WU_ARRAY_BYTES, &maps.z[l], fb, m0, nb, g);
-                        if (MOM) tma_load_3d(dst + 3 * WU_ARRAY_BYTES, &maps.v[l], fb, m0, nb, g);
+                        if (LOADS_Z) tma_load_3d(dst + WU_Z_SLOT * WU_ARRAY_BYTES, &maps.z[l], fb, m0, nb, g);
+                        if (MOM) tma_load_3d(dst + WU_V_SLOT * WU_ARRAY_BYTES, &maps.v[l], fb, m0, nb, g);
                     }
                     if (++stage == WU_STATE_STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -341,8 +347,9 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
             // The rows a thread owns inside a chunk are `ld` elements apart.  For the usual widths the pitch is a
             // compile-time constant, so every row's address is the chunk pointer plus an immediate offset and the
             // loop below carries no address arithmetic; other widths take the run-time pitch.
-            auto run_chunks = [&](auto ld_tag) {
+            auto run_chunks = [&](auto ld_tag, auto wd_tag) {
                 constexpr int LDC = decltype(ld_tag)::value;
+                constexpr bool HAS_WD = decltype(wd_tag)::value != 0;        // without weight decay its term is not computed at all
                 const long long ldv = LDC > 0 ? (long long)LDC : (long long)ld;
 #pragma unroll 1
                 for (int c = 0; c < WU_CHUNKS; ++c, yp += chunk_step, zp += chunk_step, sp += WU_CHUNK_ROWS * 64) {
@@ -365,12 +372,12 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                                 const int rr = grp * RPG + j;
                                 const uint32_t hi = sy[(col >> 6) * (WU_CHUNK_ROWS * 64) + rr * 64 + (col & 63)];
                                 const uint32_t lo = sy[WU_CHUNK_ROWS * 128 + rr * UM_BM + col];
-                                yv[j] = __uint_as_float(((hi - (lo > 0x8000u ? 1u : 0u)) << 16) | lo);
+                                yv[j] = __uint_as_float(((hi << 16) | lo) - 0x8000u);
                             } else {
                                 yv[j] = sx[WU_ARRAY_BYTES / 4 + j * UM_BM];
                             }
-                            if (USE_Z) zv[j] = sx[2 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
-                            if (MOM) vv[j] = sx[3 * (WU_ARRAY_BYTES / 4) + j * UM_BM];
+                            if (USE_Z) zv[j] = sx[WU_Z_SLOT * (WU_ARRAY_BYTES / 4) + j * UM_BM];
+                            if (MOM) vv[j] = sx[WU_V_SLOT * (WU_ARRAY_BYTES / 4) + j * UM_BM];
                         }
                     }
                     uint32_t r[RPG];
@@ -385,20 +392,18 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     auto update_row = [&](int j) {
                         const long long o = (long long)j * ldv;
                         const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : (USE_Z ? zv[j] : 0.f);
-                        float d = fmaf(p.inv_gamma, yo - xv[j], fmaf(p.wd, yo, __uint_as_float(r[j])));
+                        float d = fmaf(p.inv_gamma, yo - xv[j], HAS_WD ? fmaf(p.wd, yo, __uint_as_float(r[j])) : __uint_as_float(r[j]));
                         if (MOM) {
                             const float vn = FIRST ? d : fmaf(p.mu, vv[j], d);      // v = 0 before the first step of a round
                             vp[o] = vn;
                             d = fmaf(p.mu, vn, d);
                         }
                         const float yn = fmaf(neg_eta_p, d, yo);
-                        chk = fmaf(yn, 0.f, chk);
+                        if (USE_Z) chk = fmaf(yn, 0.f, chk);     // steps that skip z skip the check: the next step sees the same y
                         if (YSPLIT) {
-                            const uint32_t u = __float_as_uint(yn);
-                            uint32_t lo = u & 0xFFFFu;
-                            if (lo == 0x8000u && ((u >> 16) & 1u)) lo = 0x8001u;     // tie that rounds up: see the head of this file
-                            lp[o] = (uint16_t)lo;
-                            if (YWRITE) yp[o] = __uint_as_float((u & 0xFFFF0000u) | lo);
+                            const uint32_t w = bf16_split_word(yn);
+                            lp[o] = (uint16_t)w;                 // lower half; the upper half is the operand copy below
+                            if (YWRITE) yp[o] = yn;
                         } else {
                             yp[o] = yn;
                         }
@@ -407,7 +412,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                                                                                : fmaf(p.alpha, zo, one_m_alpha * yn);
                             zp[o] = zn;
                         }
-                        sp[j * 64] = __float2bfloat16_rn(yn);
+                        sp[j * 64] = bf16_weight(yn);
                     };
                     if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
@@ -419,12 +424,16 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     }
                 }
             };
-            switch (ld) {
-                case 2048: run_chunks(WuPitch<2048>()); break;
-                case 3072: run_chunks(WuPitch<3072>()); break;
-                case 4096: run_chunks(WuPitch<4096>()); break;
-                case 8192: run_chunks(WuPitch<8192>()); break;
-                default: run_chunks(WuPitch<0>()); break;
+            if (MOM || p.wd != 0.f) {
+                run_chunks(WuPitch<0>(), WuPitch<1>());
+            } else {
+                switch (ld) {
+                    case 2048: run_chunks(WuPitch<2048>(), WuPitch<0>()); break;
+                    case 3072: run_chunks(WuPitch<3072>(), WuPitch<0>()); break;
+                    case 4096: run_chunks(WuPitch<4096>(), WuPitch<0>()); break;
+                    case 8192: run_chunks(WuPitch<8192>(), WuPitch<0>()); break;
+                    default: run_chunks(WuPitch<0>(), WuPitch<0>()); break;
+                }
             }
             if (!ok) break;
             tc_fence_before();

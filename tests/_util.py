@@ -48,3 +48,12 @@ def padding_mask(model):
 def rel_l2(got, want):
     got = np.asarray(got, np.float64); want = np.asarray(want, np.float64)
     return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def bf16_weight(a):
+    """The library's bf16 copy of a weight, as fp64: the fp32 value rounded to the nearest bf16 with ties away from
+    zero (upper half of the fp32 word + 0x8000).  Activations use ties-to-even (the oracle's round_to_bf16); the two
+    differ on exact ties only."""
+    u = np.asarray(a, np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x8000) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(a))

@@ -3,8 +3,8 @@ recurrences (Eq. parle_y, parle_z): they must be identities, not approximations.
 
 1. z is touched every other inner step: z_{k+2} = alpha^2 z_k + (1 - alpha)(alpha y_{k+1} + y_{k+2}), with the
    schedule first step / (skip, two-step) pairs / one closing one-step update when L is even.
-2. y is held as two 16-bit planes: bf16(y) rounded to nearest even + the lower half of the fp32 word, the one
-   ambiguous tie stored one ulp higher."""
+2. y is held as two 16-bit planes, the halves of (fp32 word + 0x8000): the upper one is y rounded to bf16 (nearest,
+   ties away from zero), and ((upper << 16) | lower) - 0x8000 is the word again."""
 import numpy as np
 import pytest
 import torch
@@ -47,19 +47,15 @@ def test_paired_z_schedule_reproduces_the_step_by_step_z(L):
 
 
 def encode_planes(y):
-    u = y.view(np.uint32)
-    lo = (u & 0xFFFF).astype(np.uint32)
-    upper = u >> 16
-    hi = torch.from_numpy(y.copy()).to(torch.bfloat16).view(torch.int16).numpy().astype(np.uint32) & 0xFFFF   # RNE
-    lo = np.where((lo == 0x8000) & (upper & 1 == 1), 0x8001, lo)
-    return hi, lo
+    w = (y.view(np.uint32).astype(np.uint64) + 0x8000) & 0xFFFFFFFF
+    return (w >> 16).astype(np.uint32), (w & 0xFFFF).astype(np.uint32)
 
 
 def decode_planes(hi, lo):
-    return (((hi - (lo > 0x8000)) << 16) | lo).astype(np.uint32).view(np.float32)
+    return ((((hi.astype(np.uint64) << 16) | lo) - 0x8000) & 0xFFFFFFFF).astype(np.uint32).view(np.float32)
 
 
-def test_two_plane_y_round_trips_exactly_except_the_documented_tie():
+def test_two_plane_y_round_trips_exactly_and_its_upper_plane_is_the_nearest_bf16():
     rng = np.random.default_rng(7)
     y = rng.standard_normal(1 << 20).astype(np.float32) * np.float32(0.05)
     bits = y.view(np.uint32).copy()
@@ -68,10 +64,17 @@ def test_two_plane_y_round_trips_exactly_except_the_documented_tie():
     bits[8192:8200] = [0, 0x80000000, 0x00008000, 0x00018000, 0x3F7FFFFF, 0xBF7F8000, 0x00000001, 0x7F000000]
     y = bits.view(np.float32)
     hi, lo = encode_planes(y)
-    back = decode_planes(hi, lo)
-    tie_up = ((bits & 0xFFFF) == 0x8000) & ((bits >> 16) & 1 == 1)
-    assert tie_up.sum() > 1000
-    assert np.array_equal(back[~tie_up].view(np.uint32), bits[~tie_up])
-    assert np.array_equal(back[tie_up].view(np.uint32), bits[tie_up] + 1)       # one fp32 ulp up, same bf16 operand
-    again_hi, again_lo = encode_planes(back)
-    assert np.array_equal(again_hi, hi) and np.array_equal(again_lo, lo)
+    assert np.array_equal(decode_planes(hi, lo).view(np.uint32), bits)           # exact, ties included
+    # the upper plane against the definition of rounding to the nearest bf16, worked out in fp64:
+    # the two neighbours are the truncated word and the next one up in magnitude; ties go to the larger magnitude
+    down = (bits & 0xFFFF0000).view(np.float32).astype(np.float64)
+    up = ((bits & 0xFFFF0000) + 0x10000).astype(np.uint32).view(np.float32).astype(np.float64)
+    v = y.astype(np.float64)
+    want = np.where(np.abs(v - down) < np.abs(up - v), down, up)
+    got = (hi << 16).astype(np.uint32).view(np.float32).astype(np.float64)
+    assert np.array_equal(got, want)
+    # it differs from torch's ties-to-even conversion on ties under an even upper half only
+    rne = torch.from_numpy(y.copy()).to(torch.bfloat16).view(torch.int16).numpy().astype(np.uint32) & 0xFFFF
+    differ = rne != hi
+    tie_even = ((bits & 0xFFFF) == 0x8000) & ((bits >> 16) & 1 == 0)
+    assert np.array_equal(differ, tie_even) and differ.sum() > 1000
