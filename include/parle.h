@@ -224,6 +224,12 @@ int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
  * (none: the k order is the same). */
 int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
 
+/* bf16 path: forward and data-gradient products of the hidden layers (Section 1.1 / 2.1) whose weight matrix has at
+ * least 256 output rows run on pairs of SMs (one two-CTA tensor-core instruction per 256 x batch-tile block, the two CTAs
+ * sharing the activation tile).  on (the default) / off: the one-SM kernel for every product.  Same products, same
+ * reduction order.  EUNSUPPORTED on an fp32 context. */
+int parle_set_pair_gemm(parle_ctx *ctx, int on);
+
 /* Nesterov momentum on the y^a and x^a steps (Remark in Section 3.1; none on xbar).  The paper does not
  * print the form; the one taken is that of SGD with Nesterov momentum: for a step with direction d and
  * step size s,  v <- mu v + d,  p <- p - s (d + mu v), with

@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
         "parle_fp32_tensor_cores_active": (ci, [vp]),
         "parle_set_weight_decay": (ci, [vp, cd]),
         "parle_set_wide_tile_threshold": (ci, [vp, ci]),
+        "parle_set_pair_gemm": (ci, [vp, ci]),
         "parle_bind_momentum": (ci, [vp, vp, vp]),
         "parle_set_momentum": (ci, [vp, cd]),
         "parle_scoping": (ci, [cd, cd, C.c_longlong, C.c_longlong, cd, cd, C.POINTER(cd), C.POINTER(cd)]),
@@ -260,6 +261,10 @@ class Parle:
 
     def set_wide_tile_threshold(self, tiles_per_sm: int):
         self._check(self._L.parle_set_wide_tile_threshold(self._h, tiles_per_sm), "parle_set_wide_tile_threshold")
+
+    def set_pair_gemm(self, on: bool):
+        """bf16 path: hidden-layer forward / data-gradient products on pairs of SMs (default on)."""
+        self._check(self._L.parle_set_pair_gemm(self._h, 1 if on else 0), "parle_set_pair_gemm")
 
     def set_weight_decay(self, lam: float):
         self._check(self._L.parle_set_weight_decay(self._h, lam), "parle_set_weight_decay")

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libparle.so")
 SOURCES = ["parle_api.cu", "static_loss.cu"]
-HEADERS = ["common.cuh", "mlp_simt.cuh", "umma_gemm.cuh", "umma_wgrad_update.cuh", "umma_tf32x3.cuh", "update_kernels.cuh"]
+HEADERS = ["common.cuh", "mlp_simt.cuh", "umma_gemm.cuh", "umma_pair_gemm.cuh", "umma_wgrad_update.cuh", "umma_tf32x3.cuh", "update_kernels.cuh"]
 
 
 def _nvcc() -> str:

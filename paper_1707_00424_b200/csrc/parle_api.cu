@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "mlp_simt.cuh"
 #include "umma_gemm.cuh"
+#include "umma_pair_gemm.cuh"
 #include "umma_wgrad_update.cuh"
 #include "umma_tf32x3.cuh"
 #include "update_kernels.cuh"
@@ -63,6 +64,7 @@ struct RoundKey {
     const void *inputs, *labels, *loss;
     float scal[7];                   // 1/gamma, 1/rho, alpha, eta, eta', weight decay, momentum
     int fused, wide_thr, shadow_is_x, fresh;   // L == 0: a single inner step (fresh = first of its round)
+    int pair_gemm;
     int paired_z, z_mode;            // whole rounds: Eq. (parle_z) in pairs or not; single steps: how this step treats z
     int split_y, y_step;             // whole rounds: y in two 16-bit planes or not; single steps: bit 0 = in that mode, bit 1 = stores fp32 y
     const void *ptrs[9];             // x, y, z, grad, xbar, workspace, vy, vx, stream
@@ -106,6 +108,9 @@ struct parle_ctx {
     CUtensorMap tm_fwd_a[PARLE_MAX_LAYERS], tm_fwd_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_dg_a[PARLE_MAX_LAYERS], tm_dg_b[PARLE_MAX_LAYERS];
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
+    // forward / data-gradient products on pairs of SMs: the activation operand in boxes of half a batch tile
+    CUtensorMap tm_pf_x[PARLE_MAX_LAYERS], tm_pd_x[PARLE_MAX_LAYERS];
+    bool pair_gemm;                  // use the pair kernel where the shapes allow (parle_set_pair_gemm)
     // fp32 configurations on the tensor cores (three tf32 products per GEMM)
     int t3_mode;                     // 0 = never, 1 = when the layers are wide enough to fill 128-row tiles, 2 = whenever possible
     bool t3_shapes_ok;               // widths and batch are multiples of 4 (16-byte rows for TMA)
@@ -412,6 +417,44 @@ inline bool use_t3(const parle_ctx *c) {
     return true;
 }
 
+// Batch tile of the pair kernel: 128 rows, or 256 when the batch has more than 128.
+inline int pair_batch_tile(const parle_ctx *c) { return c->batch > 128 ? 256 : 128; }
+// The pair kernel takes a product when its weight operand has at least one full pair tile of output features.
+inline bool use_pair_gemm(const parle_ctx *c, int features) { return c->pair_gemm && features >= 2 * UP_BM; }
+
+template <int EPI, int BNB>
+int launch_pair_bn(parle_ctx *c, int cls, const CUtensorMap &w, const CUtensorMap &x, UmmaPairParams p) {
+    p.groups = c->n;
+    p.tiles_f = (p.F + 2 * UP_BM - 1) / (2 * UP_BM);
+    p.tiles_b = (p.Bt + BNB - 1) / BNB;
+    p.status = c->status_dev;
+    const int tiles = p.groups * p.tiles_f * p.tiles_b, pairs = c->sm_count / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (tiles < pairs ? tiles : pairs));
+    cfg.blockDim = dim3(UP_THREADS);
+    cfg.dynamicSmemBytes = UpShape<BNB>::SMEM_BYTES;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    prof_begin(c, cls);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, umma_pair_gemm_kernel<EPI, BNB>, w, x, p);
+    if (e != cudaSuccess) { prof_end(c); return cuda_fail(c, e); }
+    PARLE_LAUNCHED(c);
+    return PARLE_OK;
+}
+template <int EPI>
+int launch_pair(parle_ctx *c, int cls, const CUtensorMap &w, const CUtensorMap &x, const UmmaPairParams &p) {
+    return pair_batch_tile(c) == 256 ? launch_pair_bn<EPI, 256>(c, cls, w, x, p) : launch_pair_bn<EPI, 128>(c, cls, w, x, p);
+}
+template <int EPI>
+cudaError_t allow_pair_smem() {
+    cudaError_t e = cudaFuncSetAttribute(umma_pair_gemm_kernel<EPI, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpShape<128>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(umma_pair_gemm_kernel<EPI, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpShape<256>::SMEM_BYTES);
+}
+
 int build_tensor_maps(parle_ctx *c) {
     const Workspace &w = c->ws;
     const size_t n = c->n, B = c->batch;
@@ -423,6 +466,8 @@ int build_tensor_maps(parle_ctx *c) {
         const __nv_bfloat16 *W = shadow + c->sh_off[l];
         // forward: A = layer input [B, din], B = W [dout, din], both K-major (K = din)
         PARLE_TRY(encode_bf16_map(c, &c->tm_fwd_a[l], a_in, din, B, n, din, B * din, UM_BK, UM_BM));
+        // the same input as the shared operand of a pair of CTAs: boxes of half a batch tile
+        PARLE_TRY(encode_bf16_map(c, &c->tm_pf_x[l], a_in, din, B, n, din, B * din, UM_BK, pair_batch_tile(c) / 2));
         PARLE_TRY(encode_blocked_map(c, &c->tm_fwd_b[l], W, c->sh_cb[l], c->sh_rb[l], n, c->sh_stride, 128));
         // weight gradient, computed transposed (dW^T = input^T dH): A = input^T [din, B], B = dH^T [dout, B],
         // both K-major (K = batch)
@@ -443,6 +488,8 @@ int build_tensor_maps(parle_ctx *c) {
             PARLE_TRY(encode_bf16_map(c, &c->tm_dg_a[l], ws_ptr<__nv_bfloat16>(c, w.dhb[l]), dout, B, n,
                                       w.dh_ld[l], B * (size_t)w.dh_ld[l], UM_BK, UM_BM));
             PARLE_TRY(encode_blocked_map(c, &c->tm_dg_b[l], W, c->sh_cb[l], c->sh_rb[l], n, c->sh_stride, 64));
+            PARLE_TRY(encode_bf16_map(c, &c->tm_pd_x[l], ws_ptr<__nv_bfloat16>(c, w.dhb[l]), dout, B, n,
+                                      w.dh_ld[l], B * (size_t)w.dh_ld[l], UM_BK, pair_batch_tile(c) / 2));
         }
     }
     return PARLE_OK;
@@ -743,7 +790,14 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
         UmmaParams p = {};
         p.M = B; p.N = dout; p.K = din;
         p.bias = params + c->layers[l].b_off; p.bias_gs = S;
-        if (l + 1 < nl) {
+        if (l + 1 < nl && use_pair_gemm(c, dout)) {
+            UmmaPairParams q = {};                              // H_l^T = W_l H_{l-1}^T on pairs of SMs
+            q.F = dout; q.Bt = B; q.K = din;
+            q.bias = p.bias; q.bias_gs = S;
+            q.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); q.out_gs = (long long)B * dout; q.out_ld = dout;
+            q.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); q.outT_gs = (long long)B * dout; q.outT_ld = B;
+            PARLE_TRY((launch_pair<UPE_FWD_HIDDEN>(c, KC_FWD_GEMM, c->tm_fwd_b[l], c->tm_pf_x[l], q)));
+        } else if (l + 1 < nl) {
             p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
             p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
             PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
@@ -767,6 +821,14 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     }
     auto dgrad = [&](int l) -> int {                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
         const int din = c->dims[l], dout = c->dims[l + 1];
+        if (use_pair_gemm(c, din)) {
+            UmmaPairParams q = {};                              // dH_{l-1}^T = W_l^T dH_l^T on pairs of SMs
+            q.F = din; q.Bt = B; q.K = dout;
+            q.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); q.out_gs = (long long)B * w.dh_ld[l - 1]; q.out_ld = w.dh_ld[l - 1];
+            q.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); q.outT_gs = (long long)B * din; q.outT_ld = B;
+            q.maskT = ws_ptr<__nv_bfloat16>(c, w.hbT[l - 1]); q.maskT_gs = (long long)B * din; q.maskT_ld = B;
+            return launch_pair<UPE_DGRAD>(c, KC_DGRAD_GEMM, c->tm_dg_b[l], c->tm_pd_x[l], q);
+        }
         UmmaParams d = {};
         d.M = B; d.N = din; d.K = dout;
         d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
@@ -949,6 +1011,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
     c->paired_z = true;
     c->split_y = true;
     c->wide_tiles_per_sm = 4;
+    c->pair_gemm = true;
     c->last_ksplit = 1;
     if (c->fused_update) {
         // the last forward layer often has one tile per replica: when its tiles would leave most SMs idle, its k-blocks are
@@ -1035,6 +1098,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
 #undef PARLE_WU_SMEM
         c->mom_maps = false;
         PARLE_CUDA(c, (allow_big_smem<UEPI_DGRAD, UB_BLOCKED_MN>()));
+        PARLE_CUDA(c, allow_pair_smem<UPE_FWD_HIDDEN>());
+        PARLE_CUDA(c, allow_pair_smem<UPE_DGRAD>());
         PARLE_TRY(build_tensor_maps(c));
         // rows / columns of the blocked weight copy beyond the matrices are never written: they must read as zero
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.shadow), 0, (size_t)c->n * c->sh_stride * 2, c->stream));
@@ -1159,6 +1224,7 @@ static RoundKey make_round_key(const parle_ctx *c, int L, const void *in, const 
     const float sc[7] = {c->inv_gamma, c->inv_rho, c->alpha, c->eta, c->eta_prime, c->weight_decay, c->momentum};
     memcpy(k.scal, sc, sizeof(sc));
     k.fused = c->fused_update; k.wide_thr = c->wide_tiles_per_sm; k.shadow_is_x = c->shadow_is_x; k.fresh = c->fresh;
+    k.pair_gemm = c->pair_gemm;
     k.paired_z = c->paired_z; k.z_mode = c->z_mode;
     k.split_y = c->split_y; k.y_step = (c->y_split_step ? 1 : 0) | (c->y_write_step ? 2 : 0);
     const void *pt[9] = {c->buf.x, c->buf.y, c->buf.z, c->buf.grad, c->buf.xbar, c->buf.workspace, c->vy, c->vx, c->stream};
@@ -1392,6 +1458,13 @@ int parle_fp32_tensor_cores_active(const parle_ctx *c) { return c ? (use_t3(c) ?
 int parle_set_wide_tile_threshold(parle_ctx *c, int tiles_per_sm) {
     if (!c || tiles_per_sm < 0) return PARLE_EINVAL;
     c->wide_tiles_per_sm = tiles_per_sm;
+    return PARLE_OK;
+}
+
+int parle_set_pair_gemm(parle_ctx *c, int on) {
+    if (!c) return PARLE_EINVAL;
+    if (c->gemm_dtype != PARLE_GEMM_BF16) return PARLE_EUNSUPPORTED;
+    c->pair_gemm = on != 0;
     return PARLE_OK;
 }
 
