@@ -226,9 +226,14 @@ int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
 
 /* bf16 path: forward and data-gradient products of the hidden layers (Section 1.1 / 2.1) whose weight matrix has at
  * least 256 output rows run on pairs of SMs (one two-CTA tensor-core instruction per 256 x batch-tile block, the two CTAs
- * sharing the activation tile).  on (the default) / off: the one-SM kernel for every product.  Same products, same
- * reduction order.  EUNSUPPORTED on an fp32 context. */
-int parle_set_pair_gemm(parle_ctx *ctx, int on);
+ * sharing the activation tile).  Consecutive such layers can go into ONE launch, whose tiles wait, per replica, for the
+ * layer before them (progress counters in the workspace; the weights of a tile are fetched while it waits).  mode 3:
+ * always chained; 2 (the default): chained where a layer gives a pair of SMs at most two tiles (the case in which a
+ * launch per layer leaves its start-up and epilogue exposed); 1: one launch per layer; 0: the one-SM kernel for every
+ * product.  Same products, same reduction order: the
+ * results do not depend on the mode.  EINVAL for another mode, EUNSUPPORTED on an fp32 context.  A chained launch whose
+ * wait ran out (PARLE_FLAG_WAIT_LIMIT) may leave its counters non-zero: bind again before the next step. */
+int parle_set_pair_gemm(parle_ctx *ctx, int mode);
 
 /* Nesterov momentum on the y^a and x^a steps (Remark in Section 3.1; none on xbar).  The paper does not
  * print the form; the one taken is that of SGD with Nesterov momentum: for a step with direction d and

@@ -262,9 +262,10 @@ class Parle:
     def set_wide_tile_threshold(self, tiles_per_sm: int):
         self._check(self._L.parle_set_wide_tile_threshold(self._h, tiles_per_sm), "parle_set_wide_tile_threshold")
 
-    def set_pair_gemm(self, on: bool):
-        """bf16 path: hidden-layer forward / data-gradient products on pairs of SMs (default on)."""
-        self._check(self._L.parle_set_pair_gemm(self._h, 1 if on else 0), "parle_set_pair_gemm")
+    def set_pair_gemm(self, mode: int):
+        """bf16 path: hidden-layer forward / data-gradient products on pairs of SMs: 0 never, 1 one launch per layer,
+        2 (default) consecutive layers chained in one launch where that pays, 3 always chained."""
+        self._check(self._L.parle_set_pair_gemm(self._h, int(mode)), "parle_set_pair_gemm")
 
     def set_weight_decay(self, lam: float):
         self._check(self._L.parle_set_weight_decay(self._h, lam), "parle_set_weight_decay")

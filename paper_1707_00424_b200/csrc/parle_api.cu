@@ -51,6 +51,7 @@ struct Workspace {
     size_t dhs[PARLE_MAX_LAYERS][2], dhT[PARLE_MAX_LAYERS][2];   // their gradients [n, B, ld_l] (ld_l = d_{l+1} rounded up to 4) and transposed [n, d_{l+1}, B]
     size_t ylo;                        // bf16 mode: low 16 bits of the fp32 words of y, [n, stride] uint16 (whole rounds keep y as bf16 copy + this)
     size_t sched;                      // bf16 mode: two ints, the tile counters of the fused weight-gradient kernel (zero between launches)
+    size_t pair_sync;                  // bf16 mode: per-(link, replica) progress counters of the chained pair kernel (zero between launches)
     size_t stage_in[2], stage_lab[2], stage_loss[2];   // double-buffered staging for the host-buffer entry points
     size_t total;
 };
@@ -110,7 +111,7 @@ struct parle_ctx {
     CUtensorMap tm_wg_a[PARLE_MAX_LAYERS], tm_wg_b[PARLE_MAX_LAYERS];
     // forward / data-gradient products on pairs of SMs: the activation operand in boxes of half a batch tile
     CUtensorMap tm_pf_x[PARLE_MAX_LAYERS], tm_pd_x[PARLE_MAX_LAYERS];
-    bool pair_gemm;                  // use the pair kernel where the shapes allow (parle_set_pair_gemm)
+    int pair_gemm;                   // pair kernel where the shapes allow: 0 = never, 1 = one launch per layer, 2 = chained where it pays, 3 = always chained
     // fp32 configurations on the tensor cores (three tf32 products per GEMM)
     int t3_mode;                     // 0 = never, 1 = when the layers are wide enough to fill 128-row tiles, 2 = whenever possible
     bool t3_shapes_ok;               // widths and batch are multiples of 4 (16-byte rows for TMA)
@@ -215,6 +216,7 @@ void plan_workspace(parle_ctx *c) {
         }
         w.ylo = take(n * c->stride * sizeof(uint16_t));
         w.sched = take(2 * sizeof(int));
+        w.pair_sync = take(UP_SYNC_INTS * sizeof(int));
     }
     w.row_loss = take(n * B * sizeof(float));
     for (int b = 0; b < 2; ++b) {
@@ -420,15 +422,56 @@ inline bool use_t3(const parle_ctx *c) {
 // Batch tile of the pair kernel: 128 rows, or 256 when the batch has more than 128.
 inline int pair_batch_tile(const parle_ctx *c) { return c->batch > 128 ? 256 : 128; }
 // The pair kernel takes a product when its weight operand has at least one full pair tile of output features.
-inline bool use_pair_gemm(const parle_ctx *c, int features) { return c->pair_gemm && features >= 2 * UP_BM; }
+inline bool use_pair_gemm(const parle_ctx *c, int features) { return c->pair_gemm > 0 && features >= 2 * UP_BM; }
+// Chain a product with `features` output rows to its predecessor in one launch?  Mode 3: always.  Mode 2: when the
+// product gives a pair of SMs at most two tiles -- there the start-up and the epilogue of a launch have nothing to
+// hide behind; with many tiles per pair they already overlap with the neighbouring tiles and separate launches do as well.
+inline bool chain_pair_gemm(const parle_ctx *c, int features) {
+    if (c->pair_gemm >= 3) return true;
+    if (c->pair_gemm < 2) return false;
+    const int bt = pair_batch_tile(c);
+    const long long tiles = (long long)c->n * ((features + 2 * UP_BM - 1) / (2 * UP_BM)) * ((c->batch + bt - 1) / bt);
+    return tiles <= 2LL * (c->sm_count / 2);
+}
 
+// One launch of the pair kernel over a chain of products: forward, the hidden layers [first, last] in ascending order
+// (each reads the activations the one before it wrote); backward, the data gradients of layers first, first - 1, ...,
+// last (each reads the gradient the one before it wrote).
 template <int EPI, int BNB>
-int launch_pair_bn(parle_ctx *c, int cls, const CUtensorMap &w, const CUtensorMap &x, UmmaPairParams p) {
-    p.groups = c->n;
-    p.tiles_f = (p.F + 2 * UP_BM - 1) / (2 * UP_BM);
-    p.tiles_b = (p.Bt + BNB - 1) / BNB;
+int launch_pair_bn(parle_ctx *c, int cls, int first, int last) {
+    const Workspace &w = c->ws;
+    const int B = c->batch;
+    const long long S = (long long)c->stride;
+    const float *params = c->fresh ? c->buf.x : c->buf.y;      // fp32 biases come from the master copy
+    UpMaps maps;
+    UmmaPairParams p = {};
+    p.Bt = B; p.groups = c->n; p.tiles_b = (B + BNB - 1) / BNB;
+    int tiles = 0, k = 0;
+    const int step = EPI == UPE_FWD_HIDDEN ? 1 : -1;
+    for (int l = first; l != last + step; l += step, ++k) {
+        const int din = c->dims[l], dout = c->dims[l + 1];
+        UpLink &q = p.link[k];
+        if (EPI == UPE_FWD_HIDDEN) {                            // H_l^T = W_l H_{l-1}^T
+            q.F = dout; q.K = din;
+            q.bias = params + c->layers[l].b_off; q.bias_gs = S;
+            q.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); q.out_gs = (long long)B * dout; q.out_ld = dout;
+            q.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); q.outT_gs = (long long)B * dout; q.outT_ld = B;
+            maps.w[k] = c->tm_fwd_b[l]; maps.x[k] = c->tm_pf_x[l];
+        } else {                                                // dH_{l-1}^T = W_l^T dH_l^T, masked by H_{l-1} > 0
+            q.F = din; q.K = dout;
+            q.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); q.out_gs = (long long)B * w.dh_ld[l - 1]; q.out_ld = w.dh_ld[l - 1];
+            q.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); q.outT_gs = (long long)B * din; q.outT_ld = B;
+            q.maskT = ws_ptr<__nv_bfloat16>(c, w.hbT[l - 1]); q.maskT_gs = (long long)B * din; q.maskT_ld = B;
+            maps.w[k] = c->tm_dg_b[l]; maps.x[k] = c->tm_pd_x[l];
+        }
+        q.tiles_f = (q.F + 2 * UP_BM - 1) / (2 * UP_BM);
+        q.tile_begin = tiles;
+        tiles += c->n * q.tiles_f * p.tiles_b;
+    }
+    p.n_links = k; p.total_tiles = tiles;
+    p.sync = ws_ptr<int>(c, w.pair_sync);
     p.status = c->status_dev;
-    const int tiles = p.groups * p.tiles_f * p.tiles_b, pairs = c->sm_count / 2;
+    const int pairs = c->sm_count / 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (tiles < pairs ? tiles : pairs));
     cfg.blockDim = dim3(UP_THREADS);
@@ -439,14 +482,14 @@ int launch_pair_bn(parle_ctx *c, int cls, const CUtensorMap &w, const CUtensorMa
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     prof_begin(c, cls);
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, umma_pair_gemm_kernel<EPI, BNB>, w, x, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, umma_pair_gemm_kernel<EPI, BNB>, maps, p);
     if (e != cudaSuccess) { prof_end(c); return cuda_fail(c, e); }
     PARLE_LAUNCHED(c);
     return PARLE_OK;
 }
 template <int EPI>
-int launch_pair(parle_ctx *c, int cls, const CUtensorMap &w, const CUtensorMap &x, const UmmaPairParams &p) {
-    return pair_batch_tile(c) == 256 ? launch_pair_bn<EPI, 256>(c, cls, w, x, p) : launch_pair_bn<EPI, 128>(c, cls, w, x, p);
+int launch_pair(parle_ctx *c, int cls, int first, int last) {
+    return pair_batch_tile(c) == 256 ? launch_pair_bn<EPI, 256>(c, cls, first, last) : launch_pair_bn<EPI, 128>(c, cls, first, last);
 }
 template <int EPI>
 cudaError_t allow_pair_smem() {
@@ -787,17 +830,17 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     }
     for (int l = 0; l < nl; ++l) {
         const int din = c->dims[l], dout = c->dims[l + 1];
+        if (l + 1 < nl && use_pair_gemm(c, dout)) {
+            int e = l;                                          // hidden layers l .. e on pairs of SMs, chained in one launch
+            while (e + 2 < nl && use_pair_gemm(c, c->dims[e + 2]) && chain_pair_gemm(c, c->dims[e + 2])) ++e;
+            PARLE_TRY(launch_pair<UPE_FWD_HIDDEN>(c, KC_FWD_GEMM, l, e));
+            l = e;
+            continue;
+        }
         UmmaParams p = {};
         p.M = B; p.N = dout; p.K = din;
         p.bias = params + c->layers[l].b_off; p.bias_gs = S;
-        if (l + 1 < nl && use_pair_gemm(c, dout)) {
-            UmmaPairParams q = {};                              // H_l^T = W_l H_{l-1}^T on pairs of SMs
-            q.F = dout; q.Bt = B; q.K = din;
-            q.bias = p.bias; q.bias_gs = S;
-            q.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); q.out_gs = (long long)B * dout; q.out_ld = dout;
-            q.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); q.outT_gs = (long long)B * dout; q.outT_ld = B;
-            PARLE_TRY((launch_pair<UPE_FWD_HIDDEN>(c, KC_FWD_GEMM, c->tm_fwd_b[l], c->tm_pf_x[l], q)));
-        } else if (l + 1 < nl) {
+        if (l + 1 < nl) {
             p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
             p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
             PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
@@ -821,14 +864,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     }
     auto dgrad = [&](int l) -> int {                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
         const int din = c->dims[l], dout = c->dims[l + 1];
-        if (use_pair_gemm(c, din)) {
-            UmmaPairParams q = {};                              // dH_{l-1}^T = W_l^T dH_l^T on pairs of SMs
-            q.F = din; q.Bt = B; q.K = dout;
-            q.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); q.out_gs = (long long)B * w.dh_ld[l - 1]; q.out_ld = w.dh_ld[l - 1];
-            q.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l - 1]); q.outT_gs = (long long)B * din; q.outT_ld = B;
-            q.maskT = ws_ptr<__nv_bfloat16>(c, w.hbT[l - 1]); q.maskT_gs = (long long)B * din; q.maskT_ld = B;
-            return launch_pair<UPE_DGRAD>(c, KC_DGRAD_GEMM, c->tm_dg_b[l], c->tm_pd_x[l], q);
-        }
+        if (use_pair_gemm(c, din)) return launch_pair<UPE_DGRAD>(c, KC_DGRAD_GEMM, l, l);
         UmmaParams d = {};
         d.M = B; d.N = din; d.K = dout;
         d.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l - 1]); d.out_gs = (long long)B * w.dh_ld[l - 1]; d.out_ld = w.dh_ld[l - 1];
@@ -855,7 +891,16 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     // Fused: the weight gradient never reaches memory.  All data-gradient products go first (they read the bf16
     // weight copies that the fused kernel overwrites); then ONE launch of the fused kernel walks the W tiles of
     // every layer, so the stream of x, y, z through the SMs starts up and drains once per step, not once per layer.
-    for (int l = nl - 1; l > 0; --l) PARLE_TRY(dgrad(l));
+    for (int l = nl - 1; l > 0; --l) {
+        if (use_pair_gemm(c, c->dims[l])) {
+            int e = l;                                          // data gradients of layers l, l - 1, ..., e chained in one launch
+            while (e - 1 > 0 && use_pair_gemm(c, c->dims[e - 1]) && chain_pair_gemm(c, c->dims[e - 1])) --e;
+            PARLE_TRY(launch_pair<UPE_DGRAD>(c, KC_DGRAD_GEMM, l, e));
+            l = e;
+            continue;
+        }
+        PARLE_TRY(dgrad(l));
+    }
     WgradUpdateParams p = {};
     p.K = B; p.groups = n; p.n_layers = nl;
     int tiles = 0;
@@ -1011,7 +1056,7 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
     c->paired_z = true;
     c->split_y = true;
     c->wide_tiles_per_sm = 4;
-    c->pair_gemm = true;
+    c->pair_gemm = 2;
     c->last_ksplit = 1;
     if (c->fused_update) {
         // the last forward layer often has one tile per replica: when its tiles would leave most SMs idle, its k-blocks are
@@ -1105,6 +1150,7 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.shadow), 0, (size_t)c->n * c->sh_stride * 2, c->stream));
         // tile counters of the fused weight-gradient kernel: every launch leaves them at zero again
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.sched), 0, 2 * sizeof(int), c->stream));
+        PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.pair_sync), 0, UP_SYNC_INTS * sizeof(int), c->stream));
     }
     c->t3_ready = false;
     if (c->t3_shapes_ok) {
@@ -1461,10 +1507,10 @@ int parle_set_wide_tile_threshold(parle_ctx *c, int tiles_per_sm) {
     return PARLE_OK;
 }
 
-int parle_set_pair_gemm(parle_ctx *c, int on) {
-    if (!c) return PARLE_EINVAL;
+int parle_set_pair_gemm(parle_ctx *c, int mode) {
+    if (!c || mode < 0 || mode > 3) return PARLE_EINVAL;
     if (c->gemm_dtype != PARLE_GEMM_BF16) return PARLE_EUNSUPPORTED;
-    c->pair_gemm = on != 0;
+    c->pair_gemm = mode;
     return PARLE_OK;
 }
 

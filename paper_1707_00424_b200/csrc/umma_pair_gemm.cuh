@@ -24,6 +24,18 @@
 //   * the epilogue warps of both CTAs arrive on the leader's "accumulator empty" barrier.
 // Tensor memory is allocated and freed by warp 1 of both CTAs (cta_group::2).  Every wait is bounded; the two CTAs
 // meet at a cluster barrier before tensor memory is released.
+//
+// Several layers in one launch.  At batch 128 a layer is one tile per pair, so a launch per layer pays its start-up
+// (barriers, tensor memory, the first weights' latency) and its epilogue with nothing to overlap them with.  A launch
+// therefore takes a chain of products, each reading what the one before it wrote (forward: hidden layers 1, 2, ...;
+// backward: the data gradients from the top down).  The tiles of all links form one list, link by link; a pair
+// walks its share of the list in order.  Only the activation operand of a tile depends on the link before it (all
+// tiles of that link for the same replica), the weights do not: the producer fetches the weights of the first
+// k-blocks, then waits until the replica's counter of the previous link has reached its full count, then fetches the
+// activations.  So the weight stream of the next layer runs under the epilogue of this one.  The counters live in the
+// caller's workspace (an epilogue warp adds 1 per tile after a device-wide fence), are polled with acquire loads and
+// a bounded wait, and are zeroed again by the last CTA to leave.
+
 #pragma once
 
 #include "umma_gemm.cuh"
@@ -34,6 +46,8 @@ constexpr int UP_BM = 128;                                  // output features p
 constexpr int UP_A_BYTES = UP_BM * UM_BK * 2;               // 16 KiB of weights per k-block
 constexpr int UP_RING_BYTES = 192 * 1024;
 constexpr int UP_THREADS = 320;                             // warp 0 producer, 1 MMA, 2..9 epilogue
+constexpr int UP_MAX_LINKS = PARLE_MAX_LAYERS;
+constexpr int UP_SYNC_INTS = UP_MAX_LINKS * PARLE_MAX_REPLICAS + 1;   // per-(link, replica) counters + the exit counter
 
 template <int BNB> struct UpShape {
     static_assert(BNB == 128 || BNB == 256, "batch tile");
@@ -49,15 +63,25 @@ enum UmmaPairEpilogue {
     UPE_DGRAD = 1          // * (H_{l-1}[b, f] > 0)
 };
 
-struct UmmaPairParams {
-    int F, Bt, K;                     // output features (rows of the weight operand), batch rows, reduction length
-    int groups, tiles_f, tiles_b;     // replicas; 256-feature and BNB-row tiles per replica
+// One product of a chain: out^T [F, Bt] = W-operand [F, K] x X [Bt, K]^T.
+struct UpLink {
+    int F, K;                         // output features (rows of the weight operand), reduction length
+    int tiles_f;                      // 256-feature tiles per replica
+    int tile_begin;                   // index of the link's first tile in the launch's list
     const float *bias; long long bias_gs;
     __nv_bfloat16 *out; long long out_gs; int out_ld;          // [Bt, out_ld]
     __nv_bfloat16 *outT; long long outT_gs; int outT_ld;       // [F, outT_ld]
     const __nv_bfloat16 *maskT; long long maskT_gs; int maskT_ld;   // data gradient: H_{l-1}^T [F, maskT_ld]
+};
+struct UmmaPairParams {
+    int Bt, groups, tiles_b;          // batch rows, replicas, BNB-row tiles per replica
+    int n_links, total_tiles;
+    UpLink link[UP_MAX_LINKS];        // link k > 0 reads, as its X operand, the `out` of link k - 1
+    int *sync;                        // sync[k * groups + g]: epilogue warps that have stored their part of a tile of (link k,
+                                      // replica g); sync[UP_MAX_LINKS * PARLE_MAX_REPLICAS]: CTAs that have left.  All zero between launches
     int *status;
 };
+struct UpMaps { CUtensorMap w[UP_MAX_LINKS], x[UP_MAX_LINKS]; };
 
 // ---------------------------------------------------------------- PTX wrappers (pair forms)
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -113,11 +137,29 @@ __host__ __device__ constexpr uint32_t make_pair_idesc(bool a_mn_major, int bn) 
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) |
            ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
+__device__ __forceinline__ int ld_acquire_gpu(const int *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Bounded wait until *counter >= need (another CTA's epilogue warps count up).  Returns false on a time-out or when
+// another role of this CTA gave up.
+__device__ __forceinline__ bool wait_counter(const int *counter, int need, volatile int *abort_flag) {
+    if (ld_acquire_gpu(counter) >= need) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (ld_acquire_gpu(counter) >= need) return true;
+        __nanosleep(64);
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > UM_WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+    }
+}
 
 template <int EPI, int BNB>
 __global__ void __launch_bounds__(UP_THREADS, 1)
-umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                      const UmmaPairParams p) {
+umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant__ UmmaPairParams p) {
     using SH = UpShape<BNB>;
     constexpr int STAGES = SH::STAGES, STAGE_BYTES = SH::STAGE_BYTES;
     constexpr bool A_MN = (EPI == UPE_DGRAD);
@@ -137,8 +179,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                               // 0 = leader of the pair
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int total_tiles = p.groups * p.tiles_f * p.tiles_b;
-    const int num_kb = (p.K + UM_BK - 1) / UM_BK;
+    const int total_tiles = p.total_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -158,8 +199,12 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    auto tile_coords = [&](int t, int &g, int &f0, int &b0) {
-        const int per_g = p.tiles_f * p.tiles_b;
+    // tile t -> link k, replica g, first feature f0 of the pair, first batch row b0
+    auto tile_coords = [&](int t, int &k, int &g, int &f0, int &b0) {
+        k = 0;
+        while (k + 1 < p.n_links && t >= p.link[k + 1].tile_begin) ++k;
+        const int per_g = p.link[k].tiles_f * p.tiles_b;
+        t -= p.link[k].tile_begin;
         g = t / per_g;
         const int r = t - g * per_g;
         b0 = (r % p.tiles_b) * BNB;
@@ -170,26 +215,54 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         // ------------------------------------------------ TMA producer: this CTA's rows of W and its half of the batch tile
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
+            auto load_w = [&](int k, int kb, int st, int fr, int g) {
+                const uint32_t sa = ring + st * STAGE_BYTES;
+                const uint32_t fb = mapa_shared(bar_full + 8 * st, 0);     // both CTAs' copies complete on the leader's barrier
+                if (!A_MN) {
+                    // K-major weights: block (row block fr/128, column block kb) of the blocked copy
+                    tma_pair_load_5d(sa, &maps.w[k], fb, 0, 0, kb, fr / 128, g);
+                } else {
+                    // MN-major weights: k-rows kb*64 .. +63 = half of row block kb/2; features fr .. fr+127 = two column blocks
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tma_pair_load_5d(sa + h * (UP_A_BYTES / 2), &maps.w[k], fb, 0, (kb & 1) * 64, fr / 64 + h, kb >> 1, g);
+                }
+            };
+            auto load_x = [&](int k, int kb, int st, int br, int g) {
+                tma_pair_load_3d(ring + st * STAGE_BYTES + UP_A_BYTES, &maps.x[k], mapa_shared(bar_full + 8 * st, 0), kb * UM_BK, br, g);
+            };
             for (int t = pair; t < total_tiles && ok; t += num_pairs) {
-                int g, f0, b0; tile_coords(t, g, f0, b0);
+                int k, g, f0, b0; tile_coords(t, k, g, f0, b0);
+                const int num_kb = (p.link[k].K + UM_BK - 1) / UM_BK;
                 const int fr = f0 + (int)rank * UP_BM;                     // first feature of this CTA
                 const int br = b0 + (int)rank * (BNB / 2);                 // first batch row of this CTA's half
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + UP_A_BYTES;
-                    const uint32_t fb_local = bar_full + 8 * stage;
-                    if (rank == 0) mbar_expect_tx(fb_local, 2 * STAGE_BYTES);   // both CTAs' copies complete on the leader's barrier
-                    const uint32_t fb = mapa_shared(fb_local, 0);
-                    if (!A_MN) {
-                        // K-major weights: block (row block fr/128, column block kb) of the blocked copy
-                        tma_pair_load_5d(sa, &tmW, fb, 0, 0, kb, fr / 128, g);
-                    } else {
-                        // MN-major weights: k-rows kb*64 .. +63 = half of row block kb/2; features fr .. fr+127 = two column blocks
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-                            tma_pair_load_5d(sa + h * (UP_A_BYTES / 2), &tmW, fb, 0, (kb & 1) * 64, fr / 64 + h, kb >> 1, g);
+                int kb = 0;
+                if (k > 0) {
+                    // The activations of this tile are what link k - 1 wrote for this replica; its weights depend on
+                    // nothing.  Weights of the first k-blocks first, then the wait, then their activations.
+                    const int ahead = num_kb < STAGES ? num_kb : STAGES;
+                    int st = stage; uint32_t ph = phase;
+                    for (int i = 0; i < ahead; ++i) {
+                        if (!mbar_wait(bar_empty + 8 * st, ph ^ 1u, abort_flag)) { ok = false; break; }
+                        if (rank == 0) mbar_expect_tx(bar_full + 8 * st, 2 * STAGE_BYTES);
+                        load_w(k, i, st, fr, g);
+                        if (++st == STAGES) { st = 0; ph ^= 1u; }
                     }
-                    tma_pair_load_3d(sb, &tmX, fb, kb * UM_BK, br, g);
+                    if (!ok) break;
+                    const int need = p.link[k - 1].tiles_f * p.tiles_b * 16;   // 8 epilogue warps of 2 CTAs per tile
+                    if (!wait_counter(p.sync + (k - 1) * p.groups + g, need, abort_flag)) { ok = false; break; }
+                    asm volatile("fence.proxy.async;" ::: "memory");       // the TMA reads below come after the acquire above
+                    for (int i = 0; i < ahead; ++i) {
+                        load_x(k, i, stage, br, g);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    kb = ahead;
+                }
+                for (; kb < num_kb; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2 * STAGE_BYTES);
+                    load_w(k, kb, stage, fr, g);
+                    load_x(k, kb, stage, br, g);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -206,6 +279,8 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             constexpr uint32_t idesc = make_pair_idesc(A_MN, BNB);
             int stage = 0; uint32_t phase = 0; int acc = 0; uint32_t acc_phase = 0; bool ok = true;
             for (int t = pair; t < total_tiles && ok; t += num_pairs) {
+                int k, g, f0, b0; tile_coords(t, k, g, f0, b0);
+                const int num_kb = (p.link[k].K + UM_BK - 1) / UM_BK;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BNB;
@@ -216,11 +291,11 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     const uint64_t adesc = A_MN ? make_smem_desc(sa, UP_A_BYTES / 2, 1024) : make_smem_desc(sa, 16, 1024);
                     const uint64_t bdesc = make_smem_desc(sb, 16, 1024);
 #pragma unroll
-                    for (int k = 0; k < UM_BK / 16; ++k) {
+                    for (int kk = 0; kk < UM_BK / 16; ++kk) {
                         // K-major: 16 bf16 = 32 B further along the row; MN-major: two 8-row groups = 2048 B
-                        const uint64_t a_k = adesc + (uint64_t)(A_MN ? k * 128 : k * 2);
-                        const uint64_t b_k = bdesc + (uint64_t)(k * 2);
-                        tc_pair_mma_bf16(d_tmem, a_k, b_k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        const uint64_t a_k = adesc + (uint64_t)(A_MN ? kk * 128 : kk * 2);
+                        const uint64_t b_k = bdesc + (uint64_t)(kk * 2);
+                        tc_pair_mma_bf16(d_tmem, a_k, b_k, idesc, (kb | kk) != 0 ? 1u : 0u);
                     }
                     tc_pair_commit(bar_empty + 8 * stage, 3);              // the stage is free in both CTAs once these retire
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -239,18 +314,19 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         int acc = 0; uint32_t acc_phase = 0;
         const uint32_t tempty_leader = mapa_shared(bar_tempty, 0);
         for (int t = pair; t < total_tiles; t += num_pairs) {
-            int g, f0, b0; tile_coords(t, g, f0, b0);
+            int k, g, f0, b0; tile_coords(t, k, g, f0, b0);
+            const UpLink &L = p.link[k];
             const int fw = f0 + (int)rank * UP_BM + q * 32;  // first feature of this warp
             const int f = fw + lane;                         // feature of this thread (= its tensor-memory lane)
-            const bool f_ok = f < p.F;
+            const bool f_ok = f < L.F;
             float bias_v = 0.f;
             uint4 mk[MASK_AHEAD ? CPW : 1][4];
-            if (EPI == UPE_FWD_HIDDEN && f_ok) bias_v = __ldg(p.bias + (long long)g * p.bias_gs + f);
+            if (EPI == UPE_FWD_HIDDEN && f_ok) bias_v = __ldg(L.bias + (long long)g * L.bias_gs + f);
             if (EPI == UPE_DGRAD && MASK_AHEAD) {
 #pragma unroll
                 for (int cc = 0; cc < CPW; ++cc) {
                     const int bb = b0 + (CPW * half + cc) * 32;
-                    const __nv_bfloat16 *mkp = p.maskT + (long long)g * p.maskT_gs + (long long)f * p.maskT_ld + bb;
+                    const __nv_bfloat16 *mkp = L.maskT + (long long)g * L.maskT_gs + (long long)f * L.maskT_ld + bb;
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8) {
                         mk[cc][j8] = make_uint4(0u, 0u, 0u, 0u);
@@ -267,7 +343,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 const int bb = b0 + c * 32;                  // first batch row of the chunk
                 if (bb >= p.Bt) break;                       // warp-uniform
                 if (EPI == UPE_DGRAD && !MASK_AHEAD) {
-                    const __nv_bfloat16 *mkp = p.maskT + (long long)g * p.maskT_gs + (long long)f * p.maskT_ld + bb;
+                    const __nv_bfloat16 *mkp = L.maskT + (long long)g * L.maskT_gs + (long long)f * L.maskT_ld + bb;
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8) {
                         mk[0][j8] = make_uint4(0u, 0u, 0u, 0u);
@@ -301,7 +377,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     pk[j] = *reinterpret_cast<uint32_t *>(&t2);
                 }
                 if (f_ok) {
-                    __nv_bfloat16 *oT = p.outT + (long long)g * p.outT_gs + (long long)f * p.outT_ld + bb;
+                    __nv_bfloat16 *oT = L.outT + (long long)g * L.outT_gs + (long long)f * L.outT_ld + bb;
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8)
                         if (bb + j8 * 8 < p.Bt)              // Bt % 8 == 0: the whole group is inside
@@ -316,13 +392,13 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     __syncwarp();
                     const int seg = lane & 3;                              // 8 features each
                     const int fs = fw + seg * 8;
-                    if (fs < p.F) {                                        // F % 8 == 0: the whole group is inside
-                        __nv_bfloat16 *o = p.out + (long long)g * p.out_gs + fs;
+                    if (fs < L.F) {                                        // F % 8 == 0: the whole group is inside
+                        __nv_bfloat16 *o = L.out + (long long)g * L.out_gs + fs;
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int bj = (lane >> 2) + 8 * i;
                             if (bb + bj < p.Bt)
-                                *reinterpret_cast<uint4 *>(o + (long long)(bb + bj) * p.out_ld) =
+                                *reinterpret_cast<uint4 *>(o + (long long)(bb + bj) * L.out_ld) =
                                     *reinterpret_cast<const uint4 *>(sT + bj * UM_EPI_PITCH + seg * 8);
                         }
                     }
@@ -331,7 +407,13 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * acc);
+            if (lane == 0) {
+                mbar_arrive_cluster(tempty_leader + 8 * acc);
+                if (k + 1 < p.n_links) {                     // the next link reads what this warp has just stored
+                    __threadfence();
+                    atomicAdd(p.sync + k * p.groups + g, 1);
+                }
+            }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -339,6 +421,16 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_before();
     cluster_sync_all();                                      // nobody touches the peer's shared or tensor memory after this
     if (threadIdx.x == 0 && *abort_flag) p.status[SLOT_WAIT_LIMIT] = 1;
+    if (threadIdx.x == 0 && p.n_links > 1) {
+        // every wait of this CTA on the counters is over; the last CTA to leave zeroes them for the next launch
+        int *leave = p.sync + UP_MAX_LINKS * PARLE_MAX_REPLICAS;
+        __threadfence();
+        if (atomicAdd(leave, 1) == (int)gridDim.x - 1) {
+            __threadfence();
+            for (int i = 0; i < (p.n_links - 1) * p.groups; ++i) p.sync[i] = 0;
+            *leave = 0;
+        }
+    }
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem_base), "r"(SH::TMEM_COLS) : "memory");

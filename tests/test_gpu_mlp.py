@@ -697,28 +697,34 @@ def test_split_y_rounds_keep_y_exactly_bf16(L, mu, dims, batch):
 
 
 @pytest.mark.parametrize("n,dims,batch", [(2, (320, 1152, 648, 101), 256), (3, (256, 512, 384, 10), 128),
-                                          (2, (200, 328, 264, 101), 136), (1, (64, 256, 256, 8), 16)])
+                                          (2, (200, 328, 264, 101), 136), (1, (64, 256, 256, 8), 16),
+                                          (5, (512, 1024, 768, 1024, 512, 256), 128), (16, (256, 256, 512, 256, 264, 16), 64)])
 def test_pair_gemm_gives_the_same_step_bf16(n, dims, batch):
     """Hidden-layer forward / data-gradient products on pairs of SMs (weights as the A operand of a two-CTA
     instruction, the activation tile shared by the pair) against the one-SM kernel: same products in the same k
-    order, so activations, their gradients, the weight gradient and the updated state agree bit for bit.  Batch tiles
-    of 128 and 256 rows, ragged feature and batch tails, a batch far smaller than the tile."""
+    order, so activations, their gradients, the weight gradient and the updated state agree bit for bit -- one launch
+    per layer, and consecutive layers chained in one launch whose tiles wait for the layer before them.  Batch tiles of
+    128 and 256 rows, ragged feature and batch tails, a batch far smaller than the tile."""
     cfg = si.C1.scaled(name="pair", n=n, dims=dims, batch=batch, gemm_dtype=1, L=2)
     X, c = si.round_batches(cfg, 0)
     nh = cfg.n_layers - 1
     res = []
-    for pair in (False, True):
-        m, *_ = make(cfg, fused=False)
+    for pair, fused in ((0, False), (1, False), (3, False), (0, True), (3, True)):
+        m, *_ = make(cfg, fused=fused)
         m.set_pair_gemm(pair)
         m.round_begin()
         for l in range(cfg.L):
             m.inner_step(torch.from_numpy(X[l]).to(DEV), torch.from_numpy(c[l]).to(DEV))
         torch.cuda.synchronize()
         assert m.status() == 0
-        res.append([m.y.clone(), m.grad.clone(), m.debug_buffer(m.DBG_LOGITS).clone()] +
+        res.append([m.y.clone(), m.debug_buffer(m.DBG_LOGITS).clone()] +
                    [m.debug_buffer(m.DBG_ACT, l).clone() for l in range(nh)] +
                    [m.debug_buffer(m.DBG_ACT_T, l).clone() for l in range(nh)] +
                    [m.debug_buffer(m.DBG_DACT, l).clone() for l in range(nh)] +
-                   [m.debug_buffer(m.DBG_DACT_T, l).clone() for l in range(nh)])
-    for k, (a, b) in enumerate(zip(*res)):
-        assert torch.equal(a, b), k
+                   [m.debug_buffer(m.DBG_DACT_T, l).clone() for l in range(nh)] +
+                   ([m.grad.clone()] if not fused else []))
+    # one launch per layer and the chained launch against the one-SM kernel (separate update: the gradient too);
+    # with the fused update (its data gradients all come first, in one chain) against the one-SM kernel
+    for other, base in ((1, 0), (2, 0), (4, 3)):
+        for k, (a, b) in enumerate(zip(res[other], res[base])):
+            assert torch.equal(a, b), (other, k)
