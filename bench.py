@@ -429,6 +429,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = si.CONFIGS[args.workload]
+    if args.replicas:       # a smaller copy of the workload (profiler captures); the line says so
+        cfg = cfg.scaled(n=args.replicas)
     if world > 1:           # every rank owns its own n replicas (independent streams per rank)
         cfg = cfg.scaled(seed=cfg.seed + 7919 * rank)
     W, K = max(args.warmup, 0), args.steps
@@ -446,10 +448,10 @@ def run_ours(args):
     roofline = rooflines.get(dom, {"kernel": dom, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": None, "traffic": None, "peak_source": peaks["source"]})
     extra = {}
-    if world == 1 and args.compact and args.workload == "C5":
+    if world == 1 and args.compact and args.workload == "C5" and not args.replicas:
         extra["c3"] = compact_c3(args, dev, local)
         extra["c4_sweep"] = compact_c4(dev)
-    cpu = cpu_baseline(cfg, budget_s=15.0)
+    cpu = cpu_baseline(cfg, budget_s=15.0) if args.cpu_baseline else None
     line = {
         "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": r["ms"] / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -570,6 +572,8 @@ def main():
     ap.add_argument("--split-y", type=int, default=1, help="bf16 workloads: y as bf16 copy + lower-half plane inside a round (parle_set_split_y)")
     ap.add_argument("--paired-z", type=int, default=1, help="Eq. (parle_z) two steps at a time inside a round (parle_set_paired_z_update)")
     ap.add_argument("--compact", type=int, default=1, help="one GPU, workload C5: add the compact C3 and update-sweep records to the line")
+    ap.add_argument("--replicas", type=int, default=0, help="override the workload's replica count (small cases for profiler captures)")
+    ap.add_argument("--cpu-baseline", type=int, default=1, help="0: skip the oracle timing on the host cores")
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend (gloo: with --dry, on CPUs)")
     ap.add_argument("--dry", action="store_true", help="rank logic only: no CUDA, no rounds")
     args = ap.parse_args()

@@ -234,6 +234,10 @@ __global__ void __launch_bounds__((BM / 8) * (BN / 8)) simt_gemm_tiled_kernel(Si
 // fp32 copy as a tf32-exact hi/lo pair in both layouts (dhi, dlo: [rows, ld_split]; dThi, dTlo: [C, B] per replica).
 // With parts > 1 the logits arrive as split-K partial sums: logits = bias + sum_s part_s (s in fixed order),
 // formed here first and written back over part 0 (= the logits buffer).
+// With loss != NULL the mean loss of every replica is formed here too: rows_done[g] (zero between launches) counts the
+// finished rows of replica g, and the warp that finishes the last one adds up the replica's row losses -- in the
+// same fixed order whoever does it (256 strided partial sums, then a binary tree), so the result does not depend on which
+// warp that is -- and puts the counter back to zero.
 __global__ void __launch_bounds__(256)
 softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict__ labels,
                            float *__restrict__ d32, __nv_bfloat16 *__restrict__ dbf,
@@ -241,7 +245,8 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
                            int rows, int B, int C, int ld_b, int *status,
                            int parts = 1, long long part_stride = 0, const float *__restrict__ bias = nullptr,
                            long long bias_gs = 0, float *__restrict__ dThi = nullptr, float *__restrict__ dTlo = nullptr,
-                           float *__restrict__ dhi = nullptr, float *__restrict__ dlo = nullptr, int ld_split = 0) {
+                           float *__restrict__ dhi = nullptr, float *__restrict__ dlo = nullptr, int ld_split = 0,
+                           float *__restrict__ loss = nullptr, int *__restrict__ rows_done = nullptr) {
     const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const int lane = threadIdx.x % 32;
     if (row >= rows) return;
@@ -326,22 +331,30 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
         row_loss[row] = label_ok ? (mx + __logf(s) - label_logit) : 0.f;
         if (!label_ok) status[SLOT_BAD_LABEL] = 1;
     }
-}
-
-// loss[g] = (1/B) sum_i row_loss[g, i]; one block per replica, fixed-order tree.
-__global__ void __launch_bounds__(256)
-loss_mean_kernel(const float *__restrict__ row_loss, float *__restrict__ loss, int B) {
-    __shared__ float sh[256];
-    const int g = blockIdx.x;
-    float s = 0.f;
-    for (int i = threadIdx.x; i < B; i += 256) s += row_loss[(size_t)g * B + i];
-    sh[threadIdx.x] = s;
-    __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) {
-        if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
-        __syncthreads();
+    if (loss) {
+        int before = 0;
+        if (lane == 0) {
+            __threadfence();                                 // this row's loss is visible before it is counted
+            before = atomicAdd(rows_done + g, 1);
+        }
+        before = __shfl_sync(0xffffffffu, before, 0);
+        if (before == B - 1) {                               // the replica's last row: all its row losses are in memory
+            __threadfence();
+            const float *rl = row_loss + (size_t)g * B;
+            float part[8];                                   // partial sums of "threads" lane, lane + 32, ..., lane + 224 of a 256-wide sum
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                part[k] = 0.f;
+                for (int r = lane + 32 * k; r < B; r += 256) part[k] += __ldcg(rl + r);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) part[k] += part[k + 4];          // tree step 128
+            part[0] += part[2]; part[1] += part[3];                       // 64
+            float t = part[0] + part[1];                                  // 32
+            for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
+            if (lane == 0) { loss[g] = t / (float)B; rows_done[g] = 0; }
+        }
     }
-    if (threadIdx.x == 0) loss[g] = sh[0] / (float)B;
 }
 
 // db[g, j] = sum_i dH[g, i, j] from fp32 dH [n, B, d] (thread per column).

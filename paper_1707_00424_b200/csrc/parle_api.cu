@@ -24,11 +24,11 @@ constexpr int kProfCapacity = 65536;       // launches recorded between two parl
 constexpr int kPlanSmCount = 148;
 
 enum KernelClass {
-    KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_LOSS_MEAN, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
+    KC_INPUT_CVT = 0, KC_FWD_GEMM, KC_SOFTMAX_CE, KC_WGRAD_GEMM, KC_BIAS_GRAD, KC_DGRAD_GEMM,
     KC_INNER_UPDATE, KC_OUTER_MEAN, KC_MEAN, KC_TO_BF16, KC_WGRAD_UPDATE, KC_TAIL_UPDATE, KC_COUNT
 };
 const char *const kClassNames[KC_COUNT] = {
-    "input_to_bf16", "fwd_gemm", "softmax_ce_backward", "loss_mean", "wgrad_gemm", "bias_grad", "dgrad_gemm",
+    "input_to_bf16", "fwd_gemm", "softmax_ce_backward", "wgrad_gemm", "bias_grad", "dgrad_gemm",
     "inner_update", "outer_mean", "mean", "to_bf16", "wgrad_gemm_fused_update", "tail_update"};
 
 struct Workspace {
@@ -42,6 +42,7 @@ struct Workspace {
     size_t dhb[PARLE_MAX_LAYERS], dhbT[PARLE_MAX_LAYERS];    // their gradients, both layouts
     int dh_ld[PARLE_MAX_LAYERS];       // row pitch of dhb[l] (d_{l+1} rounded up to 8)
     size_t row_loss;                   // [n,B] fp32
+    size_t rows_done;                  // [n] ints: rows of a replica the softmax kernel has finished (zero between launches)
     // fp32 mode on the tensor cores (3 x tf32): tf32-exact hi/lo pairs, index [0] = hi, [1] = lo
     size_t t3_logits;                  // fp32 logits [n, B, C] x t3_ksplit partial sums
     size_t w_split[2];                 // parameters [n, stride]
@@ -219,6 +220,7 @@ void plan_workspace(parle_ctx *c) {
         w.pair_sync = take(UP_SYNC_INTS * sizeof(int));
     }
     w.row_loss = take(n * B * sizeof(float));
+    w.rows_done = take(n * sizeof(int));
     for (int b = 0; b < 2; ++b) {
         w.stage_in[b] = take(n * B * c->dims[0] * sizeof(float));
         w.stage_lab[b] = take(n * B * sizeof(int32_t));
@@ -731,13 +733,9 @@ int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labe
         ws_ptr<float>(c, w.t3_logits), labels, nullptr, nullptr, nullptr, ws_ptr<float>(c, w.row_loss), rows, B, C, 0,
         c->status_dev, c->t3_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
         ws_ptr<float>(c, w.dhT[nl - 1][0]), ws_ptr<float>(c, w.dhT[nl - 1][1]),
-        ws_ptr<float>(c, w.dhs[nl - 1][0]), ws_ptr<float>(c, w.dhs[nl - 1][1]), (int)round_up(C, 4));
+        ws_ptr<float>(c, w.dhs[nl - 1][0]), ws_ptr<float>(c, w.dhs[nl - 1][1]), (int)round_up(C, 4),
+        loss_out, ws_ptr<int>(c, w.rows_done));
     PARLE_LAUNCHED(c);
-    if (loss_out) {
-        prof_begin(c, KC_LOSS_MEAN);
-        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
-        PARLE_LAUNCHED(c);
-    }
     for (int l = nl - 1; l >= 0; --l) {
         const int din = c->dims[l], dout = c->dims[l + 1];
         T3Params p = {};                                        // dW_l^T = H_{l-1}^T dH_l
@@ -783,13 +781,9 @@ int forward_backward_fp32(parle_ctx *c, const float *inputs, const int32_t *labe
     prof_begin(c, KC_SOFTMAX_CE);
     softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.act[nl - 1]), labels, ws_ptr<float>(c, w.dact[nl - 1]), nullptr, nullptr,
-        ws_ptr<float>(c, w.row_loss), rows, B, C, 0, c->status_dev);
+        ws_ptr<float>(c, w.row_loss), rows, B, C, 0, c->status_dev, 1, 0, nullptr, 0, nullptr, nullptr, nullptr, nullptr, 0,
+        loss_out, ws_ptr<int>(c, w.rows_done));
     PARLE_LAUNCHED(c);
-    if (loss_out) {
-        prof_begin(c, KC_LOSS_MEAN);
-        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
-        PARLE_LAUNCHED(c);
-    }
     for (int l = nl - 1; l >= 0; --l) {
         const int din = c->dims[l], dout = c->dims[l + 1];
         const float *act_in = l == 0 ? inputs : ws_ptr<float>(c, w.act[l - 1]);
@@ -855,13 +849,9 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
         ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
-        c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S);
+        c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
+        nullptr, nullptr, nullptr, nullptr, 0, loss_out, ws_ptr<int>(c, w.rows_done));
     PARLE_LAUNCHED(c);
-    if (loss_out) {
-        prof_begin(c, KC_LOSS_MEAN);
-        loss_mean_kernel<<<n, 256, 0, c->stream>>>(ws_ptr<float>(c, w.row_loss), loss_out, B);
-        PARLE_LAUNCHED(c);
-    }
     auto dgrad = [&](int l) -> int {                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
         const int din = c->dims[l], dout = c->dims[l + 1];
         if (use_pair_gemm(c, din)) return launch_pair<UPE_DGRAD>(c, KC_DGRAD_GEMM, l, l);
@@ -1152,6 +1142,8 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.sched), 0, 2 * sizeof(int), c->stream));
         PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.pair_sync), 0, UP_SYNC_INTS * sizeof(int), c->stream));
     }
+    if (c->n_layers > 0)            // row counters of the loss kernel: every launch leaves them at zero again
+        PARLE_CUDA(c, cudaMemsetAsync(ws_ptr<char>(c, c->ws.rows_done), 0, (size_t)c->n * sizeof(int), c->stream));
     c->t3_ready = false;
     if (c->t3_shapes_ok) {
         int major = 0;
