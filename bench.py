@@ -121,13 +121,17 @@ def dense_to_padded(model, cfg, replica_layers):
 
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture
-# (profiles/ncu_full_gemms_and_fused_update_C3.md), valid only while the kernel source is unchanged.
-NCU_TRAFFIC = {("C3", "wgrad_gemm_fused_update"): {
-    # dram__bytes_read.sum + dram__bytes_write.sum of one launch (all layers, all replicas): mean of the two variants
-    # that alternate inside a round, "z untouched" (985.3 + 433.0 MB) and "two-step z" (1462.6 + 900.7 MB)
-    "bytes": (985.298e6 + 432.966e6 + 1462.564e6 + 900.722e6) / 2,
-    "sources": ("paper_1707_00424_b200/csrc/umma_wgrad_update.cuh", "paper_1707_00424_b200/csrc/umma_gemm.cuh"),
-    "sources_sha256_16": "45c6fe3d686ff3ef"}}
+# (profiles/ncu_fused_update_and_pair_gemm_C5_one_replica.md), valid only while the kernel source is unchanged.
+# The capture ran a one-replica copy of the workload (3.9 GB of state); the kernel's traffic is proportional to the
+# number of replicas (every replica's weights are streamed once, nothing is shared between replicas), so the figure
+# below is the captured one times 16.
+NCU_TRAFFIC = {("C5", "wgrad_gemm_fused_update"): {
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch at n = 1: mean of the two variants that alternate inside
+    # a round, "z untouched" (1991.8 + 924.3 MB) and "two-step z" (3008.8 + 1888.3 MB)
+    "bytes": 16 * (1991.816704e6 + 924.272384e6 + 3008.821504e6 + 1888.308992e6) / 2,
+    "sources": ("paper_1707_00424_b200/csrc/umma_wgrad_update.cuh", "paper_1707_00424_b200/csrc/umma_gemm.cuh",
+                "paper_1707_00424_b200/csrc/common.cuh"),
+    "sources_sha256_16": "dba91041703a64ea"}}
 
 
 def sources_digest(sources):

@@ -628,7 +628,7 @@ int run_split_transpose(parle_ctx *c, const float *src);
 
 template <bool FIRST, bool MOM, bool SPLIT, int ZMODE>
 void launch_inner_update(parle_ctx *c, int grid, const float4 *g, float4 *y, const float4 *x, float4 *z, size_t n4, float wd) {
-    constexpr int U = 2;
+    constexpr int U = FIRST ? 4 : 2;          // the first step of a round reads two arrays instead of four: more of them in flight per thread
     inner_update_kernel<FIRST, U, MOM, SPLIT, ZMODE><<<grid, kUpdThreads, 0, c->stream>>>(
         g, y, x, z, n4, c->eta_prime, c->inv_gamma, c->alpha, wd, c->status_dev,
         MOM ? reinterpret_cast<float4 *>(c->vy) : nullptr, c->momentum,
