@@ -224,6 +224,15 @@ int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
  * (none: the k order is the same). */
 int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
 
+/* bf16 path, networks with at most 128 classes.  on (the default where the last layer has enough tiles to run without a
+ * split along K; with a few tiles only, as in an 8-replica batch-128 workload, the split GEMM followed by the loss kernel
+ * is faster and stays the default): the softmax cross-entropy backward of Section 1.1's
+ * loss runs in the epilogue of the last forward layer's GEMM (a logit row lies in one tile: the two warps that hold its
+ * halves exchange maximum, sum and label logit), which also writes the row losses and the replicas' mean losses; the
+ * layer is then not split along K.  off, or more classes: a kernel of its own after the GEMM.  The two agree to fp32
+ * rounding (different summation order of the exponentials).  EUNSUPPORTED on an fp32 context. */
+int parle_set_fused_loss(parle_ctx *ctx, int on);
+
 /* bf16 path: forward and data-gradient products of the hidden layers (Section 1.1 / 2.1) whose weight matrix has at
  * least 256 output rows run on pairs of SMs (one two-CTA tensor-core instruction per 256 x batch-tile block, the two CTAs
  * sharing the activation tile).  Consecutive such layers can go into ONE launch, whose tiles wait, per replica, for the

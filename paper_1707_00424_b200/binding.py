@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         "parle_set_weight_decay": (ci, [vp, cd]),
         "parle_set_wide_tile_threshold": (ci, [vp, ci]),
         "parle_set_pair_gemm": (ci, [vp, ci]),
+        "parle_set_fused_loss": (ci, [vp, ci]),
         "parle_bind_momentum": (ci, [vp, vp, vp]),
         "parle_set_momentum": (ci, [vp, cd]),
         "parle_scoping": (ci, [cd, cd, C.c_longlong, C.c_longlong, cd, cd, C.POINTER(cd), C.POINTER(cd)]),
@@ -261,6 +262,10 @@ class Parle:
 
     def set_wide_tile_threshold(self, tiles_per_sm: int):
         self._check(self._L.parle_set_wide_tile_threshold(self._h, tiles_per_sm), "parle_set_wide_tile_threshold")
+
+    def set_fused_loss(self, on: bool):
+        """bf16 path, at most 128 classes: softmax cross-entropy backward in the last forward GEMM's epilogue (default on)."""
+        self._check(self._L.parle_set_fused_loss(self._h, 1 if on else 0), "parle_set_fused_loss")
 
     def set_pair_gemm(self, mode: int):
         """bf16 path: hidden-layer forward / data-gradient products on pairs of SMs: 0 never, 1 one launch per layer,

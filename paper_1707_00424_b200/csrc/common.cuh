@@ -38,6 +38,35 @@ __device__ __forceinline__ __nv_bfloat16 bf16_weight(float v) {
     return __ushort_as_bfloat16((unsigned short)(bf16_split_word(v) >> 16));
 }
 
+// Mean loss of a replica, formed by whichever warp finishes the replica's last rows.  `count` rows of replica g (their
+// losses already stored in row_loss by this warp) are reported; rows_done[g] (zero between launches) counts them, and
+// the warp that completes the B rows adds all B row losses up in one fixed order (256 strided partial sums, then a
+// binary tree), stores loss[g] and puts the counter back to zero.  Called by all 32 lanes.
+static __device__ __noinline__ void replica_loss_finish(const float *row_loss, float *loss, int *rows_done,
+                                                    int g, int B, int count, int lane) {
+    int before = 0;
+    if (lane == 0 && count > 0) {
+        __threadfence();                                     // the row losses are visible before they are counted
+        before = atomicAdd(rows_done + g, count);
+    }
+    before = __shfl_sync(0xffffffffu, before, 0);
+    if (count <= 0 || before + count != B) return;
+    __threadfence();
+    const float *rl = row_loss + (size_t)g * B;
+    float part[8];                                           // partial sums of "threads" lane, lane + 32, ..., lane + 224 of a 256-wide sum
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        part[k] = 0.f;
+        for (int r = lane + 32 * k; r < B; r += 256) part[k] += __ldcg(rl + r);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) part[k] += part[k + 4];      // tree step 128
+    part[0] += part[2]; part[1] += part[3];                   // 64
+    float t = part[0] + part[1];                              // 32
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
+    if (lane == 0) { loss[g] = t / (float)B; rows_done[g] = 0; }
+}
+
 struct LayerPlan {
     int d_in, d_out;
     size_t w_off, b_off;          // element offsets inside one replica's vector

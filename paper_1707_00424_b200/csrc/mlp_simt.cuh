@@ -331,30 +331,7 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
         row_loss[row] = label_ok ? (mx + __logf(s) - label_logit) : 0.f;
         if (!label_ok) status[SLOT_BAD_LABEL] = 1;
     }
-    if (loss) {
-        int before = 0;
-        if (lane == 0) {
-            __threadfence();                                 // this row's loss is visible before it is counted
-            before = atomicAdd(rows_done + g, 1);
-        }
-        before = __shfl_sync(0xffffffffu, before, 0);
-        if (before == B - 1) {                               // the replica's last row: all its row losses are in memory
-            __threadfence();
-            const float *rl = row_loss + (size_t)g * B;
-            float part[8];                                   // partial sums of "threads" lane, lane + 32, ..., lane + 224 of a 256-wide sum
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                part[k] = 0.f;
-                for (int r = lane + 32 * k; r < B; r += 256) part[k] += __ldcg(rl + r);
-            }
-#pragma unroll
-            for (int k = 0; k < 4; ++k) part[k] += part[k + 4];          // tree step 128
-            part[0] += part[2]; part[1] += part[3];                       // 64
-            float t = part[0] + part[1];                                  // 32
-            for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
-            if (lane == 0) { loss[g] = t / (float)B; rows_done[g] = 0; }
-        }
-    }
+    if (loss) replica_loss_finish(row_loss, loss, rows_done, g, B, 1, lane);
 }
 
 // db[g, j] = sum_i dH[g, i, j] from fp32 dH [n, B, d] (thread per column).

@@ -66,7 +66,7 @@ struct RoundKey {
     const void *inputs, *labels, *loss;
     float scal[7];                   // 1/gamma, 1/rho, alpha, eta, eta', weight decay, momentum
     int fused, wide_thr, shadow_is_x, fresh;   // L == 0: a single inner step (fresh = first of its round)
-    int pair_gemm;
+    int pair_gemm, fused_loss;
     int paired_z, z_mode;            // whole rounds: Eq. (parle_z) in pairs or not; single steps: how this step treats z
     int split_y, y_step;             // whole rounds: y in two 16-bit planes or not; single steps: bit 0 = in that mode, bit 1 = stores fp32 y
     const void *ptrs[9];             // x, y, z, grad, xbar, workspace, vy, vx, stream
@@ -103,6 +103,7 @@ struct parle_ctx {
     bool y_split_step, y_write_step; // this step runs in that mode / also stores the fp32 y (set per step by the round drivers)
     int z_mode;                      // how the next fused step treats z (WU_Z_*); set per step by the round drivers
     bool fused_update;               // bf16 path: apply Eq. (parle_y)/(parle_z) inside the weight-gradient GEMM
+    bool fused_loss;                 // bf16 path, at most 128 classes: softmax cross-entropy backward inside the last forward GEMM's epilogue
     int steps_in_round;
     long long launches;
     int last_cuda;
@@ -815,6 +816,7 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     const int nl = c->n_layers, n = c->n, B = c->batch;
     const long long S = (long long)c->stride;
     const float *params = c->fresh ? c->buf.x : c->buf.y;      // fp32 biases come from the master copy
+    const bool loss_in_epilogue = c->fused_loss && c->dims[nl] <= 128;
     {
         const int d0 = c->dims[0];
         prof_begin(c, KC_INPUT_CVT);
@@ -838,20 +840,31 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
             p.out = ws_ptr<__nv_bfloat16>(c, w.hb[l]); p.out_gs = (long long)B * dout; p.out_ld = dout;
             p.outT = ws_ptr<__nv_bfloat16>(c, w.hbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
             PARLE_TRY((launch_umma<UEPI_FWD_HIDDEN, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
+        } else if (loss_in_epilogue) {
+            // the last layer with the loss: logits, dlogits (both layouts), row losses and the mean loss from one kernel
+            p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
+            p.out = ws_ptr<__nv_bfloat16>(c, w.dhb[l]); p.out_gs = (long long)B * w.dh_ld[l]; p.out_ld = w.dh_ld[l];
+            p.outT = ws_ptr<__nv_bfloat16>(c, w.dhbT[l]); p.outT_gs = (long long)B * dout; p.outT_ld = B;
+            p.labels = labels; p.row_loss = ws_ptr<float>(c, w.row_loss);
+            p.loss = loss_out; p.rows_done = ws_ptr<int>(c, w.rows_done);
+            p.ksplit = 1;
+            PARLE_TRY((launch_umma_bn<UEPI_FWD_LAST_CE, UB_BLOCKED_K, 128>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         } else {
             p.outf = ws_ptr<float>(c, w.logits); p.outf_gs = (long long)B * dout; p.outf_ld = dout;
             p.ksplit = c->last_ksplit; p.part_ss = (long long)n * B * dout;
             PARLE_TRY((launch_umma<UEPI_FWD_LAST, UB_BLOCKED_K>(c, KC_FWD_GEMM, c->tm_fwd_a[l], c->tm_fwd_b[l], p)));
         }
     }
-    const int C = c->dims[nl], rows = n * B;
-    prof_begin(c, KC_SOFTMAX_CE);
-    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
-        ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
-        ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
-        c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
-        nullptr, nullptr, nullptr, nullptr, 0, loss_out, ws_ptr<int>(c, w.rows_done));
-    PARLE_LAUNCHED(c);
+    if (!loss_in_epilogue) {
+        const int C = c->dims[nl], rows = n * B;
+        prof_begin(c, KC_SOFTMAX_CE);
+        softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+            ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
+            ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
+            c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
+            nullptr, nullptr, nullptr, nullptr, 0, loss_out, ws_ptr<int>(c, w.rows_done));
+        PARLE_LAUNCHED(c);
+    }
     auto dgrad = [&](int l) -> int {                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
         const int din = c->dims[l], dout = c->dims[l + 1];
         if (use_pair_gemm(c, din)) return launch_pair<UPE_DGRAD>(c, KC_DGRAD_GEMM, l, l);
@@ -1059,6 +1072,10 @@ int parle_init(parle_ctx **out, int n, const parle_model *model, double gamma, d
         if (s > num_kb / 2) s = num_kb / 2;
         if (s >= 2) c->last_ksplit = s;
     }
+    // The loss goes into the last layer's epilogue by default only where that layer has tiles enough not to be split
+    // along K: with a handful of tiles (C3: 8) one CTA per tile streaming the whole K is slower than the split GEMM plus
+    // the loss kernel (measured: +25 us per inner step).
+    c->fused_loss = c->fused_update && c->last_ksplit == 1 && c->dims[c->n_layers] <= 128;
     plan_workspace(c);
     *out = c;
     return PARLE_OK;
@@ -1121,6 +1138,7 @@ int parle_bind(parle_ctx *c, const parle_buffers *b, void *cuda_stream) {
         if (major != 10) return PARLE_EUNSUPPORTED;             // tcgen05 kernels need sm_100
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_HIDDEN, UB_BLOCKED_K>()));
         PARLE_CUDA(c, (allow_big_smem<UEPI_FWD_LAST, UB_BLOCKED_K>()));
+        PARLE_CUDA(c, cudaFuncSetAttribute(umma_gemm_kernel<UEPI_FWD_LAST_CE, UB_BLOCKED_K, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UM_SMEM_BYTES));
         PARLE_CUDA(c, (allow_big_smem<UEPI_WGRAD, UB_ROWMAJOR_K>()));
 #define PARLE_WU_SMEM(FIRST, SH, MOM, ZM) \
         PARLE_CUDA(c, cudaFuncSetAttribute(umma_wgrad_update_kernel<FIRST, SH, MOM, ZM, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SH::SMEM_BYTES)); \
@@ -1262,7 +1280,7 @@ static RoundKey make_round_key(const parle_ctx *c, int L, const void *in, const 
     const float sc[7] = {c->inv_gamma, c->inv_rho, c->alpha, c->eta, c->eta_prime, c->weight_decay, c->momentum};
     memcpy(k.scal, sc, sizeof(sc));
     k.fused = c->fused_update; k.wide_thr = c->wide_tiles_per_sm; k.shadow_is_x = c->shadow_is_x; k.fresh = c->fresh;
-    k.pair_gemm = c->pair_gemm;
+    k.pair_gemm = c->pair_gemm; k.fused_loss = c->fused_loss;
     k.paired_z = c->paired_z; k.z_mode = c->z_mode;
     k.split_y = c->split_y; k.y_step = (c->y_split_step ? 1 : 0) | (c->y_write_step ? 2 : 0);
     const void *pt[9] = {c->buf.x, c->buf.y, c->buf.z, c->buf.grad, c->buf.xbar, c->buf.workspace, c->vy, c->vx, c->stream};
@@ -1496,6 +1514,13 @@ int parle_fp32_tensor_cores_active(const parle_ctx *c) { return c ? (use_t3(c) ?
 int parle_set_wide_tile_threshold(parle_ctx *c, int tiles_per_sm) {
     if (!c || tiles_per_sm < 0) return PARLE_EINVAL;
     c->wide_tiles_per_sm = tiles_per_sm;
+    return PARLE_OK;
+}
+
+int parle_set_fused_loss(parle_ctx *c, int on) {
+    if (!c) return PARLE_EINVAL;
+    if (c->gemm_dtype != PARLE_GEMM_BF16 || c->n_layers == 0) return on ? PARLE_EUNSUPPORTED : PARLE_OK;
+    c->fused_loss = on != 0;
     return PARLE_OK;
 }
 

@@ -56,7 +56,9 @@ enum UmmaEpilogue {
     UEPI_FWD_HIDDEN = 0,   // + bias[n], ReLU, bf16 out [M,ld] and transposed out [N,ldT]
     UEPI_FWD_LAST = 1,     // + bias[n], fp32 out [M,ld]
     UEPI_DGRAD = 2,        // * (mask[m,n] > 0), bf16 out and transposed out
-    UEPI_WGRAD = 3         // fp32 out, transposed: element (m, n) -> outf[n * ld + m]
+    UEPI_WGRAD = 3,        // fp32 out, transposed: element (m, n) -> outf[n * ld + m]
+    UEPI_FWD_LAST_CE = 4   // last layer with the loss in the epilogue (N <= 128): + bias[n], fp32 logits out, then row-wise
+                           // softmax cross-entropy: dlogits = (softmax - onehot)/M as bf16 in both layouts, row losses, mean loss
 };
 
 struct UmmaParams {
@@ -70,6 +72,9 @@ struct UmmaParams {
     // split-K (UEPI_FWD_LAST only): each tile's k-blocks are divided among ksplit work items, each of which
     // stores its raw partial sums (no bias) at outf + split * part_ss; a later kernel adds them up in fixed order
     int ksplit; long long part_ss;
+    // UEPI_FWD_LAST_CE: labels [groups, M]; dlogits bf16 [M, dbf_ld] and transposed [N, M] per replica (out / outT fields);
+    // row_loss [groups, M]; loss [groups] or NULL with its row counters (see replica_loss_finish)
+    const int32_t *labels; float *row_loss; float *loss; int *rows_done;
     int *status;
 };
 
@@ -357,7 +362,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             constexpr bool MASK_AHEAD = (BN == 128);         // wide tiles: the mask is read chunk by chunk (registers)
             float bias_lane[CPW];                            // bias[nb + lane] of this warp's chunks
             uint4 mk[MASK_AHEAD ? CPW : 1][4];               // ReLU mask source: 32 bf16 of row m per chunk
-            if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_FWD_LAST) {
+            if (EPI == UEPI_FWD_HIDDEN || EPI == UEPI_FWD_LAST || EPI == UEPI_FWD_LAST_CE) {
                 const float *bias = p.bias + (long long)g * p.bias_gs;
 #pragma unroll
                 for (int cc = 0; cc < CPW; ++cc) {
@@ -380,7 +385,129 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            {
+            if (EPI == UEPI_FWD_LAST_CE) {
+                // The whole logit row of a batch entry lies in this tile (N <= 128): this warp holds columns 64*half .. +63
+                // of its 32 rows, its partner warp (same lane quarter, other half) the rest.  The two exchange the row
+                // maximum, the sum of exponentials and the label's logit through their scratch tiles (named barrier of
+                // the 64 threads), then each forms its half of dlogits = (softmax - onehot)/M.
+                static_assert(EPI != UEPI_FWD_LAST_CE || BN == 128, "loss epilogue: one 128-wide tile per row");
+                float *mine = reinterpret_cast<float *>(epi_scratch + (warp - 2) * UM_EPI_SCRATCH);
+                const float *theirs = reinterpret_cast<const float *>(epi_scratch + ((warp - 2) ^ 4) * UM_EPI_SCRATCH);
+                auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory"); };
+                float v[2][32];
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    uint32_t r[32];
+                    tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + (2 * half + cc) * 32), r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[cc][j] = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane[cc], j);
+                }
+                const int c0 = n0 + half * 64;                   // first column of this warp
+                const int label = m_ok ? p.labels[(long long)g * p.M + m] : 0;
+                const bool label_ok = label >= 0 && label < p.N;
+                float mx = -INFINITY, cand = 0.f;
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int col = c0 + cc * 32 + j;
+                        if (col < p.N) mx = fmaxf(mx, v[cc][j]);
+                        if (col == label) cand = v[cc][j];
+                    }
+                mine[lane] = mx; mine[64 + lane] = cand;
+                pair_sync();
+                mx = fmaxf(mx, theirs[lane]);
+                const float label_logit = half == 0 ? cand + theirs[64 + lane] : theirs[64 + lane] + cand;
+                float se = 0.f;
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c0 + cc * 32 + j < p.N) se += __expf(v[cc][j] - mx);
+                mine[32 + lane] = se;
+                pair_sync();
+                const float s_all = half == 0 ? se + theirs[32 + lane] : theirs[32 + lane] + se;     // same sum in both warps
+                const float inv_s = 1.f / s_all, inv_M = 1.f / (float)p.M;
+                if (m_ok) {                                      // fp32 logits, as the plain last-layer epilogue stores them
+                    float *o = p.outf + (long long)g * p.outf_gs + (long long)m * p.outf_ld + c0;
+                    const bool vec = (p.outf_ld & 3) == 0;       // rows start 16-byte aligned: four columns per store
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const int col = c0 + cc * 32 + j;
+                            if (vec && col + 3 < p.N) {
+                                *reinterpret_cast<float4 *>(o + cc * 32 + j) = make_float4(v[cc][j], v[cc][j + 1], v[cc][j + 2], v[cc][j + 3]);
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k)
+                                    if (col + k < p.N) o[cc * 32 + j + k] = v[cc][j + k];
+                            }
+                        }
+                }
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int col = c0 + cc * 32 + j;
+                        float d = __expf(v[cc][j] - mx) * inv_s;
+                        if (col == label) d -= 1.f;
+                        v[cc][j] = col < p.N ? d * inv_M : 0.f;
+                    }
+                if (half == 0) {
+                    if (m_ok) {
+                        p.row_loss[(long long)g * p.M + m] = label_ok ? (mx + __logf(s_all) - label_logit) : 0.f;
+                        if (!label_ok) p.status[SLOT_BAD_LABEL] = 1;
+                    }
+                    __syncwarp();
+                    if (p.loss) {
+                        int cnt = p.M - (m0 + q * 32);
+                        cnt = cnt < 0 ? 0 : (cnt > 32 ? 32 : cnt);
+                        replica_loss_finish(p.row_loss, p.loss, p.rows_done, g, p.M, cnt, lane);
+                    }
+                }
+                pair_sync();                                     // the partner has read this warp's scratch: it is free for the transposition
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int nb = c0 + cc * 32;
+                    if (nb >= p.out_ld) break;                   // warp-uniform (out_ld = N rounded up to 8)
+                    if (m_ok) {                                  // [M, out_ld]: 32 consecutive columns of the thread's row
+                        __nv_bfloat16 *o = p.out + (long long)g * p.out_gs + (long long)m * p.out_ld + nb;
+#pragma unroll
+                        for (int j8 = 0; j8 < 32; j8 += 8) {
+                            if (nb + j8 < p.out_ld) {
+                                uint4 pk;
+                                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[cc][j8 + 0], v[cc][j8 + 1]);
+                                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[cc][j8 + 2], v[cc][j8 + 3]);
+                                __nv_bfloat162 t2 = __floats2bfloat162_rn(v[cc][j8 + 4], v[cc][j8 + 5]);
+                                __nv_bfloat162 t3 = __floats2bfloat162_rn(v[cc][j8 + 6], v[cc][j8 + 7]);
+                                pk.x = *reinterpret_cast<uint32_t *>(&t0); pk.y = *reinterpret_cast<uint32_t *>(&t1);
+                                pk.z = *reinterpret_cast<uint32_t *>(&t2); pk.w = *reinterpret_cast<uint32_t *>(&t3);
+                                *reinterpret_cast<uint4 *>(o + j8) = pk;
+                            }
+                        }
+                    }
+                    // [N, M]: through the scratch tile, 8 consecutive batch rows of one class per store
+                    __nv_bfloat16 *sT = reinterpret_cast<__nv_bfloat16 *>(mine);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) sT[j * UM_EPI_PITCH + lane] = __float2bfloat16_rn(v[cc][j]);
+                    __syncwarp();
+                    const int seg = lane & 3;
+                    const int mrow = m0 + q * 32 + seg * 8;
+                    if (mrow < p.M) {
+                        __nv_bfloat16 *oT = p.outT + (long long)g * p.outT_gs + mrow;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int f = (lane >> 2) + 8 * i;
+                            if (nb + f < p.N)
+                                *reinterpret_cast<uint4 *>(oT + (long long)(nb + f) * p.outT_ld) =
+                                    *reinterpret_cast<const uint4 *>(sT + f * UM_EPI_PITCH + seg * 8);
+                        }
+                    }
+                    __syncwarp();
+                }
+            } else {
 #pragma unroll
             for (int cc = 0; cc < CPW; ++cc) {
                 const int c = CPW * half + cc;

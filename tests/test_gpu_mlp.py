@@ -728,3 +728,39 @@ def test_pair_gemm_gives_the_same_step_bf16(n, dims, batch):
     for other, base in ((1, 0), (2, 0), (4, 3)):
         for k, (a, b) in enumerate(zip(res[other], res[base])):
             assert torch.equal(a, b), (other, k)
+
+
+@pytest.mark.parametrize("n,dims,batch", [(3, (64, 128, 72, 10), 16), (2, (200, 328, 136, 101), 136), (2, (256, 512, 128), 264),
+                                          (8, (3072, 2048, 2048, 2048, 100), 128)])
+def test_loss_in_the_last_gemm_epilogue_matches_the_separate_kernel_bf16(n, dims, batch):
+    """Softmax cross-entropy backward inside the last forward GEMM's epilogue (at most 128 classes) against the
+    kernel of its own: the logits are the same accumulators (bit-identical when the other path does not split K),
+    dlogits and the losses agree to fp32 rounding of the exponential sums, and both match the oracle's softmax
+    cross-entropy on those logits.  1, 2 and 3 batch tiles; 10, 100, 101 and 128 classes."""
+    cfg = si.C1.scaled(name="ce", n=n, dims=dims, batch=batch, gemm_dtype=1, L=1)
+    X, c = si.round_batches(cfg, 0)
+    C = dims[-1]
+    res = []
+    for fused_loss in (True, False):
+        m, *_ = make(cfg, fused=False)
+        m.set_fused_loss(fused_loss)
+        loss = torch.full((cfg.n,), float("nan"), device=DEV)
+        m.round_begin()
+        m.inner_step(torch.from_numpy(X[0]).to(DEV), torch.from_numpy(c[0]).to(DEV), loss)
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        res.append((m.debug_buffer(m.DBG_LOGITS).clone(), m.debug_buffer(m.DBG_DACT, cfg.n_layers - 1).float().clone(),
+                    m.debug_buffer(m.DBG_DACT_T, cfg.n_layers - 1).float().clone(), loss.clone(), m.grad.clone()))
+    (lg1, d1, dT1, l1, g1), (lg0, d0, dT0, l0, g0) = res
+    assert torch.allclose(lg1, lg0, rtol=1e-5, atol=1e-6)
+    assert torch.equal(dT1.transpose(1, 2), d1) and torch.equal(dT0.transpose(1, 2), d0)
+    # bf16 dlogits: at most one unit in the last place apart, and rarely
+    assert (d1 != d0).float().mean() < 1e-2 and torch.all((d1 - d0).abs() <= 2.0 ** -7 * d0.abs() + 1e-9)
+    assert torch.allclose(l1, l0, rtol=1e-6, atol=1e-7)
+    assert rel_l2(g1.cpu().numpy(), g0.cpu().numpy()) < 2e-3
+    lg = lg1.cpu().numpy().astype(np.float64)
+    for a in range(cfg.n):
+        want_l, want_d = po.softmax_ce(lg[a], c[0, a])
+        assert abs(l1[a].item() - want_l) <= 1e-5 * max(1.0, abs(want_l))
+        got = d1[a].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - want_d) <= 2.0 ** -7 * np.abs(want_d) + 1e-9)
