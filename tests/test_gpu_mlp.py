@@ -588,11 +588,12 @@ def test_fused_momentum_update_equals_separate_update_bf16(dims, batch, n):
         assert torch.equal(a, b)
 
 
-@pytest.mark.parametrize("gemm_dtype,dims", [(0, (64, 32, 10)), (1, (64, 128, 72, 10))])
+@pytest.mark.parametrize("gemm_dtype,dims", [(0, (64, 32, 10)), (1, (64, 128, 72, 10)), (1, (64, 256, 512, 256, 10))])
 def test_graph_rounds_equal_plain_rounds(gemm_dtype, dims):
     """parle_round replayed from a CUDA graph gives bit-identical state, also when the inputs alternate
     between two sets (two cached graphs), when a setting changes (new graph) and with more input sets than
-    the cache holds."""
+    the cache holds.  The last shape has hidden layers wide enough for the two-CTA GEMM kernel, whose cluster
+    launches chain the layers through progress counters: those launches are graph nodes like any other."""
     cfg = si.C1.scaled(dims=dims, gemm_dtype=gemm_dtype, L=4)
     sets = [si.round_batches(cfg, r) for r in range(10)]
     dev = [(torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)) for X, c in sets]
