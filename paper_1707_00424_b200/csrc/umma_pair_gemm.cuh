@@ -12,9 +12,8 @@
 // activations, against 16 + 16 or 32 + 16 KiB per 128 x 128 or 128 x 256 tile of the one-SM kernel.
 //
 // The accumulator is the transposed output: tensor-memory lane = output feature, column = batch row.  The epilogue
-// (bias + ReLU, or the ReLU mask of the data gradient) stores both layouts the other kernels read: [d, B] straight
-// from registers (a thread owns 32 consecutive batch entries of its feature) and [B, d] through a per-warp
-// shared-memory tile.
+// (bias + ReLU, or the ReLU mask of the data gradient) stores both layouts the other kernels read, [d, B] and
+// [B, d], each through a per-warp shared-memory tile so that every store instruction fills whole 32-byte sectors.
 //
 // Synchronisation inside a pair (cluster of two CTAs, rank 0 = leader):
 //   * both CTAs load their own halves with TMA (plain loads, no multicast) and signal the LEADER's "full" barrier,
@@ -51,8 +50,11 @@ constexpr int UP_SYNC_INTS = UP_MAX_LINKS * PARLE_MAX_REPLICAS + 1;   // per-(li
 
 template <int BNB> struct UpShape {
     static_assert(BNB == 128 || BNB == 256, "batch tile");
+    // 64-wide k-blocks that travel through the ring as one stage.  With the batch tile of 128 the MMAs of a k-block
+    // take the issuing thread 130 ns and the commit that frees the stage another 70 ns: two k-blocks share a commit.
+    static constexpr int KPS = BNB == 128 ? 2 : 1;
     static constexpr int B_BYTES = (BNB / 2) * UM_BK * 2;   // this CTA's half of the activation k-block
-    static constexpr int STAGE_BYTES = UP_A_BYTES + B_BYTES;
+    static constexpr int STAGE_BYTES = KPS * (UP_A_BYTES + B_BYTES);   // [W k-block 0 .. | X k-block 0 ..]
     static constexpr int STAGES = UP_RING_BYTES / STAGE_BYTES;
     static constexpr uint32_t TMEM_COLS = 2 * BNB;          // two accumulators
     static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 8 * UM_EPI_SCRATCH + 1024 /*alignment*/ + 256 /*barriers*/;
@@ -161,7 +163,7 @@ template <int EPI, int BNB>
 __global__ void __launch_bounds__(UP_THREADS, 1)
 umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant__ UmmaPairParams p) {
     using SH = UpShape<BNB>;
-    constexpr int STAGES = SH::STAGES, STAGE_BYTES = SH::STAGE_BYTES;
+    constexpr int STAGES = SH::STAGES, STAGE_BYTES = SH::STAGE_BYTES, B_BYTES = SH::B_BYTES, KPS = SH::KPS;
     constexpr bool A_MN = (EPI == UPE_DGRAD);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -215,37 +217,46 @@ umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant
         // ------------------------------------------------ TMA producer: this CTA's rows of W and its half of the batch tile
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            auto load_w = [&](int k, int kb, int st, int fr, int g) {
-                const uint32_t sa = ring + st * STAGE_BYTES;
+            // stage `st` takes the k-blocks s * KPS .. s * KPS + nb - 1 of a tile
+            auto load_w = [&](int k, int s, int nb, int st, int fr, int g) {
                 const uint32_t fb = mapa_shared(bar_full + 8 * st, 0);     // both CTAs' copies complete on the leader's barrier
-                if (!A_MN) {
-                    // K-major weights: block (row block fr/128, column block kb) of the blocked copy
-                    tma_pair_load_5d(sa, &maps.w[k], fb, 0, 0, kb, fr / 128, g);
-                } else {
-                    // MN-major weights: k-rows kb*64 .. +63 = half of row block kb/2; features fr .. fr+127 = two column blocks
+                for (int j = 0; j < nb; ++j) {
+                    const int kb = s * KPS + j;
+                    const uint32_t sa = ring + st * STAGE_BYTES + j * UP_A_BYTES;
+                    if (!A_MN) {
+                        // K-major weights: block (row block fr/128, column block kb) of the blocked copy
+                        tma_pair_load_5d(sa, &maps.w[k], fb, 0, 0, kb, fr / 128, g);
+                    } else {
+                        // MN-major weights: k-rows kb*64 .. +63 = half of row block kb/2; features fr .. fr+127 = two column blocks
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_pair_load_5d(sa + h * (UP_A_BYTES / 2), &maps.w[k], fb, 0, (kb & 1) * 64, fr / 64 + h, kb >> 1, g);
+                        for (int h = 0; h < 2; ++h)
+                            tma_pair_load_5d(sa + h * (UP_A_BYTES / 2), &maps.w[k], fb, 0, (kb & 1) * 64, fr / 64 + h, kb >> 1, g);
+                    }
                 }
             };
-            auto load_x = [&](int k, int kb, int st, int br, int g) {
-                tma_pair_load_3d(ring + st * STAGE_BYTES + UP_A_BYTES, &maps.x[k], mapa_shared(bar_full + 8 * st, 0), kb * UM_BK, br, g);
+            auto load_x = [&](int k, int s, int nb, int st, int br, int g) {
+                const uint32_t fb = mapa_shared(bar_full + 8 * st, 0);
+                for (int j = 0; j < nb; ++j)
+                    tma_pair_load_3d(ring + st * STAGE_BYTES + KPS * UP_A_BYTES + j * B_BYTES, &maps.x[k], fb, (s * KPS + j) * UM_BK, br, g);
             };
+            auto blocks_in = [&](int s, int num_kb) { return num_kb - s * KPS < KPS ? num_kb - s * KPS : KPS; };
             for (int t = pair; t < total_tiles && ok; t += num_pairs) {
                 int k, g, f0, b0; tile_coords(t, k, g, f0, b0);
                 const int num_kb = (p.link[k].K + UM_BK - 1) / UM_BK;
+                const int num_s = (num_kb + KPS - 1) / KPS;                // stages of this tile
                 const int fr = f0 + (int)rank * UP_BM;                     // first feature of this CTA
                 const int br = b0 + (int)rank * (BNB / 2);                 // first batch row of this CTA's half
-                int kb = 0;
+                int s = 0;
                 if (k > 0) {
                     // The activations of this tile are what link k - 1 wrote for this replica; its weights depend on
-                    // nothing.  Weights of the first k-blocks first, then the wait, then their activations.
-                    const int ahead = num_kb < STAGES ? num_kb : STAGES;
+                    // nothing.  Weights of the first stages first, then the wait, then their activations.
+                    const int ahead = num_s < STAGES ? num_s : STAGES;
                     int st = stage; uint32_t ph = phase;
                     for (int i = 0; i < ahead; ++i) {
                         if (!mbar_wait(bar_empty + 8 * st, ph ^ 1u, abort_flag)) { ok = false; break; }
-                        if (rank == 0) mbar_expect_tx(bar_full + 8 * st, 2 * STAGE_BYTES);
-                        load_w(k, i, st, fr, g);
+                        const int nb = blocks_in(i, num_kb);
+                        if (rank == 0) mbar_expect_tx(bar_full + 8 * st, 2 * nb * (UP_A_BYTES + B_BYTES));
+                        load_w(k, i, nb, st, fr, g);
                         if (++st == STAGES) { st = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
@@ -253,16 +264,17 @@ umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant
                     if (!wait_counter(p.sync + (k - 1) * p.groups + g, need, abort_flag)) { ok = false; break; }
                     asm volatile("fence.proxy.async;" ::: "memory");       // the TMA reads below come after the acquire above
                     for (int i = 0; i < ahead; ++i) {
-                        load_x(k, i, stage, br, g);
+                        load_x(k, i, blocks_in(i, num_kb), stage, br, g);
                         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     }
-                    kb = ahead;
+                    s = ahead;
                 }
-                for (; kb < num_kb; ++kb) {
+                for (; s < num_s; ++s) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2 * STAGE_BYTES);
-                    load_w(k, kb, stage, fr, g);
-                    load_x(k, kb, stage, br, g);
+                    const int nb = blocks_in(s, num_kb);
+                    if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2 * nb * (UP_A_BYTES + B_BYTES));
+                    load_w(k, s, nb, stage, fr, g);
+                    load_x(k, s, nb, stage, br, g);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -284,18 +296,23 @@ umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BNB;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb0 = 0; kb0 < num_kb; kb0 += KPS) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + UP_A_BYTES;
-                    const uint64_t adesc = A_MN ? make_smem_desc(sa, UP_A_BYTES / 2, 1024) : make_smem_desc(sa, 16, 1024);
-                    const uint64_t bdesc = make_smem_desc(sb, 16, 1024);
 #pragma unroll
-                    for (int kk = 0; kk < UM_BK / 16; ++kk) {
-                        // K-major: 16 bf16 = 32 B further along the row; MN-major: two 8-row groups = 2048 B
-                        const uint64_t a_k = adesc + (uint64_t)(A_MN ? kk * 128 : kk * 2);
-                        const uint64_t b_k = bdesc + (uint64_t)(kk * 2);
-                        tc_pair_mma_bf16(d_tmem, a_k, b_k, idesc, (kb | kk) != 0 ? 1u : 0u);
+                    for (int j = 0; j < KPS; ++j) {
+                        if (kb0 + j >= num_kb) break;
+                        const uint32_t sa = ring + stage * STAGE_BYTES + j * UP_A_BYTES;
+                        const uint32_t sb = ring + stage * STAGE_BYTES + KPS * UP_A_BYTES + j * B_BYTES;
+                        const uint64_t adesc = A_MN ? make_smem_desc(sa, UP_A_BYTES / 2, 1024) : make_smem_desc(sa, 16, 1024);
+                        const uint64_t bdesc = make_smem_desc(sb, 16, 1024);
+#pragma unroll
+                        for (int kk = 0; kk < UM_BK / 16; ++kk) {
+                            // K-major: 16 bf16 = 32 B further along the row; MN-major: two 8-row groups = 2048 B
+                            const uint64_t a_k = adesc + (uint64_t)(A_MN ? kk * 128 : kk * 2);
+                            const uint64_t b_k = bdesc + (uint64_t)(kk * 2);
+                            tc_pair_mma_bf16(d_tmem, a_k, b_k, idesc, (kb0 | j | kk) != 0 ? 1u : 0u);
+                        }
                     }
                     tc_pair_commit(bar_empty + 8 * stage, 3);              // the stage is free in both CTAs once these retire
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -376,17 +393,31 @@ umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant
                     __nv_bfloat162 t2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
                     pk[j] = *reinterpret_cast<uint32_t *>(&t2);
                 }
-                if (f_ok) {
-                    __nv_bfloat16 *oT = L.outT + (long long)g * L.outT_gs + (long long)f * L.outT_ld + bb;
+                __nv_bfloat16 *sT = reinterpret_cast<__nv_bfloat16 *>(epi_scratch + (warp - 2) * UM_EPI_SCRATCH);
+                {
+                    // through this warp's scratch tile (row = feature), so that four lanes store the 64 bytes a feature
+                    // has in this chunk and an instruction covers eight features: stored straight from the registers,
+                    // every lane would touch a line of its own four times over
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8)
-                        if (bb + j8 * 8 < p.Bt)              // Bt % 8 == 0: the whole group is inside
-                            *reinterpret_cast<uint4 *>(oT + j8 * 8) = make_uint4(pk[4 * j8], pk[4 * j8 + 1], pk[4 * j8 + 2], pk[4 * j8 + 3]);
+                        *reinterpret_cast<uint4 *>(sT + lane * UM_EPI_PITCH + j8 * 8) = make_uint4(pk[4 * j8], pk[4 * j8 + 1], pk[4 * j8 + 2], pk[4 * j8 + 3]);
+                    __syncwarp();
+                    const int seg = lane & 3;                              // 8 batch entries each
+                    if (bb + seg * 8 < p.Bt) {                             // Bt % 8 == 0: the whole group is inside
+                        __nv_bfloat16 *oT = L.outT + (long long)g * L.outT_gs + bb + seg * 8;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int fj = (lane >> 2) + 8 * i;
+                            if (fw + fj < L.F)
+                                *reinterpret_cast<uint4 *>(oT + (long long)(fw + fj) * L.outT_ld) =
+                                    *reinterpret_cast<const uint4 *>(sT + fj * UM_EPI_PITCH + seg * 8);
+                        }
+                    }
+                    __syncwarp();
                 }
-                // [Bt, ld]: through this warp's scratch tile (row = batch entry, column = feature), so that a lane
-                // stores 8 consecutive features of one batch row (16 bytes)
+                // [Bt, ld]: the same way with row = batch entry, column = feature, so that a lane stores 8 consecutive
+                // features of one batch row (16 bytes)
                 {
-                    __nv_bfloat16 *sT = reinterpret_cast<__nv_bfloat16 *>(epi_scratch + (warp - 2) * UM_EPI_SCRATCH);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) sT[j * UM_EPI_PITCH + lane] = __float2bfloat16_rn(v[j]);
                     __syncwarp();
