@@ -369,7 +369,6 @@ umma_pair_gemm_kernel(const __grid_constant__ UpMaps maps, const __grid_constant
                 }
                 uint32_t r[32];
                 tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BNB + c * 32), r);
-                tc_wait_ld();
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);

@@ -229,7 +229,6 @@ umma_tf32x3_kernel(const __grid_constant__ CUtensorMap tmAhi, const __grid_const
                 for (int cc = 0; cc < CPW; ++cc) {
                     uint32_t r[32];
                     tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * 128 + (half * CPW + cc) * 32), r);
-                    tc_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) sum[cc][j] += __uint_as_float(r[j]);
                 }

@@ -87,7 +87,8 @@ constexpr int WU_CHUNK_ROWS_MOM = WuMomentum::CHUNK_ROWS;      // ... of the map
 template <int N> __device__ __forceinline__ void tc_ld_cols(uint32_t taddr, uint32_t (&r)[N]);
 template <> __device__ __forceinline__ void tc_ld_cols<4>(uint32_t taddr, uint32_t (&r)[4]) { tc_ld_32x4(taddr, r); }
 template <> __device__ __forceinline__ void tc_ld_cols<8>(uint32_t taddr, uint32_t (&r)[8]) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n\t"
+                 "tcgen05.wait::ld.sync.aligned;"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(taddr) : "memory");
 }
@@ -202,7 +203,7 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
     auto take_tile = [&](int &slot, uint32_t &ph) -> int {
         if (!mbar_wait(bar_qfull + 8 * slot, ph, abort_flag)) return -2;
         const int t = tile_ids[slot];
-        mbar_arrive(bar_qempty + 8 * slot);
+        if (t >= -1) mbar_arrive(bar_qempty + 8 * slot);      // always true: the arrive waits for the index to have been read
         if (++slot == WU_TILE_SLOTS) { slot = 0; ph ^= 1u; }
         return t;
     };
@@ -323,8 +324,8 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
             // every lane waits for the tile index and reads it; lane 0 hands the slot back for the warp
             if (!__all_sync(0xffffffffu, mbar_wait(bar_qfull + 8 * qslot, qphase, abort_flag))) break;
             const int t = tile_ids[qslot];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_qempty + 8 * qslot);
+            // (the vote uses the index every lane has read: no lane's load of it is still on its way at the arrive)
+            if (__all_sync(0xffffffffu, t >= -1) && lane == 0) mbar_arrive(bar_qempty + 8 * qslot);
             if (++qslot == WU_TILE_SLOTS) { qslot = 0; qphase ^= 1u; }
             if (t < 0) break;
             int l, g, m0, n0; coords(t, l, g, m0, n0);
@@ -383,45 +384,54 @@ umma_wgrad_update_kernel(const __grid_constant__ WuMaps maps, const __grid_const
                     uint32_t r[RPG];
                     tc_ld_cols<RPG>(tmem_base + ((uint32_t)(q * 32) << 16) +
                                     (uint32_t)(acc * UM_BN + c * WU_CHUNK_ROWS + grp * RPG), r);
-                    tc_wait_ld();
-                    // the values are in registers: hand the stage back to the loader
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
-                    if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
-                    const int rows = m_ok ? (N - nb) : 0;        // rows of this thread that exist
-                    auto update_row = [&](int j) {
-                        const long long o = (long long)j * ldv;
+                    // Eq. (parle_y) and (parle_z) for the RPG rows of this thread, in registers.  Rows past the end of
+                    // the layer hold whatever the box was filled with; they are computed and never stored.
+                    float yn[RPG], zn[RPG];
+#pragma unroll
+                    for (int j = 0; j < RPG; ++j) {
                         const float yo = FIRST ? xv[j] : yv[j], zo = FIRST ? xv[j] : (USE_Z ? zv[j] : 0.f);
                         float d = fmaf(p.inv_gamma, yo - xv[j], HAS_WD ? fmaf(p.wd, yo, __uint_as_float(r[j])) : __uint_as_float(r[j]));
                         if (MOM) {
                             const float vn = FIRST ? d : fmaf(p.mu, vv[j], d);      // v = 0 before the first step of a round
-                            vp[o] = vn;
+                            vv[j] = vn;
                             d = fmaf(p.mu, vn, d);
                         }
-                        const float yn = fmaf(neg_eta_p, d, yo);
-                        if (USE_Z) chk = fmaf(yn, 0.f, chk);     // steps that skip z skip the check: the next step sees the same y
+                        yn[j] = fmaf(neg_eta_p, d, yo);
+                        zn[j] = !USE_Z ? 0.f
+                              : (!FIRST && ZMODE == WU_Z_DOUBLE) ? fmaf(alpha_sq, zo, one_m_alpha * fmaf(p.alpha, yo, yn[j]))
+                                                                 : fmaf(p.alpha, zo, one_m_alpha * yn[j]);
+                    }
+                    const int rows = m_ok ? (N - nb) : 0;        // rows of this thread that exist
+                    auto store_row = [&](int j) {
+                        const long long o = (long long)j * ldv;
+                        if (MOM) vp[o] = vv[j];
+                        if (USE_Z) chk = fmaf(yn[j], 0.f, chk);  // steps that skip z skip the check: the next step sees the same y
                         if (YSPLIT) {
-                            const uint32_t w = bf16_split_word(yn);
+                            const uint32_t w = bf16_split_word(yn[j]);
                             lp[o] = (uint16_t)w;                 // lower half; the upper half is the operand copy below
-                            if (YWRITE) yp[o] = yn;
+                            if (YWRITE) yp[o] = yn[j];
                         } else {
-                            yp[o] = yn;
+                            yp[o] = yn[j];
                         }
-                        if (USE_Z) {
-                            const float zn = (!FIRST && ZMODE == WU_Z_DOUBLE) ? fmaf(alpha_sq, zo, one_m_alpha * fmaf(p.alpha, yo, yn))
-                                                                               : fmaf(p.alpha, zo, one_m_alpha * yn);
-                            zp[o] = zn;
-                        }
-                        sp[j * 64] = bf16_weight(yn);
+                        if (USE_Z) zp[o] = zn[j];
+                        sp[j * 64] = bf16_weight(yn[j]);
                     };
                     if (rows >= RPG) {                           // common case: no per-row bounds checks
 #pragma unroll
-                        for (int j = 0; j < RPG; ++j) update_row(j);
+                        for (int j = 0; j < RPG; ++j) store_row(j);
                     } else {
 #pragma unroll
                         for (int j = 0; j < RPG; ++j)
-                            if (j < rows) update_row(j);
+                            if (j < rows) store_row(j);
                     }
+                    // Only now is the stage handed back to the loader.  A shared-memory load that has merely been issued does
+                    // not hold back an arrive, and arithmetic on its result may be scheduled after one: with the arrive placed
+                    // right after the loads, and the load/store unit kept busy by another kernel's CTAs on the same SM, the
+                    // loader's next copy was seen to land in the stage before such a load had read it.  The stores above use
+                    // every value read from the stage and, being memory operations, stay in front of the arrive.
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sempty + 8 * stage);
+                    if (++stage == WU_STATE_STAGES) { stage = 0; sphase ^= 1u; }
                 }
             };
             if (MOM || p.wd != 0.f) {
