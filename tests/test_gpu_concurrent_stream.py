@@ -55,3 +55,56 @@ def test_fused_update_is_exact_with_a_busy_second_stream_bf16():
                 assert torch.equal(a, b), (rep, name, int((a != b).sum()))
     finally:
         busy.close()
+
+
+@pytest.mark.parametrize("name", ["C3", "C5/2", "C2"])
+def test_rounds_are_reproducible_with_a_busy_second_stream(name):
+    """Whole rounds (graph replay: chained two-CTA GEMMs, loss, fused update with paired z and two-plane y; for the fp32
+    workload the three-product tf32 kernels and the separate update) give the same bits with and without the second stream's
+    kernel resident: no hand-off between warps of any kernel depends on how fast its neighbours run."""
+    pytest.importorskip("cuda.bindings")
+    from _busy_kernel import BusyKernel
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16 << 30:
+        pytest.skip("needs 16 GiB of free device memory")
+    if name == "C3":
+        cfg = si.C3.scaled(name="C3x3", n=3, L=6)
+    elif name == "C5/2":
+        cfg = si.C5.scaled(name="C5/2", n=3, dims=(2048, 4096, 4096, 4096, 1000), L=5)
+    else:
+        cfg = si.C2.scaled(name="C2x4", n=4, L=6)
+    X, c = si.round_batches(cfg, 0)
+    Xd, cd = torch.from_numpy(X).to(DEV), torch.from_numpy(c).to(DEV)
+
+    def rounds(busy):
+        m = pb.Parle(cfg.n, cfg.dims, cfg.batch, cfg.gemm_dtype, eta=cfg.eta, eta_prime=cfg.eta_prime, alpha=cfg.alpha,
+                     gamma=cfg.gamma, rho=cfg.rho).alloc(DEV)
+        gen = torch.Generator(device=DEV).manual_seed(3)
+        for a in range(cfg.n):
+            for l in range(cfg.n_layers):
+                w_off, _ = m.layer_offset(l)
+                m.x[a, w_off:w_off + cfg.dims[l] * cfg.dims[l + 1]].normal_(0.0, cfg.dims[l] ** -0.5, generator=gen)
+        m.mean()
+        m.set_round_graphs(True)
+        loss = torch.zeros(cfg.L, cfg.n, device=DEV)
+        torch.cuda.synchronize()
+        for r in range(3):
+            if busy is not None:
+                busy.launch(times=32)
+            m.round(cfg.L, Xd, cd, loss)
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        out = (m.x.clone(), m.xbar.clone(), m.y.clone(), m.z.clone(), loss.clone())
+        del m
+        torch.cuda.empty_cache()
+        return out
+
+    want = rounds(None)
+    busy = BusyKernel(DEV)
+    try:
+        for rep in range(2):
+            got = rounds(busy)
+            for nm, a, b in zip(("x", "xbar", "y", "z", "loss"), want, got):
+                assert torch.equal(a, b), (rep, nm, int((a != b).sum()))
+    finally:
+        busy.close()
