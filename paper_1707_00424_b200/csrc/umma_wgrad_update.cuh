@@ -79,7 +79,7 @@ struct WuShape {
     static_assert(stages(NA) >= 2 && 8 * (2 * WU_OP_STAGES + 4 + 2 * MAX_STAGES + 2 * WU_TILE_SLOTS) + 8 + 4 * WU_TILE_SLOTS <= WU_CTL_BYTES,
                   "stage count");
 };
-using WuDefault = WuShape<4, 32>;
+using WuDefault = WuShape<2, 32>;
 using WuMomentum = WuShape<4, 16, 4>;                          // with the momentum buffer staged too: 16-row chunks
 constexpr int WU_CHUNK_ROWS = WuDefault::CHUNK_ROWS;           // TMA box height of the x/y/z tensor maps
 constexpr int WU_CHUNK_ROWS_MOM = WuMomentum::CHUNK_ROWS;      // ... of the maps used by the momentum variant
