@@ -743,10 +743,6 @@ int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labe
         p.M = din; p.N = dout; p.K = B;
         p.outf = c->buf.grad + c->layers[l].w_off; p.outf_gs = S; p.outf_ld = din;
         PARLE_TRY(launch_t3<T3_WGRAD>(c, KC_WGRAD_GEMM, c->t3_bn_wg[l], c->t3_wa[l], c->t3_wb[l], p));
-        prof_begin(c, KC_BIAS_GRAD);
-        bias_grad_split_kernel<<<dim3((dout + 7) / 8, n), 256, 0, c->stream>>>(
-            ws_ptr<float>(c, w.dhT[l][0]), ws_ptr<float>(c, w.dhT[l][1]), c->buf.grad + c->layers[l].b_off, S, B, dout);
-        PARLE_LAUNCHED(c);
         if (l > 0) {                                            // dH_{l-1} = (dH_l W_l) * 1[H_{l-1} > 0]
             T3Params d = {};
             d.M = B; d.N = din; d.K = dout;
@@ -758,6 +754,18 @@ int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labe
             d.mask_gs = (long long)B * din; d.mask_ld = B;
             PARLE_TRY(launch_t3<T3_DGRAD>(c, KC_DGRAD_GEMM, c->t3_bn_dg[l], c->t3_da[l], c->t3_db[l], d));
         }
+    }
+    {                                                           // bias gradients of all layers: one launch
+        BiasGradPlan bp = {};
+        int dmax = 0;
+        for (int l = 0; l < nl; ++l) {
+            bp.hi[l] = ws_ptr<float>(c, w.dhT[l][0]); bp.lo[l] = ws_ptr<float>(c, w.dhT[l][1]);
+            bp.b_off[l] = (long long)c->layers[l].b_off; bp.d[l] = c->dims[l + 1];
+            if (c->dims[l + 1] > dmax) dmax = c->dims[l + 1];
+        }
+        prof_begin(c, KC_BIAS_GRAD);
+        bias_grad_split_kernel<<<dim3((dmax + 7) / 8, n, nl), 256, 0, c->stream>>>(bp, c->buf.grad, S, B);
+        PARLE_LAUNCHED(c);
     }
     return PARLE_OK;
 }

@@ -401,18 +401,24 @@ split_transpose_kernel(const TransposePlan tp, const float *__restrict__ src, lo
     }
 }
 
-// db[g, j] = sum_i dH^T[g, j, i] from the hi/lo pair [n, d, B]: one warp per row, fixed-order tree.
+// db_l[g, j] = sum_i dH_l^T[g, j, i] from the hi/lo pairs [n, d_l, B] of all layers in one launch (blockIdx.z = layer):
+// one warp per row, fixed-order tree.
+struct BiasGradPlan {
+    const float *hi[PARLE_MAX_LAYERS], *lo[PARLE_MAX_LAYERS];
+    long long b_off[PARLE_MAX_LAYERS];              // offset of the layer's biases inside a replica's gradient
+    int d[PARLE_MAX_LAYERS];
+};
 __global__ void __launch_bounds__(256)
-bias_grad_split_kernel(const float *__restrict__ dThi, const float *__restrict__ dTlo, float *__restrict__ grad,
-                       long long grad_gs, int B, int d) {
+bias_grad_split_kernel(const __grid_constant__ BiasGradPlan bp, float *__restrict__ grad, long long grad_gs, int B) {
+    const int l = blockIdx.z, d = bp.d[l];
     const int j = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
     const int g = blockIdx.y;
     if (j >= d) return;
-    const float *ph = dThi + ((size_t)g * d + j) * B, *pl = dTlo + ((size_t)g * d + j) * B;
+    const float *ph = bp.hi[l] + ((size_t)g * d + j) * B, *pl = bp.lo[l] + ((size_t)g * d + j) * B;
     float s = 0.f;
     for (int i = lane; i < B; i += 32) s += ph[i] + pl[i];
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) grad[(long long)g * grad_gs + j] = s;
+    if (lane == 0) grad[(long long)g * grad_gs + bp.b_off[l] + j] = s;
 }
 
 }  // namespace parle
