@@ -238,6 +238,10 @@ __global__ void __launch_bounds__((BM / 8) * (BN / 8)) simt_gemm_tiled_kernel(Si
 // finished rows of replica g, and the warp that finishes the last one adds up the replica's row losses -- in the
 // same fixed order whoever does it (256 strided partial sums, then a binary tree), so the result does not depend on which
 // warp that is -- and puts the counter back to zero.
+// TR = 16 (bf16 copies only; B % 16 == 0; dynamic shared memory of 16 * C bf16): a block takes 16 consecutive rows, two per
+// warp, keeps their bf16 dlogits in shared memory and writes the transposed copy dbfT from there, 32 bytes (16 rows of one
+// class) per store instead of one 2-byte element per lane.  Same arithmetic, same values.
+template <int TR = 0>
 __global__ void __launch_bounds__(256)
 softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict__ labels,
                            float *__restrict__ d32, __nv_bfloat16 *__restrict__ dbf,
@@ -247,91 +251,110 @@ softmax_ce_backward_kernel(float *__restrict__ logits, const int32_t *__restrict
                            long long bias_gs = 0, float *__restrict__ dThi = nullptr, float *__restrict__ dTlo = nullptr,
                            float *__restrict__ dhi = nullptr, float *__restrict__ dlo = nullptr, int ld_split = 0,
                            float *__restrict__ loss = nullptr, int *__restrict__ rows_done = nullptr) {
-    const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    extern __shared__ __align__(16) unsigned char sce_tile_raw[];
+    __nv_bfloat16 *tile = reinterpret_cast<__nv_bfloat16 *>(sce_tile_raw);      // TR > 0: [TR][C]
     const int lane = threadIdx.x % 32;
-    if (row >= rows) return;
-    float *lg = logits + (size_t)row * C;
-    const int label = labels[row];
-    const bool label_ok = (label >= 0 && label < C);
-    const float inv_B = 1.f / (float)B;
-    const int g = row / B, i = row % B;
-    const float *bg = parts > 1 ? bias + (long long)g * bias_gs : nullptr;
-    // logit j of this row: with split-K partial sums, bias + sum_s part_s in fixed order (all loads in flight first)
-    auto logit = [&](int j) -> float {
-        if (parts <= 1) return lg[j];
-        float pv[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) pv[q] = (q < parts) ? lg[(long long)q * part_stride + j] : 0.f;
-        float s = pv[0];
-#pragma unroll
-        for (int q = 1; q < 8; ++q) s += pv[q];
-        return s + bg[j];
-    };
-    auto emit = [&](int j, float d) {                // d = dlogits[row, j]
-        if (d32) d32[(size_t)row * C + j] = d;
-        if (dbf) {
-            const __nv_bfloat16 h = __float2bfloat16_rn(d);
-            dbf[((size_t)g * B + i) * ld_b + j] = h;
-            dbfT[((size_t)g * C + j) * B + i] = h;
-        }
-        if (dThi) {                                  // tf32-exact hi/lo pair, [B, ld_split] and transposed [C, B] per replica
-            float hi, lo;
-            split_tf32(d, hi, lo);
-            dThi[((size_t)g * C + j) * B + i] = hi;
-            dTlo[((size_t)g * C + j) * B + i] = lo;
-            dhi[(size_t)row * ld_split + j] = hi;
-            dlo[(size_t)row * ld_split + j] = lo;
-        }
-    };
-    constexpr int VR = 4;                            // up to 128 classes: the row stays in registers (one pass over memory)
-    float mx = -INFINITY, s = 0.f, label_logit = 0.f;
-    if (C <= 32 * VR) {
-        float v[VR];
-#pragma unroll
-        for (int k = 0; k < VR; ++k) {
-            const int j = lane + 32 * k;
-            v[k] = j < C ? logit(j) : -INFINITY;
-            if (parts > 1 && j < C) lg[j] = v[k];    // the logits buffer then holds the complete logits
-            mx = fmaxf(mx, v[k]);
-        }
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-#pragma unroll
-        for (int k = 0; k < VR; ++k)
-            if (lane + 32 * k < C) s += __expf(v[k] - mx);
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        const float inv_s = 1.f / s;
-        float cand = 0.f;
-#pragma unroll
-        for (int k = 0; k < VR; ++k) {
-            const int j = lane + 32 * k;
-            if (k == (label >> 5)) cand = v[k];
-            if (j < C) {
-                float d = __expf(v[k] - mx) * inv_s;
+    for (int rr = 0; rr < (TR > 0 ? TR / 8 : 1); ++rr) {
+        const int lr = rr * 8 + threadIdx.x / 32;                                   // row inside the block's tile
+        const int row = TR > 0 ? blockIdx.x * TR + lr : blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+        if (row >= rows) { if (TR > 0) continue; else return; }
+        float *lg = logits + (size_t)row * C;
+        const int label = labels[row];
+        const bool label_ok = (label >= 0 && label < C);
+        const float inv_B = 1.f / (float)B;
+        const int g = row / B, i = row % B;
+        const float *bg = parts > 1 ? bias + (long long)g * bias_gs : nullptr;
+        // logit j of this row: with split-K partial sums, bias + sum_s part_s in fixed order (all loads in flight first)
+        auto logit = [&](int j) -> float {
+            if (parts <= 1) return lg[j];
+            float pv[8];
+    #pragma unroll
+            for (int q = 0; q < 8; ++q) pv[q] = (q < parts) ? lg[(long long)q * part_stride + j] : 0.f;
+            float s = pv[0];
+    #pragma unroll
+            for (int q = 1; q < 8; ++q) s += pv[q];
+            return s + bg[j];
+        };
+        auto emit = [&](int j, float d) {                // d = dlogits[row, j]
+            if (d32) d32[(size_t)row * C + j] = d;
+            if (dbf) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(d);
+                dbf[((size_t)g * B + i) * ld_b + j] = h;
+                if (TR > 0) tile[lr * C + j] = h; else dbfT[((size_t)g * C + j) * B + i] = h;
+            }
+            if (dThi) {                                  // tf32-exact hi/lo pair, [B, ld_split] and transposed [C, B] per replica
+                float hi, lo;
+                split_tf32(d, hi, lo);
+                dThi[((size_t)g * C + j) * B + i] = hi;
+                dTlo[((size_t)g * C + j) * B + i] = lo;
+                dhi[(size_t)row * ld_split + j] = hi;
+                dlo[(size_t)row * ld_split + j] = lo;
+            }
+        };
+        constexpr int VR = 4;                            // up to 128 classes: the row stays in registers (one pass over memory)
+        float mx = -INFINITY, s = 0.f, label_logit = 0.f;
+        if (C <= 32 * VR) {
+            float v[VR];
+    #pragma unroll
+            for (int k = 0; k < VR; ++k) {
+                const int j = lane + 32 * k;
+                v[k] = j < C ? logit(j) : -INFINITY;
+                if (parts > 1 && j < C) lg[j] = v[k];    // the logits buffer then holds the complete logits
+                mx = fmaxf(mx, v[k]);
+            }
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    #pragma unroll
+            for (int k = 0; k < VR; ++k)
+                if (lane + 32 * k < C) s += __expf(v[k] - mx);
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const float inv_s = 1.f / s;
+            float cand = 0.f;
+    #pragma unroll
+            for (int k = 0; k < VR; ++k) {
+                const int j = lane + 32 * k;
+                if (k == (label >> 5)) cand = v[k];
+                if (j < C) {
+                    float d = __expf(v[k] - mx) * inv_s;
+                    if (j == label) d -= 1.f;
+                    emit(j, d * inv_B);
+                }
+            }
+            label_logit = __shfl_sync(0xffffffffu, cand, label & 31);
+        } else {
+            if (parts > 1)
+                for (int j = lane; j < C; j += 32) lg[j] = logit(j);      // read back below by the same lane
+            for (int j = lane; j < C; j += 32) mx = fmaxf(mx, lg[j]);
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            for (int j = lane; j < C; j += 32) s += __expf(lg[j] - mx);
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const float inv_s = 1.f / s;
+            for (int j = lane; j < C; j += 32) {
+                float d = __expf(lg[j] - mx) * inv_s;
                 if (j == label) d -= 1.f;
                 emit(j, d * inv_B);
             }
+            if (lane == 0 && label_ok) label_logit = lg[label];
         }
-        label_logit = __shfl_sync(0xffffffffu, cand, label & 31);
-    } else {
-        if (parts > 1)
-            for (int j = lane; j < C; j += 32) lg[j] = logit(j);      // read back below by the same lane
-        for (int j = lane; j < C; j += 32) mx = fmaxf(mx, lg[j]);
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        for (int j = lane; j < C; j += 32) s += __expf(lg[j] - mx);
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        const float inv_s = 1.f / s;
-        for (int j = lane; j < C; j += 32) {
-            float d = __expf(lg[j] - mx) * inv_s;
-            if (j == label) d -= 1.f;
-            emit(j, d * inv_B);
+        if (lane == 0) {
+            row_loss[row] = label_ok ? (mx + __logf(s) - label_logit) : 0.f;
+            if (!label_ok) status[SLOT_BAD_LABEL] = 1;
         }
-        if (lane == 0 && label_ok) label_logit = lg[label];
+        if (loss) replica_loss_finish(row_loss, loss, rows_done, g, B, 1, lane);
     }
-    if (lane == 0) {
-        row_loss[row] = label_ok ? (mx + __logf(s) - label_logit) : 0.f;
-        if (!label_ok) status[SLOT_BAD_LABEL] = 1;
+    if (TR > 0) {
+        __syncthreads();
+        const long long r0 = (long long)blockIdx.x * TR;                        // first row of the tile: same replica throughout
+        const int g0 = (int)(r0 / B), i0 = (int)(r0 % B);
+        for (int j = threadIdx.x; j < C; j += blockDim.x) {
+            uint4 v[TR > 0 ? TR / 8 : 1];
+            __nv_bfloat16 *e = reinterpret_cast<__nv_bfloat16 *>(v);
+#pragma unroll
+            for (int r = 0; r < TR; ++r) e[r] = tile[r * C + j];
+            uint4 *dst = reinterpret_cast<uint4 *>(dbfT + ((size_t)g0 * C + j) * B + i0);
+#pragma unroll
+            for (int q = 0; q < TR / 8; ++q) dst[q] = v[q];
+        }
     }
-    if (loss) replica_loss_finish(row_loss, loss, rows_done, g, B, 1, lane);
 }
 
 // db[g, j] = sum_i dH[g, i, j] from fp32 dH [n, B, d] (thread per column).

@@ -730,7 +730,7 @@ int forward_backward_tf32(parle_ctx *c, const float *inputs, const int32_t *labe
     }
     const int C = c->dims[nl], rows = n * B;
     prof_begin(c, KC_SOFTMAX_CE);
-    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+    softmax_ce_backward_kernel<0><<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.t3_logits), labels, nullptr, nullptr, nullptr, ws_ptr<float>(c, w.row_loss), rows, B, C, 0,
         c->status_dev, c->t3_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
         ws_ptr<float>(c, w.dhT[nl - 1][0]), ws_ptr<float>(c, w.dhT[nl - 1][1]),
@@ -788,7 +788,7 @@ int forward_backward_fp32(parle_ctx *c, const float *inputs, const int32_t *labe
     }
     const int C = c->dims[nl], rows = n * B;
     prof_begin(c, KC_SOFTMAX_CE);
-    softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+    softmax_ce_backward_kernel<0><<<(rows + 7) / 8, 256, 0, c->stream>>>(
         ws_ptr<float>(c, w.act[nl - 1]), labels, ws_ptr<float>(c, w.dact[nl - 1]), nullptr, nullptr,
         ws_ptr<float>(c, w.row_loss), rows, B, C, 0, c->status_dev, 1, 0, nullptr, 0, nullptr, nullptr, nullptr, nullptr, 0,
         loss_out, ws_ptr<int>(c, w.rows_done));
@@ -866,7 +866,11 @@ int forward_backward_bf16(parle_ctx *c, const float *inputs, const int32_t *labe
     if (!loss_in_epilogue) {
         const int C = c->dims[nl], rows = n * B;
         prof_begin(c, KC_SOFTMAX_CE);
-        softmax_ce_backward_kernel<<<(rows + 7) / 8, 256, 0, c->stream>>>(
+        // batches of a multiple of 16 rows (and rows that fit 48 KB of shared memory 16 at a time): the transposed copy
+        // goes out in whole 32-byte sectors
+        const bool tiled = B % 16 == 0 && (size_t)16 * C * sizeof(__nv_bfloat16) <= 48 * 1024;
+        auto *kern = tiled ? softmax_ce_backward_kernel<16> : softmax_ce_backward_kernel<0>;
+        kern<<<tiled ? rows / 16 : (rows + 7) / 8, 256, tiled ? (size_t)16 * C * sizeof(__nv_bfloat16) : 0, c->stream>>>(
             ws_ptr<float>(c, w.logits), labels, nullptr, ws_ptr<__nv_bfloat16>(c, w.dhb[nl - 1]),
             ws_ptr<__nv_bfloat16>(c, w.dhbT[nl - 1]), ws_ptr<float>(c, w.row_loss), rows, B, C, w.dh_ld[nl - 1],
             c->status_dev, c->last_ksplit, (long long)n * B * C, params + c->layers[nl - 1].b_off, S,
