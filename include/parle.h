@@ -220,8 +220,10 @@ int parle_set_lr(parle_ctx *ctx, double eta, double eta_prime);
 
 /* Tuning knob of the bf16 forward / data-gradient GEMMs: tiles of 128 x 256 instead of 128 x 128 are used
  * when the batch has at least 256 rows and at least `tiles_per_sm` wide tiles fall on every SM (default 4;
- * 0 = whenever the batch allows).  Results do not depend on it beyond fp32 summation order inside a tile
- * (none: the k order is the same). */
+ * 0 = whenever the batch allows), and also where the 128-wide tiling needs more than one pass over the SMs
+ * while the wide one fits in a single, mostly full pass (this second rule is off for values above 1024, which
+ * therefore keep every product on 128-wide tiles).  Results do not depend on it beyond fp32 summation order
+ * inside a tile (none: the k order is the same). */
 int parle_set_wide_tile_threshold(parle_ctx *ctx, int tiles_per_sm);
 
 /* bf16 path, networks with at most 128 classes.  on (the default where the last layer has enough tiles to run without a

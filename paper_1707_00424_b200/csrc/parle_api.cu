@@ -556,12 +556,17 @@ int launch_umma_bn(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMa
 }
 
 // 256-wide tiles where the product is compute-bound and still leaves every SM several tiles
-// (batch of at least 256 rows and four 128 x 256 tiles per SM); 128-wide tiles otherwise.
+// (batch of at least 256 rows and four 128 x 256 tiles per SM), or where they turn two passes over the SMs into
+// one (more 128-wide tiles than SMs, at most one 256-wide tile per SM: a tile then moves 48 instead of 64 KiB into
+// shared memory per 128 x 256 x 64 block of the product); 128-wide tiles otherwise.
 template <int EPI, int BKIND>
 int launch_umma(parle_ctx *c, int cls, const CUtensorMap &a, const CUtensorMap &b, const UmmaParams &p) {
     if (BKIND != UB_ROWMAJOR_K && p.M >= 256) {
-        const long long wide_tiles = (long long)c->n * ((p.M + UM_BM - 1) / UM_BM) * ((p.N + 255) / 256);
-        if (wide_tiles >= (long long)c->wide_tiles_per_sm * c->sm_count) return launch_umma_bn<EPI, BKIND, 256>(c, cls, a, b, p);
+        const long long per_n = (long long)c->n * ((p.M + UM_BM - 1) / UM_BM);
+        const long long wide_tiles = per_n * ((p.N + 255) / 256), narrow_tiles = per_n * ((p.N + 127) / 128);
+        if (wide_tiles >= (long long)c->wide_tiles_per_sm * c->sm_count ||
+            (c->wide_tiles_per_sm <= 1024 && narrow_tiles > c->sm_count && wide_tiles <= c->sm_count && 4 * wide_tiles >= 3 * c->sm_count))
+            return launch_umma_bn<EPI, BKIND, 256>(c, cls, a, b, p);
     }
     return launch_umma_bn<EPI, BKIND, 128>(c, cls, a, b, p);
 }
